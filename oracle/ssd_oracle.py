@@ -1,0 +1,85 @@
+"""ctypes/numpy front end of the C oracle (oracle/ssd_oracle.c). TEST INFRASTRUCTURE ONLY.
+
+Every array is converted to contiguous float64 before the call; the C code holds all of the
+arithmetic (Eq. 1 forward; Algorithm 2 backward along the sequence axis).
+"""
+import ctypes
+
+import numpy as np
+
+from . import build as _build
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(_build.build())
+        dp = ctypes.POINTER(ctypes.c_double)
+        lib.ssd_oracle_fwd.restype = ctypes.c_int
+        lib.ssd_oracle_fwd.argtypes = [ctypes.c_int] * 7 + [dp] * 10
+        lib.ssd_oracle_bwd.restype = ctypes.c_int
+        lib.ssd_oracle_bwd.argtypes = [ctypes.c_int] * 7 + [dp] * 16
+        lib.ssd_oracle_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def threads() -> int:
+    """Number of host threads the oracle's (batch, head) loops use."""
+    return int(_load().ssd_oracle_threads())
+
+
+def _f64(a):
+    return None if a is None else np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+
+
+def _p(a):
+    dp = ctypes.POINTER(ctypes.c_double)
+    return ctypes.cast(None, dp) if a is None else a.ctypes.data_as(dp)
+
+
+def _dims(x, Bm):
+    B, L, H, P = x.shape
+    G, N = Bm.shape[2], Bm.shape[3]
+    return B, L, H, P, N, G
+
+
+def ssd_fwd(x, dt, A, Bm, Cm, D, h0=None, seg=0):
+    """Eq. 1, one step at a time. Returns (y, h_final, boundary) with boundary[:,k] the state
+    entering segment k (None when seg == 0)."""
+    x, dt, A, Bm, Cm, D, h0 = map(_f64, (x, dt, A, Bm, Cm, D, h0))
+    B, L, H, P, N, G = _dims(x, Bm)
+    assert dt.shape == (B, L, H) and A.shape == (H,) and D.shape == (H,)
+    assert Bm.shape == (B, L, G, N) and Cm.shape == (B, L, G, N)
+    assert h0 is None or h0.shape == (B, H, P, N)
+    y = np.empty((B, L, H, P))
+    hf = np.empty((B, H, P, N))
+    bd = None
+    if seg > 0:
+        bd = np.empty((B, (L + seg - 1) // seg, H, P, N))
+    rc = _load().ssd_oracle_fwd(B, L, H, P, N, G, int(seg), _p(x), _p(dt), _p(A), _p(Bm), _p(Cm),
+                                _p(D), _p(h0), _p(y), _p(hf), _p(bd))
+    if rc != 0:
+        raise RuntimeError("ssd_oracle_fwd failed: %d" % rc)
+    return y, hf, bd
+
+
+def ssd_bwd(x, dt, A, Bm, Cm, D, h0, dy, dh_final=None, blk=256):
+    """Reverse-mode derivative of ssd_fwd for Loss = <y,dy> + <h_final,dh_final>, walking blocks of
+    `blk` steps in reverse with recompute from the block-entry state (Algorithm 2).
+    Returns dict(dx, ddt, dA, dB, dC, dD, dh0)."""
+    x, dt, A, Bm, Cm, D, h0, dy, dh_final = map(_f64, (x, dt, A, Bm, Cm, D, h0, dy, dh_final))
+    B, L, H, P, N, G = _dims(x, Bm)
+    assert dy.shape == x.shape
+    out = dict(dx=np.empty_like(x), ddt=np.empty((B, L, H)), dA=np.empty(H),
+               dB=np.empty((B, L, G, N)), dC=np.empty((B, L, G, N)), dD=np.empty(H),
+               dh0=np.empty((B, H, P, N)))
+    rc = _load().ssd_oracle_bwd(B, L, H, P, N, G, int(blk), _p(x), _p(dt), _p(A), _p(Bm), _p(Cm),
+                                _p(D), _p(h0), _p(dy), _p(dh_final), _p(out["dx"]), _p(out["ddt"]),
+                                _p(out["dA"]), _p(out["dB"]), _p(out["dC"]), _p(out["dD"]),
+                                _p(out["dh0"]))
+    if rc != 0:
+        raise RuntimeError("ssd_oracle_bwd failed: %d" % rc)
+    return out
