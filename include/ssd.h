@@ -1,0 +1,147 @@
+/*
+ * libssd — the Mamba-2 SSD selective-scan layer, forward and backward, under the sequence-axis
+ * half of Multi-Axis Gradient Checkpointing (MA-GC), for NVIDIA B200 (sm_100a).
+ *
+ * The layer is the recurrence of Eq. 1 of the paper in the form Mamba-2 uses it (one scalar decay
+ * per head, the input scaled by the step size, a skip term):
+ *
+ *     h_t = exp(dt_t * A_h) * h_{t-1} + dt_t * x_t B_t^T        h_t in R^{P x N}
+ *     y_t = C_t h_t + D_h * x_t
+ *
+ * per batch b and head h; head h uses the B/C vectors of group g = h / (H/G).
+ *
+ * Conventions common to every call
+ *  - All tensor pointers are DEVICE pointers owned by the caller.  The library allocates nothing,
+ *    frees nothing and never synchronises; work is enqueued on `stream` (a cudaStream_t passed as
+ *    void*, NULL = the legacy default stream).  `shape` is a HOST pointer, read before return.
+ *  - Row-major, innermost dimension contiguous:
+ *      x, y, dy, dx        [B, L, H, P]   I/O dtype (fp32 or bf16), batch stride x_bstride
+ *      dt, ddt             [B, L, H]      fp32, batch stride dt_bstride
+ *      Bm, Cm, dB, dC      [B, L, G, N]   I/O dtype, batch stride bc_bstride
+ *      A, D, dA, dD        [H]            fp32
+ *      h0, h_final, dh_final, dh0  [B, H, P, N]  fp32, dense
+ *      boundary            [B, nseg, H, P, N]    fp32, dense, nseg = ceil(L / seg);
+ *                          boundary[:,k] is the state ENTERING segment k (boundary[:,0] = h0).
+ *    Batch strides are in elements; 0 means dense.  They let a caller pass an L-slice of a longer
+ *    tensor.  Outputs use the same strides as the matching inputs (y, dx like x; ddt like dt;
+ *    dB, dC like Bm).
+ *  - Every pointer must be 16-byte aligned and every row (H*P, G*N elements) a multiple of 16 bytes.
+ *  - `ws` is caller-provided scratch of at least ssd_workspace_bytes(shape, op) bytes, 256-byte
+ *    aligned.  Its first word is a status word the kernels set when a bounded device-side wait
+ *    gives up (see ssd_poll_status).  Calls sharing a workspace must not overlap on the GPU.
+ *  - Return value: SSD_OK (0) or a negative SSD_E* code.  On error nothing has been enqueued,
+ *    except SSD_ECUDA, which reports a failed launch part-way (ssd_last_cuda_error() gives the
+ *    CUDA code).
+ *  - Deterministic: the same inputs give the same bits run to run, and the gradients of
+ *    ssd_bwd_segmented do not depend on `seg` (seg == L is the unsegmented backward).
+ *  - Gradient outputs are overwritten, not accumulated into.
+ */
+#ifndef SSD_H_
+#define SSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SSD_VERSION 100
+
+enum { SSD_DTYPE_F32 = 0, SSD_DTYPE_BF16 = 1 };
+
+/* shape.flags */
+enum {
+    SSD_FLAG_FORCE_SIMT = 1 /* bf16 I/O: use the CUDA-core kernels instead of the tensor-core ones */
+};
+
+/* `op` of ssd_workspace_bytes */
+enum { SSD_OP_FWD = 0, SSD_OP_FWD_SEG = 1, SSD_OP_BWD_SEG = 2 };
+
+enum {
+    SSD_OK = 0,
+    SSD_EINVAL = -1,       /* null pointer, non-positive size, H % G, L % chunk, seg % chunk      */
+    SSD_EUNSUPPORTED = -2, /* P != 64, N not in {64,128}, chunk not in {64,128,256}, bad dtype    */
+    SSD_EALIGN = -3,       /* pointer or stride not 16-byte aligned                               */
+    SSD_EWORKSPACE = -4,   /* ws too small or misaligned                                          */
+    SSD_EDEVICE = -5,      /* current device is not compute capability 10.x                       */
+    SSD_ECUDA = -6,        /* a CUDA call failed; see ssd_last_cuda_error()                       */
+    SSD_ETIMEOUT = -7      /* a bounded device-side wait expired (reported by ssd_poll_status)    */
+};
+
+/*
+ * Problem description.  `chunk` is the block length of the chunked scan (the paper keeps the
+ * sequence-axis checkpoint interval a multiple of 256 for it, Section 4.1 "Memory-Efficient Setup");
+ * `seg` is that checkpoint interval s of Algorithms 1 and 2, in tokens, a multiple of `chunk`.
+ * The last segment may be shorter (L % seg != 0 is allowed); L % chunk must be 0.
+ */
+typedef struct ssd_shape {
+    int32_t B, L, H, P, N, G;
+    int32_t chunk;
+    int32_t seg;   /* 0 means L (one segment) */
+    int32_t dtype; /* SSD_DTYPE_* : type of x, Bm, Cm, y, dy, dx, dB, dC */
+    int32_t flags; /* SSD_FLAG_* */
+    int64_t x_bstride, dt_bstride, bc_bstride; /* elements; 0 => dense */
+} ssd_shape_t;
+
+/* Bytes of scratch `ws` that `op` needs for this shape (0 on an invalid shape).  Grows with
+ * seg/chunk (the per-segment chunk states: the "grid cell" term of Eq. 4), not with L, apart from
+ * 8 bytes per (batch, head, chunk) of dA/dD partial sums in the backward. */
+size_t ssd_workspace_bytes(const ssd_shape_t *shape, int op);
+
+/* Bytes of the `boundary` buffer: B * ceil(L/seg) * H * P * N * 4 (the S_ckpt of Algorithm 1). */
+size_t ssd_boundary_bytes(const ssd_shape_t *shape);
+
+/*
+ * Forward of Eq. 1 over the whole sequence.  h0 == NULL means a zero initial state; h_final may be
+ * NULL.  The sequence is processed `seg` tokens at a time (scratch is sized by seg), which does not
+ * change any output bit.
+ */
+int ssd_fwd(const ssd_shape_t *shape, const void *x, const float *dt, const float *A,
+            const void *Bm, const void *Cm, const float *D, const float *h0,
+            void *y, float *h_final, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Forward with sequence-axis checkpoints (Algorithm 1, one layer): as ssd_fwd, and in addition
+ * stores the state entering each segment of `seg` tokens into `boundary` (required, written in
+ * full, boundary[:,0] = h0 or zeros).
+ */
+int ssd_fwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, const float *A,
+                      const void *Bm, const void *Cm, const float *D, const float *h0,
+                      void *y, float *h_final, float *boundary,
+                      void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Backward with grid-cell restoration along the sequence axis (Algorithm 2, one layer):
+ * walks the segments right to left; for each, recomputes the chunk states from boundary[:,k]
+ * (Recompute_Forward), back-propagates through the segment (Backward) and hands the state
+ * gradient to the segment on its left.  For Loss = <y, dy> + <h_final, dh_final> it writes
+ * dx, ddt, dA, dB, dC, dD and (if non-NULL) dh0.  dh_final == NULL means zero (the nabla_state
+ * input of Algorithm 2).  `boundary` must come from ssd_fwd_segmented with the same shape.
+ */
+int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, const float *A,
+                      const void *Bm, const void *Cm, const float *D, const float *boundary,
+                      const void *dy, const float *dh_final,
+                      void *dx, float *ddt, float *dA, void *dB, void *dC, float *dD,
+                      float *dh0, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Reads the status word at the start of `ws` (device memory) with a blocking copy: call it after
+ * synchronising the stream.  Returns SSD_OK, SSD_ETIMEOUT if some kernel abandoned a bounded wait
+ * (its outputs are then undefined), or SSD_ECUDA if the copy failed.
+ */
+int ssd_poll_status(void *ws);
+
+/* Text for an SSD_* code (static storage). */
+const char *ssd_strerror(int code);
+
+/* SSD_VERSION the library was built from. */
+int ssd_version(void);
+
+/* The cudaError_t of the most recent failed CUDA call made by this library on this thread. */
+int ssd_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SSD_H_ */

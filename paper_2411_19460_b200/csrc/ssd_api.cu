@@ -1,0 +1,298 @@
+// Host side of libssd: argument validation, workspace layout, and the segment driver that runs
+// Algorithm 1 (forward, storing the state at every segment boundary) and Algorithm 2 (backward,
+// segments right to left: recompute from the stored state, back-propagate, hand dh to the left)
+// for one SSD layer.  Checkpoint memory is set by the segment length: the scratch holds the chunk
+// states of ONE segment, the boundary buffer one state per segment.
+#include <cstdio>
+#include <cstring>
+
+#include "ssd_internal.h"
+
+namespace ssd {
+
+static thread_local int g_last_cuda = 0;
+
+struct Layout {
+    size_t status, cs, dtT, Hst, Hbf, hcarry, Gst, Gbf, gcarry, ghdot, ddt_dir, rho, pB, pC, dAp, dDp;
+    size_t total;
+};
+
+struct Plan {
+    int B, L, H, P, N, G, Q, seg, nseg, ncs, nct, hpg, nsl, dtype;
+    bool use_tc;
+    int64_t x_bs, dt_bs, bc_bs;
+    size_t esz;
+};
+
+static int make_plan(const ssd_shape_t *s, Plan &pl) {
+    if (!s) return SSD_EINVAL;
+    if (s->B <= 0 || s->L <= 0 || s->H <= 0 || s->P <= 0 || s->N <= 0 || s->G <= 0 || s->chunk <= 0 ||
+        s->seg < 0)
+        return SSD_EINVAL;
+    if (s->H % s->G) return SSD_EINVAL;
+    if (s->dtype != SSD_DTYPE_F32 && s->dtype != SSD_DTYPE_BF16) return SSD_EUNSUPPORTED;
+    if (s->P != 64) return SSD_EUNSUPPORTED;
+    if (s->N != 64 && s->N != 128) return SSD_EUNSUPPORTED;
+    if (s->chunk != 64 && s->chunk != 128 && s->chunk != 256) return SSD_EUNSUPPORTED;
+    if (s->L % s->chunk) return SSD_EINVAL;
+    const int seg = s->seg == 0 ? s->L : (s->seg > s->L ? s->L : s->seg);
+    if (seg % s->chunk) return SSD_EINVAL;
+    if (s->x_bstride < 0 || s->dt_bstride < 0 || s->bc_bstride < 0) return SSD_EINVAL;
+    pl.B = s->B; pl.L = s->L; pl.H = s->H; pl.P = s->P; pl.N = s->N; pl.G = s->G; pl.Q = s->chunk;
+    pl.seg = seg;
+    pl.nseg = (s->L + seg - 1) / seg;
+    pl.ncs = seg / s->chunk;
+    pl.nct = s->L / s->chunk;
+    pl.hpg = s->H / s->G;
+    pl.dtype = s->dtype;
+    pl.esz = s->dtype == SSD_DTYPE_BF16 ? 2 : 4;
+    pl.x_bs = s->x_bstride ? s->x_bstride : (int64_t)s->L * s->H * s->P;
+    pl.dt_bs = s->dt_bstride ? s->dt_bstride : (int64_t)s->L * s->H;
+    pl.bc_bs = s->bc_bstride ? s->bc_bstride : (int64_t)s->L * s->G * s->N;
+    if (pl.x_bs < (int64_t)s->L * s->H * s->P || pl.dt_bs < (int64_t)s->L * s->H ||
+        pl.bc_bs < (int64_t)s->L * s->G * s->N)
+        return SSD_EINVAL;
+    if (((size_t)s->H * s->P * pl.esz) % 16 || ((size_t)s->G * s->N * pl.esz) % 16 ||
+        ((size_t)pl.x_bs * pl.esz) % 16 || ((size_t)pl.bc_bs * pl.esz) % 16)
+        return SSD_EALIGN;
+    pl.use_tc = false;  // tensor-core path is selected in ssd_tc.cu once available
+    pl.nsl = pl.hpg;    // CUDA-core path: one head per dB/dC partial slice
+    return SSD_OK;
+}
+
+static void make_layout(const Plan &pl, int op, Layout &lo) {
+    const size_t PN = (size_t)pl.P * pl.N, BH = (size_t)pl.B * pl.H;
+    const size_t vec = BH * pl.ncs * pl.Q * sizeof(float);
+    const size_t st = (size_t)pl.B * (pl.ncs + 1) * pl.H * PN;
+    const bool bwd = (op == SSD_OP_BWD_SEG);
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
+    memset(&lo, 0, sizeof(lo));
+    lo.status = take(256);
+    lo.cs = take(vec);
+    lo.dtT = take(vec);
+    lo.Hst = take(st * sizeof(float));
+    lo.Hbf = take(pl.use_tc ? st * 2 : 0);
+    lo.hcarry = take(BH * PN * sizeof(float));
+    if (bwd) {
+        lo.Gst = take(st * sizeof(float));
+        lo.Gbf = take(pl.use_tc ? st * 2 : 0);
+        lo.gcarry = take(BH * PN * sizeof(float));
+        lo.ghdot = take(BH * pl.ncs * 8 * sizeof(float));
+        lo.ddt_dir = take(vec);
+        lo.rho = take(vec);
+        const size_t part = (size_t)pl.B * pl.seg * pl.G * pl.nsl * pl.N * sizeof(float);
+        lo.pB = take(part);
+        lo.pC = take(part);
+        lo.dAp = take(BH * pl.nct * sizeof(float));
+        lo.dDp = take(BH * pl.nct * 4 * sizeof(float));
+    }
+    lo.total = o;
+}
+
+static bool misaligned(const void *p) { return ((uintptr_t)p & 15u) != 0; }
+
+static int check_device() {
+    static thread_local int cached_dev = -1;
+    static thread_local int cached_ok = 0;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { g_last_cuda = (int)e; return SSD_ECUDA; }
+    if (dev != cached_dev) {
+        int major = 0;
+        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess) { g_last_cuda = (int)e; return SSD_ECUDA; }
+        cached_dev = dev;
+        cached_ok = (major == 10);
+    }
+    return cached_ok ? SSD_OK : SSD_EDEVICE;
+}
+
+#define SSD_TRY(expr)                                   \
+    do {                                                \
+        cudaError_t e__ = (expr);                       \
+        if (e__ != cudaSuccess) {                       \
+            g_last_cuda = (int)e__;                     \
+            return SSD_ECUDA;                           \
+        }                                               \
+    } while (0)
+
+static void fill_params(const Plan &pl, const Layout &lo, void *ws, SegParams &sp) {
+    memset(&sp, 0, sizeof(sp));
+    sp.B = pl.B; sp.L = pl.L; sp.H = pl.H; sp.P = pl.P; sp.N = pl.N; sp.G = pl.G; sp.Q = pl.Q;
+    sp.hpg = pl.hpg; sp.ncs = pl.ncs; sp.nct = pl.nct; sp.nsl = pl.nsl;
+    sp.x_bs = pl.x_bs; sp.dt_bs = pl.dt_bs; sp.bc_bs = pl.bc_bs;
+    char *w = (char *)ws;
+    sp.status = (unsigned int *)(w + lo.status);
+    sp.cs = (float *)(w + lo.cs);
+    sp.dtT = (float *)(w + lo.dtT);
+    sp.Hst = (float *)(w + lo.Hst);
+    sp.Hbf = (__nv_bfloat16 *)(w + lo.Hbf);
+    sp.hcarry = (float *)(w + lo.hcarry);
+    sp.Gst = (float *)(w + lo.Gst);
+    sp.Gbf = (__nv_bfloat16 *)(w + lo.Gbf);
+    sp.gcarry = (float *)(w + lo.gcarry);
+    sp.ghdot = (float *)(w + lo.ghdot);
+    sp.ddt_dir = (float *)(w + lo.ddt_dir);
+    sp.rho = (float *)(w + lo.rho);
+    sp.pB = (float *)(w + lo.pB);
+    sp.pC = (float *)(w + lo.pC);
+    sp.dAp = (float *)(w + lo.dAp);
+    sp.dDp = (float *)(w + lo.dDp);
+}
+
+static void set_segment(const Plan &pl, int k, SegParams &sp) {
+    sp.t0 = k * pl.seg;
+    const int len = (pl.L - sp.t0 < pl.seg) ? pl.L - sp.t0 : pl.seg;
+    sp.nc = len / pl.Q;
+    sp.c0 = sp.t0 / pl.Q;
+}
+
+static int forward_impl(const ssd_shape_t *shape, const void *x, const float *dt, const float *A,
+                        const void *Bm, const void *Cm, const float *D, const float *h0, void *y,
+                        float *h_final, float *boundary, bool need_boundary, void *ws,
+                        size_t ws_bytes, void *stream) {
+    Plan pl;
+    int rc = make_plan(shape, pl);
+    if (rc) return rc;
+    if (!x || !dt || !A || !Bm || !Cm || !D || !y || !ws) return SSD_EINVAL;
+    if (need_boundary && !boundary) return SSD_EINVAL;
+    if (misaligned(x) || misaligned(dt) || misaligned(A) || misaligned(Bm) || misaligned(Cm) ||
+        misaligned(D) || misaligned(y) || (h0 && misaligned(h0)) || (h_final && misaligned(h_final)) ||
+        (boundary && misaligned(boundary)))
+        return SSD_EALIGN;
+    Layout lo;
+    make_layout(pl, need_boundary ? SSD_OP_FWD_SEG : SSD_OP_FWD, lo);
+    if (((uintptr_t)ws & 255u) || ws_bytes < lo.total) return SSD_EWORKSPACE;
+    rc = check_device();
+    if (rc) return rc;
+
+    cudaStream_t st = (cudaStream_t)stream;
+    SegParams sp;
+    fill_params(pl, lo, ws, sp);
+    sp.x = x; sp.dt = dt; sp.A = A; sp.Bm = Bm; sp.Cm = Cm; sp.D = D; sp.y = y;
+    SSD_TRY(cudaMemsetAsync(sp.status, 0, 256, st));
+    const long long PN = (long long)pl.P * pl.N;
+    for (int k = 0; k < pl.nseg; ++k) {
+        set_segment(pl, k, sp);
+        SSD_TRY(launch_chunk_cumsum(sp, st));
+        SSD_TRY(launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
+        const float *init = (k == 0) ? h0 : sp.hcarry;
+        float *bnd = boundary ? boundary + (size_t)k * pl.H * PN : nullptr;
+        SSD_TRY(launch_state_pass_fwd(sp, init, (long long)pl.H * PN, bnd, (long long)pl.nseg * pl.H * PN,
+                                      (k == pl.nseg - 1) ? h_final : nullptr, pl.use_tc, st));
+        SSD_TRY(launch_masked_product_simt(sp, pl.dtype, MP_FWD, st));
+    }
+    return SSD_OK;
+}
+
+}  // namespace ssd
+
+using namespace ssd;
+
+extern "C" {
+
+size_t ssd_workspace_bytes(const ssd_shape_t *shape, int op) {
+    Plan pl;
+    if (make_plan(shape, pl)) return 0;
+    if (op != SSD_OP_FWD && op != SSD_OP_FWD_SEG && op != SSD_OP_BWD_SEG) return 0;
+    Layout lo;
+    make_layout(pl, op, lo);
+    return lo.total;
+}
+
+size_t ssd_boundary_bytes(const ssd_shape_t *shape) {
+    Plan pl;
+    if (make_plan(shape, pl)) return 0;
+    return (size_t)pl.B * pl.nseg * pl.H * pl.P * pl.N * sizeof(float);
+}
+
+int ssd_fwd(const ssd_shape_t *shape, const void *x, const float *dt, const float *A, const void *Bm,
+            const void *Cm, const float *D, const float *h0, void *y, float *h_final, void *ws,
+            size_t ws_bytes, void *stream) {
+    return forward_impl(shape, x, dt, A, Bm, Cm, D, h0, y, h_final, nullptr, false, ws, ws_bytes, stream);
+}
+
+int ssd_fwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, const float *A,
+                      const void *Bm, const void *Cm, const float *D, const float *h0, void *y,
+                      float *h_final, float *boundary, void *ws, size_t ws_bytes, void *stream) {
+    return forward_impl(shape, x, dt, A, Bm, Cm, D, h0, y, h_final, boundary, true, ws, ws_bytes, stream);
+}
+
+int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, const float *A,
+                      const void *Bm, const void *Cm, const float *D, const float *boundary,
+                      const void *dy, const float *dh_final, void *dx, float *ddt, float *dA, void *dB,
+                      void *dC, float *dD, float *dh0, void *ws, size_t ws_bytes, void *stream) {
+    Plan pl;
+    int rc = make_plan(shape, pl);
+    if (rc) return rc;
+    if (!x || !dt || !A || !Bm || !Cm || !D || !boundary || !dy || !dx || !ddt || !dA || !dB || !dC ||
+        !dD || !ws)
+        return SSD_EINVAL;
+    if (misaligned(x) || misaligned(dt) || misaligned(A) || misaligned(Bm) || misaligned(Cm) ||
+        misaligned(D) || misaligned(boundary) || misaligned(dy) || (dh_final && misaligned(dh_final)) ||
+        misaligned(dx) || misaligned(ddt) || misaligned(dA) || misaligned(dB) || misaligned(dC) ||
+        misaligned(dD) || (dh0 && misaligned(dh0)))
+        return SSD_EALIGN;
+    Layout lo;
+    make_layout(pl, SSD_OP_BWD_SEG, lo);
+    if (((uintptr_t)ws & 255u) || ws_bytes < lo.total) return SSD_EWORKSPACE;
+    rc = check_device();
+    if (rc) return rc;
+
+    cudaStream_t st = (cudaStream_t)stream;
+    SegParams sp;
+    fill_params(pl, lo, ws, sp);
+    sp.x = x; sp.dt = dt; sp.A = A; sp.Bm = Bm; sp.Cm = Cm; sp.D = D; sp.dy = dy;
+    sp.dx = dx; sp.ddt = ddt; sp.dB = dB; sp.dC = dC;
+    SSD_TRY(cudaMemsetAsync(sp.status, 0, 256, st));
+    const long long PN = (long long)pl.P * pl.N;
+    for (int k = pl.nseg - 1; k >= 0; --k) {
+        set_segment(pl, k, sp);
+        // Recompute_Forward: chunk-entry states of segment k from the stored boundary state
+        SSD_TRY(launch_chunk_cumsum(sp, st));
+        SSD_TRY(launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
+        SSD_TRY(launch_state_pass_fwd(sp, boundary + (size_t)k * pl.H * PN, (long long)pl.nseg * pl.H * PN,
+                                      nullptr, 0, nullptr, pl.use_tc, st));
+        // Backward through the segment; dh enters from the right, leaves to the left
+        SSD_TRY(launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_DSTATE, st));
+        const float *ginit = (k == pl.nseg - 1) ? dh_final : sp.gcarry;
+        float *gleft = (k == 0 && dh0) ? dh0 : sp.gcarry;
+        SSD_TRY(launch_state_pass_bwd(sp, ginit, gleft, pl.use_tc, st));
+        SSD_TRY(launch_masked_product_simt(sp, pl.dtype, MP_BWD_DX, st));
+        SSD_TRY(launch_masked_product_simt(sp, pl.dtype, MP_DC, st));
+        SSD_TRY(launch_masked_product_simt(sp, pl.dtype, MP_DB, st));
+        SSD_TRY(launch_bwd_finish(sp, st));
+        SSD_TRY(launch_reduce_dbdc(sp, pl.dtype, st));
+    }
+    SSD_TRY(launch_final_dAdD(sp, dA, dD, st));
+    return SSD_OK;
+}
+
+int ssd_poll_status(void *ws) {
+    if (!ws) return SSD_EINVAL;
+    unsigned int word = 0;
+    cudaError_t e = cudaMemcpy(&word, ws, sizeof(word), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { g_last_cuda = (int)e; return SSD_ECUDA; }
+    return word ? SSD_ETIMEOUT : SSD_OK;
+}
+
+const char *ssd_strerror(int code) {
+    switch (code) {
+        case SSD_OK: return "ok";
+        case SSD_EINVAL: return "invalid argument (null pointer, bad size, H % G, L % chunk or seg % chunk)";
+        case SSD_EUNSUPPORTED: return "unsupported shape or dtype (P=64, N in {64,128}, chunk in {64,128,256})";
+        case SSD_EALIGN: return "pointer or stride not 16-byte aligned";
+        case SSD_EWORKSPACE: return "workspace too small or not 256-byte aligned";
+        case SSD_EDEVICE: return "current device is not compute capability 10.x";
+        case SSD_ECUDA: return "CUDA call failed (see ssd_last_cuda_error)";
+        case SSD_ETIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown error";
+    }
+}
+
+int ssd_version(void) { return SSD_VERSION; }
+
+int ssd_last_cuda_error(void) { return g_last_cuda; }
+
+}  // extern "C"

@@ -1,0 +1,68 @@
+// Internal declarations shared by the host driver and the kernel files of libssd.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ssd.h"
+
+namespace ssd {
+
+// Everything one segment's kernels need.  Passed by value to every kernel.
+struct SegParams {
+    int B, L, H, P, N, G, Q;
+    int hpg;       // heads per group
+    int t0;        // first token of the segment
+    int nc;        // chunks in this segment
+    int c0;        // global index of the segment's first chunk
+    int ncs;       // chunk capacity of the workspace (chunks of a full segment)
+    int nct;       // chunks in the whole sequence (L / Q)
+    int nsl;       // head slices per group in the dB/dC partial buffers
+    int64_t x_bs, dt_bs, bc_bs;  // batch strides, elements
+
+    // caller tensors
+    const void *x, *Bm, *Cm, *dy;
+    const float *dt, *A, *D;
+    void *y, *dx, *dB, *dC;
+    float *ddt;
+
+    // workspace regions (all fp32 unless noted)
+    unsigned int *status;  // [0] = error flag of bounded waits
+    float *cs;             // [B,H,ncs,Q]   inclusive cumsum of dt*A inside each chunk
+    float *dtT;            // [B,H,ncs,Q]   dt transposed to head-major
+    float *Hst;            // [B,ncs+1,H,P,N] slot c = state entering chunk c; slot nc = leaving the segment
+    float *Gst;            // [B,ncs+1,H,P,N] slot c+1 = dLoss/d(state leaving chunk c)
+    __nv_bfloat16 *Hbf;    // [B,ncs+1,H,P,N] bf16 copy of Hst (tensor-core path)
+    __nv_bfloat16 *Gbf;    // [B,ncs+1,H,P,N] bf16 copy of Gst (tensor-core path)
+    float *hcarry;         // [B,H,P,N]     state handed from segment to segment (forward)
+    float *gcarry;         // [B,H,P,N]     state gradient handed right-to-left (backward)
+    float *ghdot;          // [B,H,ncs,8]   partial sums of <Gout_c, Hout_c>
+    float *ddt_dir;        // [B,H,ncs,Q]   direct part of ddt
+    float *rho;            // [B,H,ncs,Q]   dy_t . (y_t - D x_t)
+    float *pB, *pC;        // [B,seg,G,nsl,N] per-head-slice partial dB / dC
+    float *dAp;            // [B,H,nct]     per-chunk partial of dA
+    float *dDp;            // [B,H,nct,4]   per-row-tile partial of dD
+};
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ---- kernel launchers (each returns the cudaError_t of its launch) ----
+// ssd_simt.cu : CUDA-core kernels, any I/O dtype
+cudaError_t launch_chunk_cumsum(const SegParams &p, cudaStream_t st);
+cudaError_t launch_chunk_state_simt(const SegParams &p, int dtype, int mode, cudaStream_t st);
+// init: state entering the segment (NULL = zeros), batch stride init_bs elements;
+// boundary_out (nullable): where to store that state, batch stride bnd_bs; final_out nullable.
+cudaError_t launch_state_pass_fwd(const SegParams &p, const float *init, long long init_bs,
+                                  float *boundary_out, long long bnd_bs, float *final_out,
+                                  bool want_bf16, cudaStream_t st);
+cudaError_t launch_state_pass_bwd(const SegParams &p, const float *init, float *left_out,
+                                  bool want_bf16, cudaStream_t st);
+cudaError_t launch_masked_product_simt(const SegParams &p, int dtype, int mode, cudaStream_t st);
+cudaError_t launch_bwd_finish(const SegParams &p, cudaStream_t st);
+cudaError_t launch_reduce_dbdc(const SegParams &p, int dtype, cudaStream_t st);
+cudaError_t launch_final_dAdD(const SegParams &p, float *dA, float *dD, cudaStream_t st);
+
+enum { STATE_MODE_FWD = 0, STATE_MODE_DSTATE = 1 };
+enum { MP_FWD = 0, MP_BWD_DX = 1, MP_DC = 2, MP_DB = 3 };
+
+}  // namespace ssd

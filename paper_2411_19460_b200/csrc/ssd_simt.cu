@@ -1,0 +1,648 @@
+// CUDA-core kernels of libssd: the bandwidth-bound steps (chunk cumsum, inter-chunk state
+// passing, segment-boundary store/reload, the backward's scans and reductions) for every dtype,
+// and FFMA versions of the contractions, which serve the fp32 mode (1e-4 parity rules out
+// reduced-precision tensor-core inputs) and cross-check the tensor-core kernels.
+//
+// Notation per (batch b, head h), chunk of Q steps: a_t = dt_t*A_h, cs_t = inclusive cumsum of a
+// inside the chunk, H_in = state entering the chunk, Gout = dLoss/d(state leaving the chunk).
+// All of it is Eq. 1 of the paper regrouped by chunks; the segment hand-off is Algorithms 1 and 2.
+#include "ssd_internal.h"
+
+namespace ssd {
+
+// ------------------------------------------------------------------ small helpers
+template <typename T> __device__ __forceinline__ float ldf(const T *p);
+template <> __device__ __forceinline__ float ldf<float>(const float *p) { return __ldg(p); }
+template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloat16 *p) {
+    return __bfloat162float(*p);
+}
+template <typename T> __device__ __forceinline__ void stf(T *p, float v);
+template <> __device__ __forceinline__ void stf<float>(float *p, float v) { *p = v; }
+template <> __device__ __forceinline__ void stf<__nv_bfloat16>(__nv_bfloat16 *p, float v) {
+    *p = __float2bfloat16_rn(v);
+}
+
+__device__ __forceinline__ size_t slot_off(const SegParams &p, int b, int slot, int h) {
+    return (((size_t)b * (p.ncs + 1) + slot) * p.H + h) * (size_t)(p.P * p.N);
+}
+__device__ __forceinline__ size_t vec_off(const SegParams &p, int b, int h, int c) {
+    return (((size_t)b * p.H + h) * p.ncs + c) * (size_t)p.Q;
+}
+
+// ------------------------------------------------------------------ a1: chunk cumsum
+// One CTA per (chunk, batch).  dt[b, t, :] rows are staged through shared memory 32 heads at a
+// time so global reads are coalesced; each warp then scans one head: a lane owns Q/32 consecutive
+// steps (serial prefix), lane totals are combined with a warp-shuffle scan.
+__global__ void __launch_bounds__(256) k_chunk_cumsum(SegParams p) {
+    __shared__ float tile[256][33];
+    const int c = blockIdx.x, b = blockIdx.y;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int Q = p.Q, per = Q >> 5;
+    const size_t tok0 = (size_t)p.t0 + (size_t)c * Q;
+    for (int h0 = 0; h0 < p.H; h0 += 32) {
+        const int nh = min(32, p.H - h0);
+        for (int idx = tid; idx < Q * 32; idx += 256) {
+            const int t = idx >> 5, hh = idx & 31;
+            if (hh < nh) tile[t][hh] = __ldg(p.dt + (size_t)b * p.dt_bs + (tok0 + t) * p.H + h0 + hh);
+        }
+        __syncthreads();
+        for (int hh = warp; hh < nh; hh += 8) {
+            const float Ah = __ldg(p.A + h0 + hh);
+            float a[8], d[8];
+            float run = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (j < per) {
+                    d[j] = tile[lane * per + j][hh];
+                    run += d[j] * Ah;
+                    a[j] = run;
+                }
+            float incl = run;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const float v = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += v;
+            }
+            float excl = __shfl_up_sync(0xffffffffu, incl, 1);
+            if (lane == 0) excl = 0.f;
+            const size_t o = vec_off(p, b, h0 + hh, c) + (size_t)lane * per;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (j < per) {
+                    p.cs[o + j] = a[j] + excl;
+                    p.dtT[o + j] = d[j];
+                }
+        }
+        __syncthreads();
+    }
+}
+
+cudaError_t launch_chunk_cumsum(const SegParams &p, cudaStream_t st) {
+    k_chunk_cumsum<<<dim3(p.nc, p.B), 256, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ a2 / a8: chunk state (FFMA)
+// mode FWD   : S_c[p,n] = sum_s exp(cs_last - cs_s) dt_s x_s[p] B_s[n]     -> Hst slot c+1
+// mode DSTATE: E_c[p,n] = sum_t exp(cs_t) dy_t[p] C_t[n]                   -> Gst slot c
+template <typename T, int NS>
+__global__ void __launch_bounds__(256) k_chunk_state_simt(SegParams p, int mode) {
+    __shared__ float xs[32][64];
+    __shared__ float bs[32][NS];
+    __shared__ float wsm[256];
+    const int c = blockIdx.x, h = blockIdx.y, b = blockIdx.z, g = h / p.hpg;
+    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+    const int Q = p.Q;
+    const T *rowsrc = (const T *)(mode == STATE_MODE_FWD ? p.x : p.dy);
+    const T *colsrc = (const T *)(mode == STATE_MODE_FWD ? p.Bm : p.Cm);
+    const size_t tok0 = (size_t)p.t0 + (size_t)c * Q;
+    const float *csb = p.cs + vec_off(p, b, h, c);
+    const float *dtb = p.dtT + vec_off(p, b, h, c);
+    const float cl = csb[Q - 1];
+    for (int t = tid; t < Q; t += 256)
+        wsm[t] = (mode == STATE_MODE_FWD) ? expf(fminf(cl - csb[t], 0.f)) * dtb[t] : expf(csb[t]);
+    __syncthreads();
+    constexpr int NJ = NS / 16;
+    float acc[4][NJ];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) acc[i][j] = 0.f;
+    const size_t HP = (size_t)p.H * 64, GN = (size_t)p.G * NS;
+    for (int s0 = 0; s0 < Q; s0 += 32) {
+        for (int idx = tid; idx < 32 * 64; idx += 256) {
+            const int r = idx >> 6, pp = idx & 63;
+            xs[r][pp] = ldf(rowsrc + (size_t)b * p.x_bs + (tok0 + s0 + r) * HP + (size_t)h * 64 + pp) * wsm[s0 + r];
+        }
+        for (int idx = tid; idx < 32 * NS; idx += 256) {
+            const int r = idx / NS, nn = idx % NS;
+            bs[r][nn] = ldf(colsrc + (size_t)b * p.bc_bs + (tok0 + s0 + r) * GN + (size_t)g * NS + nn);
+        }
+        __syncthreads();
+#pragma unroll 4
+        for (int kk = 0; kk < 32; ++kk) {
+            float xv[4], bv[NJ];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) xv[i] = xs[kk][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) bv[j] = bs[kk][tx + 16 * j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < NJ; ++j) acc[i][j] = fmaf(xv[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    float *out = (mode == STATE_MODE_FWD) ? p.Hst + slot_off(p, b, c + 1, h) : p.Gst + slot_off(p, b, c, h);
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) out[(size_t)(ty * 4 + i) * NS + tx + 16 * j] = acc[i][j];
+}
+
+cudaError_t launch_chunk_state_simt(const SegParams &p, int dtype, int mode, cudaStream_t st) {
+    dim3 grid(p.nc, p.H, p.B);
+    if (dtype == SSD_DTYPE_F32) {
+        if (p.N == 64) k_chunk_state_simt<float, 64><<<grid, 256, 0, st>>>(p, mode);
+        else k_chunk_state_simt<float, 128><<<grid, 256, 0, st>>>(p, mode);
+    } else {
+        if (p.N == 64) k_chunk_state_simt<__nv_bfloat16, 64><<<grid, 256, 0, st>>>(p, mode);
+        else k_chunk_state_simt<__nv_bfloat16, 128><<<grid, 256, 0, st>>>(p, mode);
+    }
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ a3 / a4: forward state passing
+// H_{c+1} = exp(cs_last,c) H_c + S_c, strictly sequential in c for every (b,h,p,n) element, so the
+// bits do not depend on how the sequence is cut into segments.  Each thread owns one float4.
+// Also stores the segment-entry state into `boundary` (the sequence-axis checkpoint) and hands the
+// segment-exit state to the next segment through hcarry.
+__global__ void __launch_bounds__(256)
+k_state_pass_fwd(SegParams p, const float *init, long long init_bs, float *boundary_out,
+                 long long bnd_bs, float *final_out, int want_bf16) {
+    const int h = blockIdx.y, b = blockIdx.z;
+    const int PN = p.P * p.N;
+    const int e = blockIdx.x * 1024 + threadIdx.x * 4;
+    const size_t bh = ((size_t)b * p.H + h) * PN + e;
+    float4 carry = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (init) carry = *reinterpret_cast<const float4 *>(init + (size_t)b * init_bs + (size_t)h * PN + e);
+    if (boundary_out)
+        *reinterpret_cast<float4 *>(boundary_out + (size_t)b * bnd_bs + (size_t)h * PN + e) = carry;
+    const float *csl = p.cs + vec_off(p, b, h, 0) + (p.Q - 1);
+    for (int c = 0; c <= p.nc; ++c) {
+        const size_t so = slot_off(p, b, c, h) + e;
+        if (c > 0) {
+            const float decay = expf(csl[(size_t)(c - 1) * p.Q]);
+            const float4 s = *reinterpret_cast<const float4 *>(p.Hst + so);
+            carry.x = fmaf(decay, carry.x, s.x);
+            carry.y = fmaf(decay, carry.y, s.y);
+            carry.z = fmaf(decay, carry.z, s.z);
+            carry.w = fmaf(decay, carry.w, s.w);
+        }
+        *reinterpret_cast<float4 *>(p.Hst + so) = carry;
+        if (want_bf16) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(carry.x, carry.y);
+            __nv_bfloat162 hi = __floats2bfloat162_rn(carry.z, carry.w);
+            uint2 pk;
+            pk.x = *reinterpret_cast<unsigned int *>(&lo);
+            pk.y = *reinterpret_cast<unsigned int *>(&hi);
+            *reinterpret_cast<uint2 *>(p.Hbf + so) = pk;
+        }
+    }
+    *reinterpret_cast<float4 *>(p.hcarry + bh) = carry;
+    if (final_out) *reinterpret_cast<float4 *>(final_out + bh) = carry;
+}
+
+cudaError_t launch_state_pass_fwd(const SegParams &p, const float *init, long long init_bs,
+                                  float *boundary_out, long long bnd_bs, float *final_out,
+                                  bool want_bf16, cudaStream_t st) {
+    dim3 grid(p.P * p.N / 1024, p.H, p.B);
+    k_state_pass_fwd<<<grid, 256, 0, st>>>(p, init, init_bs, boundary_out, bnd_bs, final_out, want_bf16 ? 1 : 0);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ a9: backward state passing
+// Gslot[nc] = gradient arriving from the segment on the right (or dh_final); going left,
+// Gslot[c] = exp(cs_last,c) Gslot[c+1] + E_c.  Gslot[c+1] is Gout of chunk c.  Also emits, per chunk,
+// the partial sums of <Gout_c, Hout_c> (one per CTA, summed later in a fixed order), which is the
+// value the within-chunk suffix scan of da starts from.
+__global__ void __launch_bounds__(256)
+k_state_pass_bwd(SegParams p, const float *init, float *left_out, int want_bf16) {
+    __shared__ float red[2][8];
+    const int h = blockIdx.y, b = blockIdx.z;
+    const int PN = p.P * p.N;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int e = blockIdx.x * 1024 + tid * 4;
+    const size_t bh = ((size_t)b * p.H + h) * PN + e;
+    float4 carry = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (init) carry = *reinterpret_cast<const float4 *>(init + bh);
+    const float *csl = p.cs + vec_off(p, b, h, 0) + (p.Q - 1);
+    for (int c = p.nc; c >= 0; --c) {
+        const size_t so = slot_off(p, b, c, h) + e;
+        if (c < p.nc) {
+            // carry is Gout of chunk c here (slot c+1); Hst slot c+1 is the state leaving chunk c
+            const float4 hv = *reinterpret_cast<const float4 *>(p.Hst + slot_off(p, b, c + 1, h) + e);
+            float part = carry.x * hv.x;
+            part = fmaf(carry.y, hv.y, part);
+            part = fmaf(carry.z, hv.z, part);
+            part = fmaf(carry.w, hv.w, part);
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+            if (lane == 0) red[c & 1][warp] = part;
+            __syncthreads();
+            if (tid == 0) {
+                float s = 0.f;
+#pragma unroll
+                for (int w = 0; w < 8; ++w) s += red[c & 1][w];
+                p.ghdot[((((size_t)b * p.H + h) * p.ncs + c) << 3) + blockIdx.x] = s;
+            }
+            const float decay = expf(csl[(size_t)c * p.Q]);
+            const float4 ev = *reinterpret_cast<const float4 *>(p.Gst + so);
+            carry.x = fmaf(decay, carry.x, ev.x);
+            carry.y = fmaf(decay, carry.y, ev.y);
+            carry.z = fmaf(decay, carry.z, ev.z);
+            carry.w = fmaf(decay, carry.w, ev.w);
+        }
+        *reinterpret_cast<float4 *>(p.Gst + so) = carry;
+        if (want_bf16) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(carry.x, carry.y);
+            __nv_bfloat162 hi = __floats2bfloat162_rn(carry.z, carry.w);
+            uint2 pk;
+            pk.x = *reinterpret_cast<unsigned int *>(&lo);
+            pk.y = *reinterpret_cast<unsigned int *>(&hi);
+            *reinterpret_cast<uint2 *>(p.Gbf + so) = pk;
+        }
+    }
+    *reinterpret_cast<float4 *>(left_out + bh) = carry;
+}
+
+cudaError_t launch_state_pass_bwd(const SegParams &p, const float *init, float *left_out,
+                                  bool want_bf16, cudaStream_t st) {
+    dim3 grid(p.P * p.N / 1024, p.H, p.B);
+    k_state_pass_bwd<<<grid, 256, 0, st>>>(p, init, left_out, want_bf16 ? 1 : 0);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ a5+a6, a10, a11: masked products (FFMA)
+// One generic "score -> decay mask -> times values (+ inter-chunk term)" kernel, 64x64 tiles:
+//   score[r,c] = <Rv_r, Cv_c>            (length KD)
+//   acc[r,:]  += mask(r,c) * score[r,c] * V_c      (width WD)
+//   acc[r,j]  += offscale_r * <Rv_r, S_j>          S = chunk state, viewed [WD, KD]
+// MP_FWD    rows t: Rv=C, Cv=B, V=x , mask=[s<=t] e^{cs_t-cs_s} dt_s, S=H_in[p][n], off e^{cs_t}
+//           y_t = acc + D x_t
+// MP_BWD_DX rows s: Rv=B, Cv=C, V=dy, mask=[t>=s] e^{cs_t-cs_s},     S=Gout[p][n], off e^{cs_last-cs_s}
+//           dx_s = D dy_s + dt_s acc ; ddt_direct_s = <x_s, acc> ; dD partial = sum dy x
+// MP_DC     rows t: Rv=dy, Cv=x, V=B, mask as MP_FWD,               S=H_in^T[n][p], off e^{cs_t}
+//           per-head dC_t = acc ; rho_t = <C_t, acc>
+// MP_DB     rows s: Rv=x, Cv=dy, V=C, mask=[t>=s] e^{cs_t-cs_s} dt_s, S=Gout^T[n][p], off dt_s e^{cs_last-cs_s}
+//           per-head dB_s = acc
+template <typename T, int NS, int MODE>
+__global__ void __launch_bounds__(256) k_masked_product_simt(SegParams p) {
+    constexpr int KD = (MODE < 2) ? NS : 64;
+    constexpr int WD = (MODE < 2) ? 64 : NS;
+    constexpr int NJ = WD / 16;
+    constexpr int KP = KD + 1;
+    constexpr bool LOWER = (MODE == MP_FWD || MODE == MP_DC);
+    extern __shared__ float sm[];
+    float *Rv = sm;
+    float *Cv = Rv + 64 * KP;
+    float *V = Cv + 64 * KP;
+    float *Mk = V + 64 * WD;
+    float *css = Mk + 64 * 65;
+    float *dts = css + 256;
+
+    const int Q = p.Q, nrt = Q >> 6;
+    const int c = blockIdx.x / nrt, rt = blockIdx.x % nrt;
+    const int h = blockIdx.y, b = blockIdx.z, g = h / p.hpg;
+    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+    const size_t tok0 = (size_t)p.t0 + (size_t)c * Q;
+    const size_t HP = (size_t)p.H * 64, GN = (size_t)p.G * NS;
+    const T *xlike_base_x = (const T *)p.x + (size_t)b * p.x_bs + tok0 * HP + (size_t)h * 64;
+    const T *xlike_base_dy = (const T *)p.dy + (size_t)b * p.x_bs + tok0 * HP + (size_t)h * 64;
+    const T *bc_base_B = (const T *)p.Bm + (size_t)b * p.bc_bs + tok0 * GN + (size_t)g * NS;
+    const T *bc_base_C = (const T *)p.Cm + (size_t)b * p.bc_bs + tok0 * GN + (size_t)g * NS;
+
+    const T *rsrc, *csrc, *vsrc;
+    size_t rstride, vstride;  // rsrc/csrc share a stride
+    if (MODE == MP_FWD) { rsrc = bc_base_C; csrc = bc_base_B; vsrc = xlike_base_x; rstride = GN; vstride = HP; }
+    else if (MODE == MP_BWD_DX) { rsrc = bc_base_B; csrc = bc_base_C; vsrc = xlike_base_dy; rstride = GN; vstride = HP; }
+    else if (MODE == MP_DC) { rsrc = xlike_base_dy; csrc = xlike_base_x; vsrc = bc_base_B; rstride = HP; vstride = GN; }
+    else { rsrc = xlike_base_x; csrc = xlike_base_dy; vsrc = bc_base_C; rstride = HP; vstride = GN; }
+
+    for (int t = tid; t < Q; t += 256) {
+        css[t] = p.cs[vec_off(p, b, h, c) + t];
+        dts[t] = p.dtT[vec_off(p, b, h, c) + t];
+    }
+    const int r0 = rt * 64;
+    for (int idx = tid; idx < 64 * KD; idx += 256) {
+        const int r = idx / KD, k = idx % KD;
+        Rv[r * KP + k] = ldf(rsrc + (size_t)(r0 + r) * rstride + k);
+    }
+    float acc[4][NJ];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) acc[i][j] = 0.f;
+    __syncthreads();
+
+    const float cs_last = css[Q - 1];
+    const int ct_begin = LOWER ? 0 : rt, ct_end = LOWER ? rt : nrt - 1;
+    for (int ct = ct_begin; ct <= ct_end; ++ct) {
+        const int c0 = ct * 64;
+        for (int idx = tid; idx < 64 * KD; idx += 256) {
+            const int r = idx / KD, k = idx % KD;
+            Cv[r * KP + k] = ldf(csrc + (size_t)(c0 + r) * rstride + k);
+        }
+        for (int idx = tid; idx < 64 * WD; idx += 256) {
+            const int r = idx / WD, j = idx % WD;
+            V[r * WD + j] = ldf(vsrc + (size_t)(c0 + r) * vstride + j);
+        }
+        __syncthreads();
+        float s[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) s[i][j] = 0.f;
+#pragma unroll 4
+        for (int k = 0; k < KD; ++k) {
+            float rv[4], cv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) rv[i] = Rv[(ty * 4 + i) * KP + k];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) cv[j] = Cv[(tx + 16 * j) * KP + k];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) s[i][j] = fmaf(rv[i], cv[j], s[i][j]);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int r = r0 + ty * 4 + i, cc = c0 + tx + 16 * j;
+                float m;
+                if (LOWER) m = (cc <= r) ? expf(fminf(css[r] - css[cc], 0.f)) * dts[cc] : 0.f;
+                else if (MODE == MP_BWD_DX) m = (cc >= r) ? expf(fminf(css[cc] - css[r], 0.f)) : 0.f;
+                else m = (cc >= r) ? expf(fminf(css[cc] - css[r], 0.f)) * dts[r] : 0.f;
+                Mk[(ty * 4 + i) * 65 + tx + 16 * j] = s[i][j] * m;
+            }
+        __syncthreads();
+#pragma unroll 4
+        for (int k = 0; k < 64; ++k) {
+            float mv[4], vv[NJ];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) mv[i] = Mk[(ty * 4 + i) * 65 + k];
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) vv[j] = V[k * WD + tx + 16 * j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < NJ; ++j) acc[i][j] = fmaf(mv[i], vv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+
+    // inter-chunk term
+    const float *St = (MODE == MP_FWD || MODE == MP_DC) ? p.Hst + slot_off(p, b, c, h)
+                                                        : p.Gst + slot_off(p, b, c + 1, h);
+    float offs[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int r = r0 + ty * 4 + i;
+        if (MODE == MP_FWD || MODE == MP_DC) offs[i] = expf(css[r]);
+        else if (MODE == MP_BWD_DX) offs[i] = expf(fminf(cs_last - css[r], 0.f));
+        else offs[i] = dts[r] * expf(fminf(cs_last - css[r], 0.f));
+    }
+#pragma unroll
+    for (int q = 0; q < WD / 64; ++q) {
+        if (MODE < 2) {
+            for (int idx = tid; idx < 64 * KD; idx += 256) {
+                const int jl = idx / KD, k = idx % KD;
+                Cv[jl * KP + k] = St[(size_t)(64 * q + jl) * NS + k];
+            }
+        } else {
+            for (int idx = tid; idx < 64 * 64; idx += 256) {
+                const int pp = idx >> 6, jl = idx & 63;
+                Cv[jl * KP + pp] = St[(size_t)pp * NS + 64 * q + jl];
+            }
+        }
+        __syncthreads();
+        float s[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) s[i][j] = 0.f;
+#pragma unroll 4
+        for (int k = 0; k < KD; ++k) {
+            float rv[4], cv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) rv[i] = Rv[(ty * 4 + i) * KP + k];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) cv[j] = Cv[(tx + 16 * j) * KP + k];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) s[i][j] = fmaf(rv[i], cv[j], s[i][j]);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][4 * q + j] = fmaf(offs[i], s[i][j], acc[i][4 * q + j]);
+        __syncthreads();
+    }
+
+    // epilogues
+    if (MODE == MP_FWD) {
+        const float Dh = __ldg(p.D + h);
+        T *yb = (T *)p.y + (size_t)b * p.x_bs + tok0 * HP + (size_t)h * 64;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) {
+                const int r = r0 + ty * 4 + i, pp = tx + 16 * j;
+                const float xv = ldf(xlike_base_x + (size_t)r * HP + pp);
+                stf(yb + (size_t)r * HP + pp, fmaf(Dh, xv, acc[i][j]));
+            }
+    } else if (MODE == MP_BWD_DX) {
+        const float Dh = __ldg(p.D + h);
+        T *dxb = (T *)p.dx + (size_t)b * p.x_bs + tok0 * HP + (size_t)h * 64;
+        float dsum = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = r0 + ty * 4 + i;
+            float dd = 0.f;
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) {
+                const int pp = tx + 16 * j;
+                const float xv = ldf(xlike_base_x + (size_t)r * HP + pp);
+                const float dyv = ldf(xlike_base_dy + (size_t)r * HP + pp);
+                stf(dxb + (size_t)r * HP + pp, fmaf(Dh, dyv, dts[r] * acc[i][j]));
+                dd = fmaf(xv, acc[i][j], dd);
+                dsum = fmaf(dyv, xv, dsum);
+            }
+#pragma unroll
+            for (int off = 8; off > 0; off >>= 1) dd += __shfl_xor_sync(0xffffffffu, dd, off);
+            if (tx == 0) p.ddt_dir[vec_off(p, b, h, c) + r] = dd;
+        }
+        // deterministic block sum of dy*x
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, off);
+        if ((tid & 31) == 0) Mk[tid >> 5] = dsum;
+        __syncthreads();
+        if (tid == 0) {
+            float s = 0.f;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) s += Mk[w];
+            p.dDp[((((size_t)b * p.H + h) * p.nct + p.c0 + c) << 2) + rt] = s;
+        }
+    } else {
+        // per-head partial dC / dB rows: [B, seg, G, nsl, N]
+        float *pb = (MODE == MP_DC) ? p.pC : p.pB;
+        const int sl = (h % p.hpg) / (p.hpg / p.nsl);
+        const size_t segcap = (size_t)p.ncs * Q;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = r0 + ty * 4 + i;
+            const size_t tl = (size_t)c * Q + r;
+            float *row = pb + ((((size_t)b * segcap + tl) * p.G + g) * p.nsl + sl) * NS;
+            float dot = 0.f;
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) {
+                const int nn = tx + 16 * j;
+                row[nn] = acc[i][j];
+                if (MODE == MP_DC) dot = fmaf(ldf(bc_base_C + (size_t)r * GN + nn), acc[i][j], dot);
+            }
+            if (MODE == MP_DC) {
+#pragma unroll
+                for (int off = 8; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+                if (tx == 0) p.rho[vec_off(p, b, h, c) + r] = dot;
+            }
+        }
+    }
+}
+
+template <typename T, int NS, int MODE>
+static cudaError_t launch_mp(const SegParams &p, cudaStream_t st) {
+    constexpr int KD = (MODE < 2) ? NS : 64;
+    constexpr int WD = (MODE < 2) ? 64 : NS;
+    const size_t smem = sizeof(float) * (2 * 64 * (KD + 1) + 64 * WD + 64 * 65 + 512);
+    cudaError_t e = cudaFuncSetAttribute(k_masked_product_simt<T, NS, MODE>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    dim3 grid(p.nc * (p.Q / 64), p.H, p.B);
+    k_masked_product_simt<T, NS, MODE><<<grid, 256, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
+template <typename T, int NS>
+static cudaError_t launch_mp_mode(const SegParams &p, int mode, cudaStream_t st) {
+    switch (mode) {
+        case MP_FWD: return launch_mp<T, NS, MP_FWD>(p, st);
+        case MP_BWD_DX: return launch_mp<T, NS, MP_BWD_DX>(p, st);
+        case MP_DC: return launch_mp<T, NS, MP_DC>(p, st);
+        default: return launch_mp<T, NS, MP_DB>(p, st);
+    }
+}
+
+cudaError_t launch_masked_product_simt(const SegParams &p, int dtype, int mode, cudaStream_t st) {
+    if (dtype == SSD_DTYPE_F32)
+        return p.N == 64 ? launch_mp_mode<float, 64>(p, mode, st) : launch_mp_mode<float, 128>(p, mode, st);
+    return p.N == 64 ? launch_mp_mode<__nv_bfloat16, 64>(p, mode, st)
+                     : launch_mp_mode<__nv_bfloat16, 128>(p, mode, st);
+}
+
+// ------------------------------------------------------------------ a12 + a13: da, ddt, dA partial
+// One warp per (b, h, chunk).  da_t = sum_{t'>=t in chunk} (rho_t' - dt_t' ddt_direct_t') + <Gout,Hout>
+// (reverse scan: serial inside a lane, warp-shuffle across lanes), ddt = ddt_direct + A da,
+// dA partial = sum_t dt_t da_t.
+__global__ void __launch_bounds__(128) k_bwd_finish(SegParams p) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int c = blockIdx.x * 4 + warp, h = blockIdx.y, b = blockIdx.z;
+    if (c >= p.nc) return;
+    const int Q = p.Q, per = Q >> 5;
+    const size_t vo = vec_off(p, b, h, c) + (size_t)lane * per;
+    const int ngh = p.P * p.N / 1024;
+    float gh = 0.f;
+    for (int i = 0; i < ngh; ++i) gh += p.ghdot[((((size_t)b * p.H + h) * p.ncs + c) << 3) + i];
+    float v[8], dtv[8], dd[8], sfx[8];
+    float run = 0.f;
+#pragma unroll
+    for (int j = 7; j >= 0; --j)
+        if (j < per) {
+            dtv[j] = p.dtT[vo + j];
+            dd[j] = p.ddt_dir[vo + j];
+            v[j] = p.rho[vo + j] - dtv[j] * dd[j];
+            run += v[j];
+            sfx[j] = run;
+        }
+    float incl = run;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const float t = __shfl_down_sync(0xffffffffu, incl, off);
+        if (lane + off < 32) incl += t;
+    }
+    float excl = __shfl_down_sync(0xffffffffu, incl, 1);
+    if (lane == 31) excl = 0.f;
+    const float Ah = __ldg(p.A + h);
+    const size_t tok0 = (size_t)p.t0 + (size_t)c * Q + (size_t)lane * per;
+    float sA = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        if (j < per) {
+            const float da = (sfx[j] + excl) + gh;
+            p.ddt[(size_t)b * p.dt_bs + (tok0 + j) * p.H + h] = fmaf(Ah, da, dd[j]);
+            sA = fmaf(dtv[j], da, sA);
+        }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sA += __shfl_xor_sync(0xffffffffu, sA, off);
+    if (lane == 0) p.dAp[((size_t)b * p.H + h) * p.nct + p.c0 + c] = sA;
+}
+
+cudaError_t launch_bwd_finish(const SegParams &p, cudaStream_t st) {
+    k_bwd_finish<<<dim3((p.nc + 3) / 4, p.H, p.B), 128, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ a11 tail: sum the head slices of a group
+template <typename T>
+__global__ void __launch_bounds__(256) k_reduce_dbdc(SegParams p) {
+    const size_t total = (size_t)p.B * p.nc * p.Q * p.G * p.N;
+    const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= total) return;
+    const int n = (int)(i % p.N);
+    size_t r = i / p.N;
+    const int g = (int)(r % p.G);
+    r /= p.G;
+    const size_t seglen = (size_t)p.nc * p.Q;
+    const size_t tl = r % seglen;
+    const int b = (int)(r / seglen);
+    const size_t segcap = (size_t)p.ncs * p.Q;
+    const size_t src = ((((size_t)b * segcap + tl) * p.G + g) * p.nsl) * p.N + n;
+    float sB = 0.f, sC = 0.f;
+    for (int s = 0; s < p.nsl; ++s) {
+        sB += p.pB[src + (size_t)s * p.N];
+        sC += p.pC[src + (size_t)s * p.N];
+    }
+    const size_t dst = (size_t)b * p.bc_bs + ((size_t)p.t0 + tl) * p.G * p.N + (size_t)g * p.N + n;
+    stf((T *)p.dB + dst, sB);
+    stf((T *)p.dC + dst, sC);
+}
+
+cudaError_t launch_reduce_dbdc(const SegParams &p, int dtype, cudaStream_t st) {
+    const size_t total = (size_t)p.B * p.nc * p.Q * p.G * p.N;
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+    if (dtype == SSD_DTYPE_F32) k_reduce_dbdc<float><<<blocks, 256, 0, st>>>(p);
+    else k_reduce_dbdc<__nv_bfloat16><<<blocks, 256, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ a13 tail: dA, dD over (batch, chunks)
+// One warp per head; lanes stride over the per-chunk partials in fp64, then a fixed shuffle tree.
+__global__ void __launch_bounds__(32) k_final_dAdD(SegParams p, float *dA, float *dD) {
+    const int h = blockIdx.x, lane = threadIdx.x;
+    const int nrt = p.Q >> 6;
+    double sA = 0.0, sD = 0.0;
+    for (int b = 0; b < p.B; ++b) {
+        const size_t base = ((size_t)b * p.H + h) * p.nct;
+        for (int c = lane; c < p.nct; c += 32) {
+            sA += (double)p.dAp[base + c];
+            for (int r = 0; r < nrt; ++r) sD += (double)p.dDp[((base + c) << 2) + r];
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        sA += __shfl_xor_sync(0xffffffffu, sA, off);
+        sD += __shfl_xor_sync(0xffffffffu, sD, off);
+    }
+    if (lane == 0) {
+        dA[h] = (float)sA;
+        dD[h] = (float)sD;
+    }
+}
+
+cudaError_t launch_final_dAdD(const SegParams &p, float *dA, float *dD, cudaStream_t st) {
+    k_final_dAdD<<<p.H, 32, 0, st>>>(p, dA, dD);
+    return cudaGetLastError();
+}
+
+}  // namespace ssd

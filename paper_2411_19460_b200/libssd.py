@@ -1,0 +1,187 @@
+"""ctypes binding of libssd (include/ssd.h).  Argument marshalling only: every step of the path
+runs in the library's CUDA kernels.  torch is used for device memory and streams, nothing else.
+There is no CPU fallback: if the shared library has not been built, loading raises.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "lib", "libssd.so")
+
+SSD_DTYPE_F32, SSD_DTYPE_BF16 = 0, 1
+SSD_FLAG_FORCE_SIMT = 1
+SSD_OP_FWD, SSD_OP_FWD_SEG, SSD_OP_BWD_SEG = 0, 1, 2
+SSD_OK, SSD_EINVAL, SSD_EUNSUPPORTED, SSD_EALIGN = 0, -1, -2, -3
+SSD_EWORKSPACE, SSD_EDEVICE, SSD_ECUDA, SSD_ETIMEOUT = -4, -5, -6, -7
+
+EXPORTS = ["ssd_workspace_bytes", "ssd_boundary_bytes", "ssd_fwd", "ssd_fwd_segmented",
+           "ssd_bwd_segmented", "ssd_poll_status", "ssd_strerror", "ssd_version",
+           "ssd_last_cuda_error"]
+
+
+class SSDShape(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("B", "L", "H", "P", "N", "G", "chunk", "seg", "dtype", "flags")] + \
+               [(n, ctypes.c_int64) for n in ("x_bstride", "dt_bstride", "bc_bstride")]
+
+
+class SSDError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        msg = lib().ssd_strerror(code).decode()
+        if code == SSD_ECUDA:
+            msg += " [cudaError %d]" % lib().ssd_last_cuda_error()
+        super().__init__("%s: %s (%d)" % (where, msg, code))
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libssd.so is not built: run `python -m paper_2411_19460_b200.build` "
+                               "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, fp, sp = ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(SSDShape)
+        L.ssd_workspace_bytes.restype = ctypes.c_size_t
+        L.ssd_workspace_bytes.argtypes = [sp, ctypes.c_int]
+        L.ssd_boundary_bytes.restype = ctypes.c_size_t
+        L.ssd_boundary_bytes.argtypes = [sp]
+        L.ssd_fwd.restype = ctypes.c_int
+        L.ssd_fwd.argtypes = [sp, vp, fp, fp, vp, vp, fp, fp, vp, fp, vp, ctypes.c_size_t, vp]
+        L.ssd_fwd_segmented.restype = ctypes.c_int
+        L.ssd_fwd_segmented.argtypes = [sp, vp, fp, fp, vp, vp, fp, fp, vp, fp, fp, vp, ctypes.c_size_t, vp]
+        L.ssd_bwd_segmented.restype = ctypes.c_int
+        L.ssd_bwd_segmented.argtypes = [sp, vp, fp, fp, vp, vp, fp, fp, vp, fp,
+                                        vp, fp, fp, vp, vp, fp, fp, vp, ctypes.c_size_t, vp]
+        L.ssd_poll_status.restype = ctypes.c_int
+        L.ssd_poll_status.argtypes = [vp]
+        L.ssd_strerror.restype = ctypes.c_char_p
+        L.ssd_strerror.argtypes = [ctypes.c_int]
+        L.ssd_version.restype = ctypes.c_int
+        L.ssd_last_cuda_error.restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def make_shape(x, Bm, chunk, seg=0, flags=0):
+    """Shape descriptor from the tensors themselves (x [B,L,H,P], Bm [B,L,G,N])."""
+    B, L, H, P = x.shape
+    G, N = Bm.shape[2], Bm.shape[3]
+    if x.dtype == torch.bfloat16:
+        dt = SSD_DTYPE_BF16
+    elif x.dtype == torch.float32:
+        dt = SSD_DTYPE_F32
+    else:
+        raise TypeError("x must be float32 or bfloat16")
+    return SSDShape(B, L, H, P, N, G, int(chunk), int(seg), dt, int(flags), 0, 0, 0)
+
+
+def workspace_bytes(shape, op):
+    return int(lib().ssd_workspace_bytes(ctypes.byref(shape), int(op)))
+
+
+def boundary_bytes(shape):
+    return int(lib().ssd_boundary_bytes(ctypes.byref(shape)))
+
+
+def alloc_workspace(shape, op, device):
+    n = workspace_bytes(shape, op)
+    if n == 0:
+        raise SSDError(SSD_EINVAL, "ssd_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def poll_status(ws):
+    return int(lib().ssd_poll_status(_ptr(ws)))
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check_inputs(x, dt, A, Bm, Cm, D):
+    for name, t in (("x", x), ("dt", dt), ("A", A), ("Bm", Bm), ("Cm", Cm), ("D", D)):
+        if not t.is_cuda or not t.is_contiguous():
+            raise ValueError("%s must be a contiguous CUDA tensor" % name)
+    if dt.dtype != torch.float32 or A.dtype != torch.float32 or D.dtype != torch.float32:
+        raise TypeError("dt, A, D must be float32")
+    if Bm.dtype != x.dtype or Cm.dtype != x.dtype:
+        raise TypeError("Bm, Cm must have the dtype of x")
+
+
+def ssd_fwd(x, dt, A, Bm, Cm, D, h0=None, *, chunk, seg=0, flags=0, y=None, h_final=None,
+            ws=None, stream=None):
+    """y, h_final = SSD forward (Eq. 1).  `seg` only sizes the scratch."""
+    _check_inputs(x, dt, A, Bm, Cm, D)
+    shape = make_shape(x, Bm, chunk, seg, flags)
+    B, L, H, P = x.shape
+    N = Bm.shape[3]
+    y = torch.empty_like(x) if y is None else y
+    h_final = torch.empty(B, H, P, N, dtype=torch.float32, device=x.device) if h_final is None else h_final
+    ws = alloc_workspace(shape, SSD_OP_FWD, x.device) if ws is None else ws
+    rc = lib().ssd_fwd(ctypes.byref(shape), _ptr(x), _ptr(dt), _ptr(A), _ptr(Bm), _ptr(Cm), _ptr(D),
+                       _ptr(h0), _ptr(y), _ptr(h_final), _ptr(ws), ws.numel(), _stream(stream))
+    if rc != SSD_OK:
+        raise SSDError(rc, "ssd_fwd")
+    return y, h_final
+
+
+def ssd_fwd_segmented(x, dt, A, Bm, Cm, D, h0=None, *, chunk, seg, flags=0, y=None, h_final=None,
+                      boundary=None, ws=None, stream=None):
+    """y, h_final, boundary = forward that also stores the state entering every segment
+    (Algorithm 1, sequence axis)."""
+    _check_inputs(x, dt, A, Bm, Cm, D)
+    shape = make_shape(x, Bm, chunk, seg, flags)
+    B, L, H, P = x.shape
+    N = Bm.shape[3]
+    y = torch.empty_like(x) if y is None else y
+    h_final = torch.empty(B, H, P, N, dtype=torch.float32, device=x.device) if h_final is None else h_final
+    if boundary is None:
+        nb = boundary_bytes(shape)
+        if nb == 0:
+            raise SSDError(SSD_EINVAL, "ssd_boundary_bytes")
+        boundary = torch.empty(B, nb // (4 * B * H * P * N), H, P, N, dtype=torch.float32, device=x.device)
+    ws = alloc_workspace(shape, SSD_OP_FWD_SEG, x.device) if ws is None else ws
+    rc = lib().ssd_fwd_segmented(ctypes.byref(shape), _ptr(x), _ptr(dt), _ptr(A), _ptr(Bm), _ptr(Cm),
+                                 _ptr(D), _ptr(h0), _ptr(y), _ptr(h_final), _ptr(boundary), _ptr(ws),
+                                 ws.numel(), _stream(stream))
+    if rc != SSD_OK:
+        raise SSDError(rc, "ssd_fwd_segmented")
+    return y, h_final, boundary
+
+
+def ssd_bwd_segmented(x, dt, A, Bm, Cm, D, boundary, dy, dh_final=None, *, chunk, seg, flags=0,
+                      out=None, want_dh0=True, ws=None, stream=None):
+    """Gradients of Loss = <y,dy> + <h_final,dh_final> by Algorithm 2 along the sequence axis.
+    Returns dict(dx, ddt, dA, dB, dC, dD, dh0)."""
+    _check_inputs(x, dt, A, Bm, Cm, D)
+    shape = make_shape(x, Bm, chunk, seg, flags)
+    B, L, H, P = x.shape
+    N = Bm.shape[3]
+    dev = x.device
+    if out is None:
+        out = dict(dx=torch.empty_like(x), ddt=torch.empty_like(dt),
+                   dA=torch.empty(H, dtype=torch.float32, device=dev),
+                   dB=torch.empty_like(Bm), dC=torch.empty_like(Cm),
+                   dD=torch.empty(H, dtype=torch.float32, device=dev),
+                   dh0=torch.empty(B, H, P, N, dtype=torch.float32, device=dev) if want_dh0 else None)
+    ws = alloc_workspace(shape, SSD_OP_BWD_SEG, dev) if ws is None else ws
+    rc = lib().ssd_bwd_segmented(ctypes.byref(shape), _ptr(x), _ptr(dt), _ptr(A), _ptr(Bm), _ptr(Cm),
+                                 _ptr(D), _ptr(boundary), _ptr(dy), _ptr(dh_final), _ptr(out["dx"]),
+                                 _ptr(out["ddt"]), _ptr(out["dA"]), _ptr(out["dB"]), _ptr(out["dC"]),
+                                 _ptr(out["dD"]), _ptr(out.get("dh0")), _ptr(ws), ws.numel(),
+                                 _stream(stream))
+    if rc != SSD_OK:
+        raise SSDError(rc, "ssd_bwd_segmented")
+    return out

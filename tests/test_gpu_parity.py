@@ -1,0 +1,99 @@
+"""GPU parity: libssd (through the C ABI) against the fp64 oracle, element by element, on seeded
+inputs that span several chunks, several segments, a ragged last segment, both dtypes, several
+chunk lengths, G > 1 and B > 1."""
+import pytest
+import torch
+
+from paper_2411_19460_b200 import libssd
+from paper_2411_19460_b200.inputs import CONFIGS, make_inputs, to_f64_numpy
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+SIMT = libssd.SSD_FLAG_FORCE_SIMT
+
+
+def small(dtype="bf16", **kw):
+    base = dict(name="small", dtype=dtype, B=1, L=1024, H=4, P=64, N=128, G=1, chunk=256, seg=512,
+                h0_std=0.1, dh_std=0.1)
+    base.update(kw)
+    return CONFIGS[0].scaled(**base)
+
+
+CASES = {
+    "cfg0_fp32": CONFIGS[0],
+    "fp32_n128_q128_dh": small("fp32", chunk=128, seg=256, L=768, G=2, B=2),
+    "fp32_q256": small("fp32", chunk=256, seg=512, L=1280),                # ragged last segment
+    "bf16_base": small("bf16"),
+    "bf16_ragged_g2_b2": small("bf16", L=1280, G=2, B=2),
+    "bf16_n64_q64": small("bf16", N=64, chunk=64, seg=128, L=448),
+    "bf16_q128_h8": small("bf16", chunk=128, seg=384, L=1152, H=8, G=4),
+    "bf16_stiff": small("bf16", a_max=64.0, dt_lo=1e-4, dt_hi=1.0, L=2048, seg=1024, H=8, G=2),
+    "bf16_one_segment": small("bf16", seg=1024),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_parity_simt(name):
+    errs = pu.full_parity(CASES[name], flags=SIMT)
+    print(name, errs)
+
+
+@pytest.mark.parametrize("name", [n for n in CASES if CASES[n].dtype == "bf16"])
+def test_parity_default_path(name):
+    errs = pu.full_parity(CASES[name], flags=0)
+    print(name, errs)
+
+
+@pytest.mark.parametrize("flags", [SIMT, 0])
+@pytest.mark.parametrize("name", ["cfg0_fp32", "bf16_ragged_g2_b2", "bf16_stiff"])
+def test_segmented_backward_bit_exact_vs_unsegmented(name, flags):
+    """The gradients must not depend on the segment length (seg == L is the unsegmented run)."""
+    cfg = CASES[name]
+    if cfg.dtype == "fp32" and flags == 0:
+        flags = SIMT
+    inp = make_inputs(cfg, "cuda")
+    a = pu.run_gpu(cfg, inp, seg=cfg.seg, flags=flags)
+    b = pu.run_gpu(cfg, inp, seg=cfg.L, flags=flags)
+    c = pu.run_gpu(cfg, inp, seg=cfg.chunk, flags=flags)
+    for k in ("y", "h_final", "dx", "ddt", "dA", "dB", "dC", "dD", "dh0"):
+        assert torch.equal(a[k], b[k]), k
+        assert torch.equal(a[k], c[k]), k
+    assert torch.equal(a["boundary"][:, 0], b["boundary"][:, 0])
+
+
+def test_deterministic_run_to_run():
+    cfg = CASES["bf16_ragged_g2_b2"]
+    inp = make_inputs(cfg, "cuda")
+    a = pu.run_gpu(cfg, inp)
+    b = pu.run_gpu(cfg, inp)
+    for k in a:
+        assert torch.equal(a[k], b[k]), k
+
+
+def test_ssd_fwd_equals_segmented_forward():
+    cfg = CASES["bf16_base"]
+    inp = make_inputs(cfg, "cuda")
+    y1, h1 = libssd.ssd_fwd(inp["x"], inp["dt"], inp["A"], inp["Bm"], inp["Cm"], inp["D"], inp["h0"],
+                            chunk=cfg.chunk)
+    y2, h2, _ = libssd.ssd_fwd_segmented(inp["x"], inp["dt"], inp["A"], inp["Bm"], inp["Cm"], inp["D"],
+                                         inp["h0"], chunk=cfg.chunk, seg=cfg.seg)
+    torch.cuda.synchronize()
+    assert torch.equal(y1, y2) and torch.equal(h1, h2)
+
+
+def test_null_h0_and_null_dh():
+    cfg = small("bf16", h0_std=0.0, dh_std=0.0)
+    errs = pu.full_parity(cfg)
+    print(errs)
+
+
+def test_status_word_clean():
+    cfg = CASES["bf16_base"]
+    inp = make_inputs(cfg, "cuda")
+    shape = libssd.make_shape(inp["x"], inp["Bm"], cfg.chunk, cfg.seg)
+    ws = libssd.alloc_workspace(shape, libssd.SSD_OP_FWD_SEG, "cuda")
+    libssd.ssd_fwd_segmented(inp["x"], inp["dt"], inp["A"], inp["Bm"], inp["Cm"], inp["D"], inp["h0"],
+                             chunk=cfg.chunk, seg=cfg.seg, ws=ws)
+    torch.cuda.synchronize()
+    assert libssd.poll_status(ws) == libssd.SSD_OK
