@@ -1,0 +1,399 @@
+#!/usr/bin/env python
+"""Benchmark of libssd: segmented SSD forward + backward (MA-GC along the sequence axis).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--seg S] [--impl ours|reference]
+
+One "step" = ssd_fwd_segmented + ssd_bwd_segmented over one batch of seeded synthetic input.
+Prints ONE JSON line (rank 0).  With N > 1 (launched by torch.distributed.run) every rank runs an
+independent replica on its own GPU: the path has no cross-GPU step, so no data-path collective is
+used; only the barrier and the max-over-ranks of the timing go through torch.distributed.
+
+`--impl reference` times the fp64 CPU oracle (oracle/), as it stands, on the host cores, on a
+bounded sample of the same workload.
+"""
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2411_19460_b200.inputs import CONFIGS, make_inputs, to_f64_numpy  # noqa: E402
+
+METRIC = "ssd_fwd_bwd_segmented_tokens_per_s"
+UNIT = "tokens/s"
+
+
+# ----------------------------------------------------------------------------- analytic model
+def kappa(Q):
+    return (Q + 1) / (2.0 * Q)
+
+
+def kind_model(cfg):
+    """Algorithmic flops and bytes per token for each kernel kind (one launch processes
+    B * segment-length tokens).  Only the lower triangle of the Q x Q products counts; elementwise
+    work and exponentials are not counted; e = bytes per I/O element."""
+    H, P, N, G, Q = cfg.H, cfg.P, cfg.N, cfg.G, cfg.chunk
+    e = 2 if cfg.dtype == "bf16" else 4
+    k = kappa(Q)
+    HPN = H * P * N
+    st = 4.0 * HPN / Q                       # one fp32 chunk state per Q tokens
+    return {
+        # kind: (bound, flops/token, bytes/token)
+        "chunk_cumsum": ("hbm", 0.0, 12.0 * H),
+        "chunk_state": ("tensor", 2.0 * HPN, e * (H * P + G * N) + st),
+        "state_pass_fwd": ("hbm", 0.0, 2.0 * st),
+        "chunk_scan_fwd": ("tensor", 2.0 * HPN + 2 * k * Q * (G * N + H * P), e * (2 * H * P + 2 * G * N) + st),
+        "dstate_contrib": ("tensor", 2.0 * HPN, e * (H * P + G * N) + st),
+        "state_pass_bwd": ("hbm", 0.0, 3.0 * st),
+        "bwd_dx": ("tensor", 2.0 * HPN + 2 * k * Q * (G * N + H * P), e * (3 * H * P + 2 * G * N) + st),
+        "bwd_dC": ("tensor", 2.0 * HPN + 2 * k * Q * (G * N + H * P), e * (2 * H * P + 2 * G * N) + st),
+        "bwd_dB": ("tensor", 2.0 * HPN + 2 * k * Q * (G * N), e * (2 * H * P + 2 * G * N) + st),
+        "bwd_finish": ("hbm", 0.0, 16.0 * H),
+        "reduce_dBdC": ("hbm", 0.0, 2.0 * e * G * N),
+        "final_dAdD": ("hbm", 0.0, 0.0),
+    }
+
+
+def step_model(cfg, seg):
+    """Whole-step algorithmic flops / bytes per token (forward + recompute + backward)."""
+    H, P, N, G, Q = cfg.H, cfg.P, cfg.N, cfg.G, cfg.chunk
+    e = 2 if cfg.dtype == "bf16" else 4
+    k = kappa(Q)
+    HPN = H * P * N
+    flops = (4 * HPN + 2 * k * Q * (G * N + H * P)) + 2 * HPN + (8 * HPN + 2 * k * Q * (3 * G * N + 2 * H * P))
+    byts = e * (6 * H * P + 7 * G * N) + 16 * H + 2 * 4.0 * HPN / seg
+    return flops, byts
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ----------------------------------------------------------------------------- clocks sampling
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device):
+        self.proc = None
+        self.path = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "--id=" + uuid, "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [s.strip() for s in line.split(",")]
+                if len(f) < 8:
+                    continue
+                try:
+                    sm.append(float(f[0]))
+                    mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                      "sw_power_cap"), f[4:8]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ----------------------------------------------------------------------------- the GPU arm
+def run_ours(args):
+    from paper_2411_19460_b200 import libssd
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    cfg = CONFIGS[args.config]
+    if cfg.layers != 1:
+        raise SystemExit("config %d is the layer-stack sweep; it is not a bench line" % args.config)
+    seg = args.seg or cfg.seg
+    flags = libssd.SSD_FLAG_FORCE_SIMT if args.simt else 0
+    inp = make_inputs(cfg, dev, seed=cfg.seed + rank)
+    x, dt, A, Bm, Cm, D, h0, dy = (inp[k] for k in ("x", "dt", "A", "Bm", "Cm", "D", "h0", "dy"))
+    B, L, H, P = x.shape
+    N = Bm.shape[3]
+    tokens = B * L
+
+    shape = libssd.make_shape(x, Bm, cfg.chunk, seg, flags)
+    ws_f = libssd.alloc_workspace(shape, libssd.SSD_OP_FWD_SEG, dev)
+    ws_b = libssd.alloc_workspace(shape, libssd.SSD_OP_BWD_SEG, dev)
+    nseg = (L + seg - 1) // seg
+    y = torch.empty_like(x)
+    hf = torch.empty(B, H, P, N, dtype=torch.float32, device=dev)
+    bd = torch.empty(B, nseg, H, P, N, dtype=torch.float32, device=dev)
+    out = dict(dx=torch.empty_like(x), ddt=torch.empty_like(dt), dA=torch.empty(H, device=dev),
+               dB=torch.empty_like(Bm), dC=torch.empty_like(Cm), dD=torch.empty(H, device=dev),
+               dh0=torch.empty(B, H, P, N, dtype=torch.float32, device=dev))
+    stream = torch.cuda.current_stream()
+
+    def step(src=None):
+        s = inp if src is None else src
+        libssd.ssd_fwd_segmented(s["x"], s["dt"], s["A"], s["Bm"], s["Cm"], s["D"], s["h0"],
+                                 chunk=cfg.chunk, seg=seg, flags=flags, y=y, h_final=hf, boundary=bd,
+                                 ws=ws_f, stream=stream)
+        libssd.ssd_bwd_segmented(s["x"], s["dt"], s["A"], s["Bm"], s["Cm"], s["D"], bd, s["dy"], None,
+                                 chunk=cfg.chunk, seg=seg, flags=flags, out=out, ws=ws_b, stream=stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(v):
+        if world == 1:
+            return v
+        t = torch.tensor([v], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident timing
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    torch.cuda.reset_peak_memory_stats(dev)
+    sampler = ClockSampler(dev) if rank == 0 else None
+    n0 = libssd.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    launches = libssd.launch_count() - n0
+    clocks = sampler.stop() if sampler else None
+    peak_mem = torch.cuda.max_memory_allocated(dev)
+    assert libssd.poll_status(ws_f) == 0 and libssd.poll_status(ws_b) == 0, "device-side wait timed out"
+    ms_per_step = ms_total / args.steps
+    value = world * tokens / (ms_per_step * 1e-3)
+
+    # ---- per-kernel-kind timing (CUDA events on the launch stream, separate pass of the same steps)
+    prof_steps = min(args.steps, 3)
+    libssd.profile(True)
+    for _ in range(prof_steps):
+        step()
+    torch.cuda.synchronize()
+    prof = libssd.profile_read()
+    libssd.profile(False)
+
+    # ---- end to end: pinned host buffers -> device -> C ABI -> results back to pinned host
+    e2e = None
+    if not args.no_e2e:
+        names_in = [k for k in ("x", "dt", "A", "Bm", "Cm", "D", "h0", "dy") if inp[k] is not None]
+        host_in = {k: torch.empty(inp[k].shape, dtype=inp[k].dtype, pin_memory=True).copy_(inp[k])
+                   for k in names_in}
+        dev_in = {k: torch.empty_like(inp[k]) for k in names_in}
+        dev_in["h0"] = dev_in.get("h0")
+        outs = dict(y=y, h_final=hf, **out)
+        host_out = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in outs.items()}
+        bi = sum(t.numel() * t.element_size() for t in host_in.values())
+        bo = sum(t.numel() * t.element_size() for t in host_out.values())
+
+        def e2e_step():
+            for k in names_in:
+                dev_in[k].copy_(host_in[k], non_blocking=True)
+            step(dev_in)
+            for k, v in outs.items():
+                host_out[k].copy_(v, non_blocking=True)
+
+        e2e_steps = max(1, min(args.steps, 5))
+        e2e_step()
+        barrier()
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
+        e2e = dict(value=world * tokens / (ms_e2e * 1e-3), unit=UNIT, h2d_bytes_per_step=bi,
+                   d2h_bytes_per_step=bo, ms_per_step=ms_e2e, steps=e2e_steps)
+        del host_in, host_out, dev_in
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    model = kind_model(cfg)
+    # dominant kernel kind = largest share of device time
+    total_prof = sum(v[0] for v in prof.values()) or 1.0
+    dom = max(prof, key=lambda k: prof[k][0])
+    dom_ms, dom_n = prof[dom]
+    bound, fl_tok, by_tok = model[dom]
+    tok_per_launch = tokens * prof_steps / max(dom_n, 1)
+    avg_s = dom_ms * 1e-3 / max(dom_n, 1)
+    if bound == "tensor":
+        achieved = fl_tok * tok_per_launch / avg_s / 1e12
+        peak = peaks["bf16_tflops_sustained"]
+        unit = "TFLOP/s"
+    else:
+        achieved = by_tok * tok_per_launch / avg_s / 1e9
+        peak = peaks["hbm_gbs"]
+        unit = "GB/s"
+    roofline = dict(kernel=dom, bound="tensor" if bound == "tensor" else "hbm", achieved=achieved, peak=peak,
+                    unit=unit, frac=achieved / peak, traffic=None, peak_source=peaks["source"],
+                    avg_launch_us=avg_s * 1e6, launches=dom_n, share_of_device_time=dom_ms / total_prof)
+    fl, by = step_model(cfg, seg)
+    t_roof = max(fl * tokens / (peaks["bf16_tflops"] * 1e12), by * tokens / (peaks["hbm_gbs"] * 1e9))
+    step_roof = dict(flops_per_token=fl, bytes_per_token=by, roofline_ms=t_roof * 1e3,
+                     frac=t_roof * 1e3 / ms_per_step)
+    kinds = {k: dict(ms_per_step=v[0] / prof_steps, launches_per_step=v[1] / prof_steps,
+                     share=v[0] / total_prof) for k, v in prof.items() if v[1]}
+
+    cpu = None
+    if not args.no_cpu:
+        cpu = cpu_baseline(cfg, inp, sample_tokens=args.cpu_tokens)
+
+    io_bytes = sum(t.numel() * t.element_size() for t in (x, dt, Bm, Cm, dy, y, out["dx"], out["ddt"],
+                                                         out["dB"], out["dC"]))
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
+        "data": "synthetic", "impl": "ours",
+        "config": {"workload": cfg.name, "B": B, "L": L, "H": H, "P": P, "N": N, "G": cfg.G,
+                   "chunk": cfg.chunk, "seg": seg, "nseg": nseg, "l2": "inputs larger than L2",
+                   "path": "simt" if (args.simt or cfg.dtype == "fp32") else "default",
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": roofline, "step_roofline": step_roof, "kernels": kinds,
+        "memory": {"peak_allocated_bytes": int(peak_mem), "workspace_fwd_bytes": ws_f.numel(),
+                   "workspace_bwd_bytes": ws_b.numel(), "boundary_bytes": bd.numel() * 4,
+                   "io_bytes": int(io_bytes)},
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- the CPU oracle legs
+def _oracle_sample(cfg, inp, sample_tokens):
+    """fp64 host copies of the first `sample_tokens` tokens (all heads) of the workload."""
+    Ls = min(cfg.L, sample_tokens)
+    sub = {k: (v[:, :Ls] if (v is not None and k in ("x", "dt", "Bm", "Cm", "dy")) else v)
+           for k, v in inp.items()}
+    return to_f64_numpy(sub), Ls
+
+
+def _time_oracle(d):
+    from oracle import ssd_oracle as orc
+    t0 = time.perf_counter()
+    y, hf, bd = orc.ssd_fwd(d["x"], d["dt"], d["A"], d["Bm"], d["Cm"], d["D"], d["h0"], seg=1024)
+    orc.ssd_bwd(d["x"], d["dt"], d["A"], d["Bm"], d["Cm"], d["D"], d["h0"], d["dy"], None, blk=256)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(cfg, inp, sample_tokens):
+    from oracle import ssd_oracle as orc
+    d, Ls = _oracle_sample(cfg, inp, sample_tokens)
+    secs = _time_oracle(d)
+    return dict(value=cfg.B * Ls / secs, unit=UNIT, cores=orc.threads(), kind="oracle",
+                sample="first %d of %d tokens, all %d heads, fwd+bwd once (%.1f s)" % (Ls, cfg.L, cfg.H, secs))
+
+
+def run_reference(args):
+    """The oracle as the reference arm: each step is fwd+bwd over a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import ssd_oracle as orc
+    cfg = CONFIGS[args.config]
+    seg = args.seg or cfg.seg
+    Ls = min(cfg.L, args.ref_tokens)
+    small = cfg.scaled(L=Ls)
+    inp = make_inputs(small, "cpu")
+    d = to_f64_numpy(inp)
+    for _ in range(args.warmup):
+        _time_oracle(d)
+    t = [_time_oracle(d) for _ in range(args.steps)]
+    secs = sum(t) / len(t)
+    value = cfg.B * Ls / secs
+    sample = "first %d of %d tokens, all %d heads, per step" % (Ls, cfg.L, cfg.H)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
+        "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "H": cfg.H, "P": cfg.P, "N": cfg.N,
+                   "G": cfg.G, "chunk": cfg.chunk, "seg": seg, "sampled_tokens": Ls},
+        "cpu_baseline": dict(value=value, unit=UNIT, cores=orc.threads(), kind="oracle", sample=sample),
+        "e2e": dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=6)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="index into the five workloads (default 2: "
+                    "Mamba-2-2.7B-dim layer, L=131072)")
+    ap.add_argument("--seg", type=int, default=0, help="override the segment length")
+    ap.add_argument("--simt", action="store_true", help="force the CUDA-core kernels")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--cpu-tokens", type=int, default=32768, help="tokens in the cpu_baseline sample")
+    ap.add_argument("--ref-tokens", type=int, default=8192, help="tokens per step of --impl reference")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

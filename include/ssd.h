@@ -141,6 +141,22 @@ int ssd_version(void);
 /* The cudaError_t of the most recent failed CUDA call made by this library on this thread. */
 int ssd_last_cuda_error(void);
 
+/*
+ * Instrumentation (not part of the method; the paper has no counterpart).
+ * ssd_launch_count: kernels this library has launched in this process so far.
+ * ssd_kernel_kinds / ssd_kernel_name: number of distinct kernel kinds and their names.
+ * ssd_profile(1) makes later calls bracket every kernel launch with a pair of CUDA events on the
+ * caller's stream (events are created on demand: the one place the library creates CUDA objects);
+ * ssd_profile(0) stops it.  ssd_profile_read waits for the recorded events, writes the summed
+ * milliseconds and the launch count per kernel kind into ms[n] / launches[n] (HOST arrays,
+ * n >= ssd_kernel_kinds()) and clears the record.  Not thread-safe; meant for benchmarks.
+ */
+long long ssd_launch_count(void);
+int ssd_kernel_kinds(void);
+const char *ssd_kernel_name(int kind);
+int ssd_profile(int enable);
+int ssd_profile_read(double *ms, long long *launches, int n);
+
 #ifdef __cplusplus
 }
 #endif

@@ -3,14 +3,44 @@
 // segments right to left: recompute from the stored state, back-propagate, hand dh to the left)
 // for one SSD layer.  Checkpoint memory is set by the segment length: the scratch holds the chunk
 // states of ONE segment, the boundary buffer one state per segment.
+#include <atomic>
 #include <cstdio>
 #include <cstring>
+#include <vector>
 
 #include "ssd_internal.h"
 
 namespace ssd {
 
 static thread_local int g_last_cuda = 0;
+
+// ---- optional instrumentation: launch counter and per-kernel-kind CUDA-event timing ----
+static std::atomic<long long> g_launches{0};
+struct ProfEvent { int kind; cudaEvent_t a, b; };
+static bool g_prof_on = false;
+static std::vector<ProfEvent> g_prof_pool;
+static size_t g_prof_used = 0;
+
+static const char *const kKindNames[KIND_COUNT] = {
+    "chunk_cumsum", "chunk_state", "state_pass_fwd", "chunk_scan_fwd", "dstate_contrib",
+    "state_pass_bwd", "bwd_dx", "bwd_dC", "bwd_dB", "bwd_finish", "reduce_dBdC", "final_dAdD"};
+
+static ProfEvent *prof_begin(int kind, cudaStream_t st) {
+    if (!g_prof_on) return nullptr;
+    if (g_prof_used == g_prof_pool.size()) {
+        ProfEvent ev;
+        ev.kind = kind;
+        if (cudaEventCreate(&ev.a) != cudaSuccess || cudaEventCreate(&ev.b) != cudaSuccess) return nullptr;
+        g_prof_pool.push_back(ev);
+    }
+    ProfEvent *ev = &g_prof_pool[g_prof_used++];
+    ev->kind = kind;
+    cudaEventRecord(ev->a, st);
+    return ev;
+}
+static void prof_end(ProfEvent *ev, cudaStream_t st) {
+    if (ev) cudaEventRecord(ev->b, st);
+}
 
 struct Layout {
     size_t status, cs, dtT, Hst, Hbf, hcarry, Gst, Gbf, gcarry, ghdot, ddt_dir, rho, pB, pC, dAp, dDp;
@@ -117,6 +147,19 @@ static int check_device() {
         }                                               \
     } while (0)
 
+// one kernel launch of kind `kind` on stream `st`
+#define SSD_LAUNCH(kind, expr)                          \
+    do {                                                \
+        ProfEvent *pe__ = prof_begin(kind, st);         \
+        cudaError_t e__ = (expr);                       \
+        prof_end(pe__, st);                             \
+        g_launches.fetch_add(1, std::memory_order_relaxed); \
+        if (e__ != cudaSuccess) {                       \
+            g_last_cuda = (int)e__;                     \
+            return SSD_ECUDA;                           \
+        }                                               \
+    } while (0)
+
 static void fill_params(const Plan &pl, const Layout &lo, void *ws, SegParams &sp) {
     memset(&sp, 0, sizeof(sp));
     sp.B = pl.B; sp.L = pl.L; sp.H = pl.H; sp.P = pl.P; sp.N = pl.N; sp.G = pl.G; sp.Q = pl.Q;
@@ -175,13 +218,13 @@ static int forward_impl(const ssd_shape_t *shape, const void *x, const float *dt
     const long long PN = (long long)pl.P * pl.N;
     for (int k = 0; k < pl.nseg; ++k) {
         set_segment(pl, k, sp);
-        SSD_TRY(launch_chunk_cumsum(sp, st));
-        SSD_TRY(launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
+        SSD_LAUNCH(KIND_CUMSUM, launch_chunk_cumsum(sp, st));
+        SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
         const float *init = (k == 0) ? h0 : sp.hcarry;
         float *bnd = boundary ? boundary + (size_t)k * pl.H * PN : nullptr;
-        SSD_TRY(launch_state_pass_fwd(sp, init, (long long)pl.H * PN, bnd, (long long)pl.nseg * pl.H * PN,
+        SSD_LAUNCH(KIND_STATE_PASS_FWD, launch_state_pass_fwd(sp, init, (long long)pl.H * PN, bnd, (long long)pl.nseg * pl.H * PN,
                                       (k == pl.nseg - 1) ? h_final : nullptr, pl.use_tc, st));
-        SSD_TRY(launch_masked_product_simt(sp, pl.dtype, MP_FWD, st));
+        SSD_LAUNCH(KIND_SCAN_FWD, launch_masked_product_simt(sp, pl.dtype, MP_FWD, st));
     }
     return SSD_OK;
 }
@@ -250,22 +293,22 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
     for (int k = pl.nseg - 1; k >= 0; --k) {
         set_segment(pl, k, sp);
         // Recompute_Forward: chunk-entry states of segment k from the stored boundary state
-        SSD_TRY(launch_chunk_cumsum(sp, st));
-        SSD_TRY(launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
-        SSD_TRY(launch_state_pass_fwd(sp, boundary + (size_t)k * pl.H * PN, (long long)pl.nseg * pl.H * PN,
+        SSD_LAUNCH(KIND_CUMSUM, launch_chunk_cumsum(sp, st));
+        SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
+        SSD_LAUNCH(KIND_STATE_PASS_FWD, launch_state_pass_fwd(sp, boundary + (size_t)k * pl.H * PN, (long long)pl.nseg * pl.H * PN,
                                       nullptr, 0, nullptr, pl.use_tc, st));
         // Backward through the segment; dh enters from the right, leaves to the left
-        SSD_TRY(launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_DSTATE, st));
+        SSD_LAUNCH(KIND_DSTATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_DSTATE, st));
         const float *ginit = (k == pl.nseg - 1) ? dh_final : sp.gcarry;
         float *gleft = (k == 0 && dh0) ? dh0 : sp.gcarry;
-        SSD_TRY(launch_state_pass_bwd(sp, ginit, gleft, pl.use_tc, st));
-        SSD_TRY(launch_masked_product_simt(sp, pl.dtype, MP_BWD_DX, st));
-        SSD_TRY(launch_masked_product_simt(sp, pl.dtype, MP_DC, st));
-        SSD_TRY(launch_masked_product_simt(sp, pl.dtype, MP_DB, st));
-        SSD_TRY(launch_bwd_finish(sp, st));
-        SSD_TRY(launch_reduce_dbdc(sp, pl.dtype, st));
+        SSD_LAUNCH(KIND_STATE_PASS_BWD, launch_state_pass_bwd(sp, ginit, gleft, pl.use_tc, st));
+        SSD_LAUNCH(KIND_BWD_DX, launch_masked_product_simt(sp, pl.dtype, MP_BWD_DX, st));
+        SSD_LAUNCH(KIND_BWD_DC, launch_masked_product_simt(sp, pl.dtype, MP_DC, st));
+        SSD_LAUNCH(KIND_BWD_DB, launch_masked_product_simt(sp, pl.dtype, MP_DB, st));
+        SSD_LAUNCH(KIND_BWD_FINISH, launch_bwd_finish(sp, st));
+        SSD_LAUNCH(KIND_REDUCE_DBDC, launch_reduce_dbdc(sp, pl.dtype, st));
     }
-    SSD_TRY(launch_final_dAdD(sp, dA, dD, st));
+    SSD_LAUNCH(KIND_FINAL, launch_final_dAdD(sp, dA, dD, st));
     return SSD_OK;
 }
 
@@ -292,6 +335,36 @@ const char *ssd_strerror(int code) {
 }
 
 int ssd_version(void) { return SSD_VERSION; }
+
+long long ssd_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int ssd_kernel_kinds(void) { return KIND_COUNT; }
+
+const char *ssd_kernel_name(int kind) {
+    return (kind >= 0 && kind < KIND_COUNT) ? kKindNames[kind] : "";
+}
+
+int ssd_profile(int enable) {
+    g_prof_on = enable != 0;
+    g_prof_used = 0;
+    return SSD_OK;
+}
+
+int ssd_profile_read(double *ms, long long *launches, int n) {
+    if (!ms || !launches || n < KIND_COUNT) return SSD_EINVAL;
+    for (int i = 0; i < n; ++i) { ms[i] = 0.0; launches[i] = 0; }
+    for (size_t i = 0; i < g_prof_used; ++i) {
+        ProfEvent &ev = g_prof_pool[i];
+        cudaError_t e = cudaEventSynchronize(ev.b);
+        float t = 0.f;
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&t, ev.a, ev.b);
+        if (e != cudaSuccess) { g_last_cuda = (int)e; return SSD_ECUDA; }
+        ms[ev.kind] += (double)t;
+        launches[ev.kind] += 1;
+    }
+    g_prof_used = 0;
+    return SSD_OK;
+}
 
 int ssd_last_cuda_error(void) { return g_last_cuda; }
 

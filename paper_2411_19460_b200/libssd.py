@@ -18,7 +18,8 @@ SSD_EWORKSPACE, SSD_EDEVICE, SSD_ECUDA, SSD_ETIMEOUT = -4, -5, -6, -7
 
 EXPORTS = ["ssd_workspace_bytes", "ssd_boundary_bytes", "ssd_fwd", "ssd_fwd_segmented",
            "ssd_bwd_segmented", "ssd_poll_status", "ssd_strerror", "ssd_version",
-           "ssd_last_cuda_error"]
+           "ssd_last_cuda_error", "ssd_launch_count", "ssd_kernel_kinds", "ssd_kernel_name",
+           "ssd_profile", "ssd_profile_read"]
 
 
 class SSDShape(ctypes.Structure):
@@ -65,6 +66,15 @@ def lib():
         L.ssd_strerror.argtypes = [ctypes.c_int]
         L.ssd_version.restype = ctypes.c_int
         L.ssd_last_cuda_error.restype = ctypes.c_int
+        L.ssd_launch_count.restype = ctypes.c_longlong
+        L.ssd_kernel_kinds.restype = ctypes.c_int
+        L.ssd_kernel_name.restype = ctypes.c_char_p
+        L.ssd_kernel_name.argtypes = [ctypes.c_int]
+        L.ssd_profile.restype = ctypes.c_int
+        L.ssd_profile.argtypes = [ctypes.c_int]
+        L.ssd_profile_read.restype = ctypes.c_int
+        L.ssd_profile_read.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_longlong),
+                                       ctypes.c_int]
         _lib = L
     return _lib
 
@@ -103,6 +113,26 @@ def alloc_workspace(shape, op, device):
 
 def poll_status(ws):
     return int(lib().ssd_poll_status(_ptr(ws)))
+
+
+def launch_count():
+    """Kernels launched by the library in this process so far."""
+    return int(lib().ssd_launch_count())
+
+
+def profile(enable):
+    lib().ssd_profile(1 if enable else 0)
+
+
+def profile_read():
+    """{kernel kind name: (total ms, launches)} since profiling was enabled; clears the record."""
+    n = lib().ssd_kernel_kinds()
+    ms = (ctypes.c_double * n)()
+    cnt = (ctypes.c_longlong * n)()
+    rc = lib().ssd_profile_read(ms, cnt, n)
+    if rc != SSD_OK:
+        raise SSDError(rc, "ssd_profile_read")
+    return {lib().ssd_kernel_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n)}
 
 
 def _stream(stream):
