@@ -66,7 +66,8 @@ enum {
     SSD_EWORKSPACE = -4,   /* ws too small or misaligned                                          */
     SSD_EDEVICE = -5,      /* current device is not compute capability 10.x                       */
     SSD_ECUDA = -6,        /* a CUDA call failed; see ssd_last_cuda_error()                       */
-    SSD_ETIMEOUT = -7      /* a bounded device-side wait expired (reported by ssd_poll_status)    */
+    SSD_ETIMEOUT = -7,     /* a bounded device-side wait expired (reported by ssd_poll_status)    */
+    SSD_ETOOLARGE = -8     /* ssd_fwd_static_ws: the shape needs more scratch than the built-in buffer */
 };
 
 /*
@@ -100,6 +101,33 @@ size_t ssd_boundary_bytes(const ssd_shape_t *shape);
 int ssd_fwd(const ssd_shape_t *shape, const void *x, const float *dt, const float *A,
             const void *Bm, const void *Cm, const float *D, const float *h0,
             void *y, float *h_final, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * ssd_fwd for callers that cannot provide scratch memory.  (The paper has no counterpart; this is
+ * a packaging variant of ssd_fwd.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- inside a region that must
+ * not call cudaMalloc (a latency-critical serving loop, a plug-in whose host owns all memory, a
+ * process that has already handed the whole device to another allocator) -- and so has no way to
+ * obtain the `ws` buffer that ssd_fwd asks for.  Here the scratch is a fixed array of
+ * SSD_STATIC_WS_BYTES bytes that lives inside the library's device image: every GPU that loads the
+ * library holds those bytes until the process exits, whether or not this call is ever used.
+ * The call itself performs no allocation of any kind; inputs and outputs are still the caller's.
+ *
+ * Same arguments and results as ssd_fwd (bit-identical outputs), minus ws / ws_bytes.
+ *  - Returns SSD_ETOOLARGE, with nothing enqueued, when ssd_workspace_bytes(shape, SSD_OP_FWD)
+ *    exceeds SSD_STATIC_WS_BYTES: shrink `seg` (scratch grows with seg/chunk, not with L) or use
+ *    ssd_fwd with your own buffer.
+ *  - The first call on each device looks up the device address of the built-in array (with that
+ *    device current).  Make that first call outside any CUDA stream capture.
+ *  - All calls on one device share the one array, and it keeps whatever the previous call left
+ *    in it; the call re-initialises the parts that must start from zero.  Two calls that overlap
+ *    on the same GPU (different streams, or different host threads) race on it: serialise them.
+ */
+#define SSD_STATIC_WS_BYTES (8u * 1024u * 1024u)
+int ssd_fwd_static_ws(const ssd_shape_t *shape, const void *x, const float *dt, const float *A,
+                      const void *Bm, const void *Cm, const float *D, const float *h0,
+                      void *y, float *h_final, void *stream);
 
 /*
  * Forward with sequence-axis checkpoints (Algorithm 1, one layer): as ssd_fwd, and in addition

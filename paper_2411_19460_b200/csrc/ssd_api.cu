@@ -6,6 +6,7 @@
 #include <atomic>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 #include "ssd_internal.h"
@@ -229,6 +230,32 @@ static int forward_impl(const ssd_shape_t *shape, const void *x, const float *dt
     return SSD_OK;
 }
 
+// ---- built-in scratch for ssd_fwd_static_ws (callers that cannot allocate) ----
+// Lives in the device image of this library: one copy per GPU that loads it, for the life of the
+// process.  In host code `g_static_ws` is only a handle for cudaGetSymbolAddress, never a pointer.
+static __device__ __align__(256) unsigned char g_static_ws[SSD_STATIC_WS_BYTES];
+
+static const int kMaxDevices = 64;
+static std::mutex g_static_mu;
+static void *g_static_addr[kMaxDevices] = {nullptr};
+
+// Device address of g_static_ws on the current device, looked up once per device.
+static int static_ws_address(void **out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { g_last_cuda = (int)e; return SSD_ECUDA; }
+    if (dev < 0 || dev >= kMaxDevices) return SSD_EDEVICE;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_addr[dev]) {
+        void *ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_ws);
+        if (e != cudaSuccess || !ptr) { g_last_cuda = (int)e; return SSD_ECUDA; }
+        g_static_addr[dev] = ptr;
+    }
+    *out = g_static_addr[dev];
+    return SSD_OK;
+}
+
 }  // namespace ssd
 
 using namespace ssd;
@@ -254,6 +281,27 @@ int ssd_fwd(const ssd_shape_t *shape, const void *x, const float *dt, const floa
             const void *Cm, const float *D, const float *h0, void *y, float *h_final, void *ws,
             size_t ws_bytes, void *stream) {
     return forward_impl(shape, x, dt, A, Bm, Cm, D, h0, y, h_final, nullptr, false, ws, ws_bytes, stream);
+}
+
+int ssd_fwd_static_ws(const ssd_shape_t *shape, const void *x, const float *dt, const float *A,
+                      const void *Bm, const void *Cm, const float *D, const float *h0, void *y,
+                      float *h_final, void *stream) {
+    Plan pl;
+    int rc = make_plan(shape, pl);
+    if (rc) return rc;
+    Layout lo;
+    make_layout(pl, SSD_OP_FWD, lo);
+    if (lo.total > (size_t)SSD_STATIC_WS_BYTES) return SSD_ETOOLARGE;
+    if (!x || !dt || !A || !Bm || !Cm || !D || !y) return SSD_EINVAL;
+    rc = check_device();
+    if (rc) return rc;
+    void *ws = nullptr;
+    rc = static_ws_address(&ws);
+    if (rc) return rc;
+    // forward_impl zeroes the status word on the stream and writes every other scratch region
+    // before reading it, so stale contents of the shared array cannot leak into the outputs.
+    return forward_impl(shape, x, dt, A, Bm, Cm, D, h0, y, h_final, nullptr, false, ws,
+                        (size_t)SSD_STATIC_WS_BYTES, stream);
 }
 
 int ssd_fwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, const float *A,
@@ -330,6 +378,7 @@ const char *ssd_strerror(int code) {
         case SSD_EDEVICE: return "current device is not compute capability 10.x";
         case SSD_ECUDA: return "CUDA call failed (see ssd_last_cuda_error)";
         case SSD_ETIMEOUT: return "a bounded device-side wait expired";
+        case SSD_ETOOLARGE: return "shape needs more scratch than the built-in static buffer (SSD_STATIC_WS_BYTES); reduce seg or pass your own workspace to ssd_fwd";
         default: return "unknown error";
     }
 }

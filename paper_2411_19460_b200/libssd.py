@@ -15,11 +15,13 @@ SSD_FLAG_FORCE_SIMT = 1
 SSD_OP_FWD, SSD_OP_FWD_SEG, SSD_OP_BWD_SEG = 0, 1, 2
 SSD_OK, SSD_EINVAL, SSD_EUNSUPPORTED, SSD_EALIGN = 0, -1, -2, -3
 SSD_EWORKSPACE, SSD_EDEVICE, SSD_ECUDA, SSD_ETIMEOUT = -4, -5, -6, -7
+SSD_ETOOLARGE = -8
+SSD_STATIC_WS_BYTES = 8 * 1024 * 1024
 
 EXPORTS = ["ssd_workspace_bytes", "ssd_boundary_bytes", "ssd_fwd", "ssd_fwd_segmented",
            "ssd_bwd_segmented", "ssd_poll_status", "ssd_strerror", "ssd_version",
            "ssd_last_cuda_error", "ssd_launch_count", "ssd_kernel_kinds", "ssd_kernel_name",
-           "ssd_profile", "ssd_profile_read"]
+           "ssd_profile", "ssd_profile_read", "ssd_fwd_static_ws"]
 
 
 class SSDShape(ctypes.Structure):
@@ -55,6 +57,8 @@ def lib():
         L.ssd_boundary_bytes.argtypes = [sp]
         L.ssd_fwd.restype = ctypes.c_int
         L.ssd_fwd.argtypes = [sp, vp, fp, fp, vp, vp, fp, fp, vp, fp, vp, ctypes.c_size_t, vp]
+        L.ssd_fwd_static_ws.restype = ctypes.c_int
+        L.ssd_fwd_static_ws.argtypes = [sp, vp, fp, fp, vp, vp, fp, fp, vp, fp, vp]
         L.ssd_fwd_segmented.restype = ctypes.c_int
         L.ssd_fwd_segmented.argtypes = [sp, vp, fp, fp, vp, vp, fp, fp, vp, fp, fp, vp, ctypes.c_size_t, vp]
         L.ssd_bwd_segmented.restype = ctypes.c_int
@@ -164,6 +168,20 @@ def ssd_fwd(x, dt, A, Bm, Cm, D, h0=None, *, chunk, seg=0, flags=0, y=None, h_fi
                        _ptr(h0), _ptr(y), _ptr(h_final), _ptr(ws), ws.numel(), _stream(stream))
     if rc != SSD_OK:
         raise SSDError(rc, "ssd_fwd")
+    return y, h_final
+
+
+def ssd_fwd_static_ws(x, dt, A, Bm, Cm, D, h0=None, *, chunk, seg=0, flags=0, y, h_final, stream=None):
+    """ssd_fwd for callers that cannot allocate: the scratch is a fixed SSD_STATIC_WS_BYTES array
+    built into the library (shared by all calls on the device: do not overlap two of them), and
+    this wrapper allocates nothing either, so `y` and `h_final` must be passed in.  Raises
+    SSDError(SSD_ETOOLARGE) when the shape needs more scratch than that; a smaller `seg` needs less."""
+    _check_inputs(x, dt, A, Bm, Cm, D)
+    shape = make_shape(x, Bm, chunk, seg, flags)
+    rc = lib().ssd_fwd_static_ws(ctypes.byref(shape), _ptr(x), _ptr(dt), _ptr(A), _ptr(Bm), _ptr(Cm),
+                                 _ptr(D), _ptr(h0), _ptr(y), _ptr(h_final), _stream(stream))
+    if rc != SSD_OK:
+        raise SSDError(rc, "ssd_fwd_static_ws")
     return y, h_final
 
 
