@@ -86,8 +86,8 @@ static int make_plan(const ssd_shape_t *s, Plan &pl) {
     if (((size_t)s->H * s->P * pl.esz) % 16 || ((size_t)s->G * s->N * pl.esz) % 16 ||
         ((size_t)pl.x_bs * pl.esz) % 16 || ((size_t)pl.bc_bs * pl.esz) % 16)
         return SSD_EALIGN;
-    pl.use_tc = false;  // tensor-core path is selected in ssd_tc.cu once available
-    pl.nsl = pl.hpg;    // CUDA-core path: one head per dB/dC partial slice
+    pl.use_tc = tc_supported(s->dtype, s->flags, s->P, s->N, s->chunk, pl.hpg);
+    pl.nsl = pl.hpg;    // CUDA-core dB/dC kernels: one head per partial slice
     return SSD_OK;
 }
 
@@ -216,11 +216,14 @@ static int forward_impl(const ssd_shape_t *shape, const void *x, const float *dt
     fill_params(pl, lo, ws, sp);
     sp.x = x; sp.dt = dt; sp.A = A; sp.Bm = Bm; sp.Cm = Cm; sp.D = D; sp.y = y;
     SSD_TRY(cudaMemsetAsync(sp.status, 0, 256, st));
+    TcMaps maps;
+    if (pl.use_tc && !tc_make_maps(sp, maps)) return SSD_ECUDA;
     const long long PN = (long long)pl.P * pl.N;
     for (int k = 0; k < pl.nseg; ++k) {
         set_segment(pl, k, sp);
         SSD_LAUNCH(KIND_CUMSUM, launch_chunk_cumsum(sp, st));
-        SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
+        if (pl.use_tc) SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_tc(sp, maps, STATE_MODE_FWD, st));
+        else SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
         const float *init = (k == 0) ? h0 : sp.hcarry;
         float *bnd = boundary ? boundary + (size_t)k * pl.H * PN : nullptr;
         SSD_LAUNCH(KIND_STATE_PASS_FWD, launch_state_pass_fwd(sp, init, (long long)pl.H * PN, bnd, (long long)pl.nseg * pl.H * PN,
@@ -337,16 +340,20 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
     sp.x = x; sp.dt = dt; sp.A = A; sp.Bm = Bm; sp.Cm = Cm; sp.D = D; sp.dy = dy;
     sp.dx = dx; sp.ddt = ddt; sp.dB = dB; sp.dC = dC;
     SSD_TRY(cudaMemsetAsync(sp.status, 0, 256, st));
+    TcMaps maps;
+    if (pl.use_tc && !tc_make_maps(sp, maps)) return SSD_ECUDA;
     const long long PN = (long long)pl.P * pl.N;
     for (int k = pl.nseg - 1; k >= 0; --k) {
         set_segment(pl, k, sp);
         // Recompute_Forward: chunk-entry states of segment k from the stored boundary state
         SSD_LAUNCH(KIND_CUMSUM, launch_chunk_cumsum(sp, st));
-        SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
+        if (pl.use_tc) SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_tc(sp, maps, STATE_MODE_FWD, st));
+        else SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
         SSD_LAUNCH(KIND_STATE_PASS_FWD, launch_state_pass_fwd(sp, boundary + (size_t)k * pl.H * PN, (long long)pl.nseg * pl.H * PN,
                                       nullptr, 0, nullptr, pl.use_tc, st));
         // Backward through the segment; dh enters from the right, leaves to the left
-        SSD_LAUNCH(KIND_DSTATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_DSTATE, st));
+        if (pl.use_tc) SSD_LAUNCH(KIND_DSTATE, launch_chunk_state_tc(sp, maps, STATE_MODE_DSTATE, st));
+        else SSD_LAUNCH(KIND_DSTATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_DSTATE, st));
         const float *ginit = (k == pl.nseg - 1) ? dh_final : sp.gcarry;
         float *gleft = (k == 0 && dh0) ? dh0 : sp.gcarry;
         SSD_LAUNCH(KIND_STATE_PASS_BWD, launch_state_pass_bwd(sp, ginit, gleft, pl.use_tc, st));

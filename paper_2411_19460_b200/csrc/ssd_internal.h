@@ -1,5 +1,6 @@
 // Internal declarations shared by the host driver and the kernel files of libssd.
 #pragma once
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -61,6 +62,15 @@ cudaError_t launch_masked_product_simt(const SegParams &p, int dtype, int mode, 
 cudaError_t launch_bwd_finish(const SegParams &p, cudaStream_t st);
 cudaError_t launch_reduce_dbdc(const SegParams &p, int dtype, cudaStream_t st);
 cudaError_t launch_final_dAdD(const SegParams &p, float *dA, float *dD, cudaStream_t st);
+
+// ssd_tc.cu : tensor-core (tcgen05 / TMEM / TMA) kernels, bf16 I/O
+struct TcMaps {
+    CUtensorMap x, dy, Bm, Cm;  // [B][L][H*64] / [B][L][G*128], box 64 x 128 rows
+    CUtensorMap Hbf, Gbf;       // bf16 chunk states as [rows][128], box 64 x 64 rows
+};
+bool tc_supported(int dtype, int flags, int P, int N, int Q, int hpg);
+bool tc_make_maps(const SegParams &p, TcMaps &m);
+cudaError_t launch_chunk_state_tc(const SegParams &p, const TcMaps &m, int mode, cudaStream_t st);
 
 enum { STATE_MODE_FWD = 0, STATE_MODE_DSTATE = 1 };
 // kernel kinds, for the launch counter and the optional per-kind timing

@@ -1,0 +1,192 @@
+// Tensor-core kernels of libssd for bf16 I/O on sm_100a: tcgen05.mma with fp32 accumulators in
+// TMEM, operands staged in shared memory by TMA (128-byte swizzle), epilogues through tcgen05.ld.
+// Shapes served: P = 64, N = 128, chunk Q = 256, an even number of heads per group.
+//
+// Notation per (batch b, head h), chunk of Q steps: a_t = dt_t*A_h, cs_t = inclusive cumsum of a
+// inside the chunk, H_in = state entering the chunk, Gout = dLoss/d(state leaving the chunk); all
+// of it is Eq. 1 of the paper regrouped by chunks.
+#include <cstring>
+
+#include "ssd_internal.h"
+#include "ssd_sm100.cuh"
+
+namespace ssd {
+
+using namespace sm100;
+
+// ------------------------------------------------------------------ host: tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// bf16 tensor [dim2][dim1][dim0] (dim0 contiguous), box {64, box_rows, 1}, 128-byte swizzle.
+static bool make_map3(CUtensorMap *m, const void *ptr, uint64_t dim0, uint64_t dim1, uint64_t dim2,
+                      uint64_t stride1_elems, uint64_t stride2_elems, uint32_t box_rows) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {dim0, dim1, dim2};
+    cuuint64_t strides[2] = {stride1_elems * 2, stride2_elems * 2};
+    cuuint32_t box[3] = {64, box_rows, 1};
+    cuuint32_t es[3] = {1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, es,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool tc_supported(int dtype, int flags, int P, int N, int Q, int hpg) {
+    return dtype == SSD_DTYPE_BF16 && !(flags & SSD_FLAG_FORCE_SIMT) && P == 64 && N == 128 && Q == 256 &&
+           (hpg % 2) == 0 && encode_fn() != nullptr;
+}
+
+// Builds the tensor maps of one API call.  x/dy/Bm/Cm may be null when the call does not use them.
+bool tc_make_maps(const SegParams &p, TcMaps &m) {
+    memset(&m, 0, sizeof(m));
+    const uint64_t HP = (uint64_t)p.H * 64, GN = (uint64_t)p.G * 128;
+    bool ok = true;
+    if (p.x) ok = ok && make_map3(&m.x, p.x, HP, p.L, p.B, HP, p.x_bs, 128);
+    if (p.dy) ok = ok && make_map3(&m.dy, p.dy, HP, p.L, p.B, HP, p.x_bs, 128);
+    if (p.Bm) ok = ok && make_map3(&m.Bm, p.Bm, GN, p.L, p.B, GN, p.bc_bs, 128);
+    if (p.Cm) ok = ok && make_map3(&m.Cm, p.Cm, GN, p.L, p.B, GN, p.bc_bs, 128);
+    // bf16 state copies viewed as [B*(ncs+1)*H*64 rows][128]
+    const uint64_t srows = (uint64_t)p.B * (p.ncs + 1) * p.H * 64;
+    if (p.Hbf) ok = ok && make_map3(&m.Hbf, p.Hbf, 128, srows, 1, 128, srows * 128, 64);
+    if (p.Gbf) ok = ok && make_map3(&m.Gbf, p.Gbf, 128, srows, 1, 128, srows * 128, 64);
+    return ok;
+}
+
+// ------------------------------------------------------------------ a2 / a8: chunk state on tensor cores
+// One CTA per (chunk, head pair, batch): D[128 = (head-in-pair, p)][N] = sum_s Xw[s][(h2,p)] * V[s][n]
+//   mode FWD   : X = x,  V = Bm, w_s = exp(cs_last - cs_s) dt_s  -> Hst slot c+1   (S_c)
+//   mode DSTATE: X = dy, V = Cm, w_t = exp(cs_t)                 -> Gst slot c     (E_c)
+// Both operands are MN-major straight from the row-major tensors (rows = time = the contraction
+// index).  The per-row weight is multiplied into the X tile in shared memory (it is uniform along
+// a row, so the swizzle does not matter), the two K halves are separate TMA transactions so the
+// second lands while the first is scaled and multiplied.
+constexpr int CS_THREADS = 128;
+constexpr int CS_SMEM = 2 * (2 * 16384 + 2 * 16384) + 1024;  // two K halves x (X pair 32 KB + V 32 KB) + align
+
+__global__ void __launch_bounds__(CS_THREADS)
+k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
+                 const __grid_constant__ CUtensorMap tmV) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    // [half][ X head0 16K | X head1 16K | V n0-63 16K | V n64-127 16K ]
+    __shared__ uint64_t bar_half[2], bar_mma;
+    __shared__ uint32_t tmem_base, abort_flag;
+    __shared__ float wsm[2][256];
+
+    const int c = blockIdx.x, hp = blockIdx.y, b = blockIdx.z;
+    const int h0 = hp * 2, g = h0 / p.hpg;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tok0 = p.t0 + c * 256;
+
+    if (tid == 0) {
+        mbar_init(&bar_half[0], 1);
+        mbar_init(&bar_half[1], 1);
+        mbar_init(&bar_mma, 1);
+        abort_flag = 0;
+        fence_barrier_init();
+        for (int half = 0; half < 2; ++half) {
+            unsigned char *st = smem + half * 65536;
+            mbar_arrive_expect_tx(&bar_half[half], 65536);
+            tma_load_3d(st, &tmX, &bar_half[half], h0 * 64, tok0 + half * 128, b);
+            tma_load_3d(st + 16384, &tmX, &bar_half[half], h0 * 64 + 64, tok0 + half * 128, b);
+            tma_load_3d(st + 32768, &tmV, &bar_half[half], g * 128, tok0 + half * 128, b);
+            tma_load_3d(st + 49152, &tmV, &bar_half[half], g * 128 + 64, tok0 + half * 128, b);
+        }
+    }
+    if (warp == 0) tmem_alloc(&tmem_base, 128);
+    // per-row weights of both heads
+    for (int i = tid; i < 512; i += CS_THREADS) {
+        const int hh = i >> 8, t = i & 255;
+        const float *csb = p.cs + ((((size_t)b * p.H + h0 + hh) * p.ncs + c) << 8);
+        float w;
+        if (mode == STATE_MODE_FWD) {
+            const float *dtb = p.dtT + ((((size_t)b * p.H + h0 + hh) * p.ncs + c) << 8);
+            w = __expf(fminf(csb[255] - csb[t], 0.f)) * dtb[t];
+        } else {
+            w = __expf(csb[t]);
+        }
+        wsm[hh][t] = w;
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tm = tmem_base;
+    const uint32_t idesc = umma_idesc_bf16(128, 128, true, true);
+
+    for (int half = 0; half < 2; ++half) {
+        unsigned char *st = smem + half * 65536;
+        mbar_wait(&bar_half[half], 0, &abort_flag, p.status);
+        // scale the X pair: 2 heads x 128 rows x 8 chunks of 16 B
+        for (int q = tid; q < 2048; q += CS_THREADS) {
+            const int hh = q >> 10, row = (q >> 3) & 127;
+            const float w = wsm[hh][half * 128 + row];
+            uint4 *ptr = reinterpret_cast<uint4 *>(st + (size_t)q * 16);
+            uint4 v = *ptr;
+            __nv_bfloat162 *e = reinterpret_cast<__nv_bfloat162 *>(&v);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                float2 f = __bfloat1622float2(e[k]);
+                e[k] = __floats2bfloat162_rn(f.x * w, f.y * w);
+            }
+            *ptr = v;
+        }
+        fence_proxy_async_smem();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after_sync();
+            const uint32_t sa = smem_u32(st), sb = smem_u32(st + 32768);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint64_t ad = umma_desc_sw128(sa + ks * 2048, 16384, 1024);
+                const uint64_t bd = umma_desc_sw128(sb + ks * 2048, 16384, 1024);
+                umma_bf16(tm, ad, bd, idesc, (half | ks) ? 1u : 0u);
+            }
+            if (half == 1) umma_commit(&bar_mma);
+        }
+    }
+    mbar_wait(&bar_mma, 0, &abort_flag, p.status);
+    tc_fence_after_sync();
+    {
+        const int hh = tid >> 6, pp = tid & 63;
+        const int slot = (mode == STATE_MODE_FWD) ? c + 1 : c;
+        float *base = (mode == STATE_MODE_FWD) ? p.Hst : p.Gst;
+        float *out = base + ((((size_t)b * (p.ncs + 1) + slot) * p.H + h0 + hh) * 64 + pp) * 128;
+#pragma unroll
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+            float v[32];
+            tmem_ld32(tm + ((uint32_t)(warp * 32) << 16) + c0, v);
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+                *reinterpret_cast<float4 *>(out + c0 + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tm, 128);
+}
+
+cudaError_t launch_chunk_state_tc(const SegParams &p, const TcMaps &m, int mode, cudaStream_t st) {
+    cudaError_t e = cudaFuncSetAttribute(k_chunk_state_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, CS_SMEM);
+    if (e != cudaSuccess) return e;
+    dim3 grid(p.nc, p.H / 2, p.B);
+    if (mode == STATE_MODE_FWD) k_chunk_state_tc<<<grid, CS_THREADS, CS_SMEM, st>>>(p, mode, m.x, m.Bm);
+    else k_chunk_state_tc<<<grid, CS_THREADS, CS_SMEM, st>>>(p, mode, m.dy, m.Cm);
+    return cudaGetLastError();
+}
+
+}  // namespace ssd
