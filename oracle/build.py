@@ -16,8 +16,9 @@ def build(force: bool = False) -> str:
             and os.path.getmtime(OUT) >= os.path.getmtime(SRC)):
         return OUT
     tmp = OUT + ".tmp.%d" % os.getpid()
-    # no -ffast-math: the oracle must keep IEEE fp64 semantics and the written order
-    cmd = ["gcc", "-O3", "-march=native", "-fopenmp", "-fPIC", "-shared",
+    # no -ffast-math: the oracle must keep IEEE fp64 semantics and the written order;
+    # no -march=native: the built library may be carried to a host with a different CPU
+    cmd = ["gcc", "-O3", "-fopenmp", "-fPIC", "-shared",
            "-std=c11", "-Wall", "-o", tmp, SRC, "-lm"]
     subprocess.run(cmd, check=True)
     os.replace(tmp, OUT)
