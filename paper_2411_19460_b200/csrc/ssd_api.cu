@@ -44,7 +44,7 @@ static void prof_end(ProfEvent *ev, cudaStream_t st) {
 }
 
 struct Layout {
-    size_t status, cs, dtT, Hst, Hbf, hcarry, Gst, Gbf, gcarry, ghdot, ddt_dir, rho, pB, pC, dAp, dDp;
+    size_t status, cs, dtT, Hst, Hbf, hcarry, Gst, Gbf, gcarry, ghdot, ddt_dir, rho, psi, psi2, pB, pC, dAp, dDp;
     size_t total;
 };
 
@@ -112,6 +112,8 @@ static void make_layout(const Plan &pl, int op, Layout &lo) {
         lo.ghdot = take(BH * pl.ncs * 8 * sizeof(float));
         lo.ddt_dir = take(vec);
         lo.rho = take(vec);
+        lo.psi = take(vec);
+        lo.psi2 = take(vec);
         const size_t part = (size_t)pl.B * pl.seg * pl.G * pl.nsl * pl.N * sizeof(float);
         lo.pB = take(part);
         lo.pC = take(part);
@@ -179,6 +181,8 @@ static void fill_params(const Plan &pl, const Layout &lo, void *ws, SegParams &s
     sp.ghdot = (float *)(w + lo.ghdot);
     sp.ddt_dir = (float *)(w + lo.ddt_dir);
     sp.rho = (float *)(w + lo.rho);
+    sp.psi = (float *)(w + lo.psi);
+    sp.psi2 = (float *)(w + lo.psi2);
     sp.pB = (float *)(w + lo.pB);
     sp.pC = (float *)(w + lo.pC);
     sp.dAp = (float *)(w + lo.dAp);
@@ -190,6 +194,16 @@ static void set_segment(const Plan &pl, int k, SegParams &sp) {
     const int len = (pl.L - sp.t0 < pl.seg) ? pl.L - sp.t0 : pl.seg;
     sp.nc = len / pl.Q;
     sp.c0 = sp.t0 / pl.Q;
+    // Head ranges per group for the scan kernels: enough CTAs for about two waves of the 148 SMs,
+    // at least two heads per CTA so the shared score tile is reused.  Their outputs are per head,
+    // so this choice cannot change any result bit.
+    const int base = sp.nc * 2 * pl.G * pl.B;
+    int want = (296 + base - 1) / base;
+    const int cap = pl.hpg >= 2 ? pl.hpg / 2 : 1;
+    if (want > cap) want = cap;
+    if (want < 1) want = 1;
+    const int hps = (pl.hpg + want - 1) / want;
+    sp.nsplit_scan = (pl.hpg + hps - 1) / hps;
 }
 
 static int forward_impl(const ssd_shape_t *shape, const void *x, const float *dt, const float *A,
@@ -228,7 +242,8 @@ static int forward_impl(const ssd_shape_t *shape, const void *x, const float *dt
         float *bnd = boundary ? boundary + (size_t)k * pl.H * PN : nullptr;
         SSD_LAUNCH(KIND_STATE_PASS_FWD, launch_state_pass_fwd(sp, init, (long long)pl.H * PN, bnd, (long long)pl.nseg * pl.H * PN,
                                       (k == pl.nseg - 1) ? h_final : nullptr, pl.use_tc, st));
-        SSD_LAUNCH(KIND_SCAN_FWD, launch_masked_product_simt(sp, pl.dtype, MP_FWD, st));
+        if (pl.use_tc) SSD_LAUNCH(KIND_SCAN_FWD, launch_scan_tc(sp, maps, SC_FWD, st));
+        else SSD_LAUNCH(KIND_SCAN_FWD, launch_masked_product_simt(sp, pl.dtype, MP_FWD, st));
     }
     return SSD_OK;
 }
@@ -357,7 +372,8 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
         const float *ginit = (k == pl.nseg - 1) ? dh_final : sp.gcarry;
         float *gleft = (k == 0 && dh0) ? dh0 : sp.gcarry;
         SSD_LAUNCH(KIND_STATE_PASS_BWD, launch_state_pass_bwd(sp, ginit, gleft, pl.use_tc, st));
-        SSD_LAUNCH(KIND_BWD_DX, launch_masked_product_simt(sp, pl.dtype, MP_BWD_DX, st));
+        if (pl.use_tc) SSD_LAUNCH(KIND_BWD_DX, launch_scan_tc(sp, maps, SC_DX, st));
+        else SSD_LAUNCH(KIND_BWD_DX, launch_masked_product_simt(sp, pl.dtype, MP_BWD_DX, st));
         SSD_LAUNCH(KIND_BWD_DC, launch_masked_product_simt(sp, pl.dtype, MP_DC, st));
         SSD_LAUNCH(KIND_BWD_DB, launch_masked_product_simt(sp, pl.dtype, MP_DB, st));
         SSD_LAUNCH(KIND_BWD_FINISH, launch_bwd_finish(sp, st));

@@ -19,6 +19,7 @@ struct SegParams {
     int ncs;       // chunk capacity of the workspace (chunks of a full segment)
     int nct;       // chunks in the whole sequence (L / Q)
     int nsl;       // head slices per group in the dB/dC partial buffers
+    int nsplit_scan;  // head ranges per group in the tensor-core scan kernels (no effect on results)
     int64_t x_bs, dt_bs, bc_bs;  // batch strides, elements
 
     // caller tensors
@@ -37,9 +38,11 @@ struct SegParams {
     __nv_bfloat16 *Gbf;    // [B,ncs+1,H,P,N] bf16 copy of Gst (tensor-core path)
     float *hcarry;         // [B,H,P,N]     state handed from segment to segment (forward)
     float *gcarry;         // [B,H,P,N]     state gradient handed right-to-left (backward)
-    float *ghdot;          // [B,H,ncs,8]   partial sums of <Gout_c, Hout_c>
+    float *ghdot;          // [B,H,ncs,8]   partial sums of exp(cs_last) <Gout_c, H_in,c>
     float *ddt_dir;        // [B,H,ncs,Q]   direct part of ddt
-    float *rho;            // [B,H,ncs,Q]   dy_t . (y_t - D x_t)
+    float *rho;            // [B,H,ncs,Q]   dy_t . (y_t - D x_t)   = C_t . dC_t of this head
+    float *psi;            // [B,H,ncs,Q]   B_t . (intra-chunk part of this head's dB_t)
+    float *psi2;           // [B,H,ncs,Q]   B_t . (inter-chunk part of this head's dB_t)
     float *pB, *pC;        // [B,seg,G,nsl,N] per-head-slice partial dB / dC
     float *dAp;            // [B,H,nct]     per-chunk partial of dA
     float *dDp;            // [B,H,nct,4]   per-row-tile partial of dD
@@ -71,6 +74,9 @@ struct TcMaps {
 bool tc_supported(int dtype, int flags, int P, int N, int Q, int hpg);
 bool tc_make_maps(const SegParams &p, TcMaps &m);
 cudaError_t launch_chunk_state_tc(const SegParams &p, const TcMaps &m, int mode, cudaStream_t st);
+// ssd_tc_scan.cu : y (SC_FWD) or dx, ddt_direct, dD partials (SC_DX)
+cudaError_t launch_scan_tc(const SegParams &p, const TcMaps &m, int mode, cudaStream_t st);
+enum { SC_FWD = 0, SC_DX = 1 };
 
 enum { STATE_MODE_FWD = 0, STATE_MODE_DSTATE = 1 };
 // kernel kinds, for the launch counter and the optional per-kind timing

@@ -204,8 +204,8 @@ cudaError_t launch_state_pass_fwd(const SegParams &p, const float *init, long lo
 // ------------------------------------------------------------------ a9: backward state passing
 // Gslot[nc] = gradient arriving from the segment on the right (or dh_final); going left,
 // Gslot[c] = exp(cs_last,c) Gslot[c+1] + E_c.  Gslot[c+1] is Gout of chunk c.  Also emits, per chunk,
-// the partial sums of <Gout_c, Hout_c> (one per CTA, summed later in a fixed order), which is the
-// value the within-chunk suffix scan of da starts from.
+// the partial sums of exp(cs_last,c) <Gout_c, H_in,c> (one per CTA, summed later in a fixed order):
+// the part of da_t that couples the gradient from the right with the state from the left.
 __global__ void __launch_bounds__(256)
 k_state_pass_bwd(SegParams p, const float *init, float *left_out, int want_bf16) {
     __shared__ float red[2][8];
@@ -220,8 +220,9 @@ k_state_pass_bwd(SegParams p, const float *init, float *left_out, int want_bf16)
     for (int c = p.nc; c >= 0; --c) {
         const size_t so = slot_off(p, b, c, h) + e;
         if (c < p.nc) {
-            // carry is Gout of chunk c here (slot c+1); Hst slot c+1 is the state leaving chunk c
-            const float4 hv = *reinterpret_cast<const float4 *>(p.Hst + slot_off(p, b, c + 1, h) + e);
+            // carry is Gout of chunk c here (slot c+1); Hst slot c is the state entering chunk c
+            const float decay = expf(csl[(size_t)c * p.Q]);
+            const float4 hv = *reinterpret_cast<const float4 *>(p.Hst + so);
             float part = carry.x * hv.x;
             part = fmaf(carry.y, hv.y, part);
             part = fmaf(carry.z, hv.z, part);
@@ -234,9 +235,8 @@ k_state_pass_bwd(SegParams p, const float *init, float *left_out, int want_bf16)
                 float s = 0.f;
 #pragma unroll
                 for (int w = 0; w < 8; ++w) s += red[c & 1][w];
-                p.ghdot[((((size_t)b * p.H + h) * p.ncs + c) << 3) + blockIdx.x] = s;
+                p.ghdot[((((size_t)b * p.H + h) * p.ncs + c) << 3) + blockIdx.x] = decay * s;
             }
-            const float decay = expf(csl[(size_t)c * p.Q]);
             const float4 ev = *reinterpret_cast<const float4 *>(p.Gst + so);
             carry.x = fmaf(decay, carry.x, ev.x);
             carry.y = fmaf(decay, carry.y, ev.y);
@@ -273,9 +273,11 @@ cudaError_t launch_state_pass_bwd(const SegParams &p, const float *init, float *
 // MP_BWD_DX rows s: Rv=B, Cv=C, V=dy, mask=[t>=s] e^{cs_t-cs_s},     S=Gout[p][n], off e^{cs_last-cs_s}
 //           dx_s = D dy_s + dt_s acc ; ddt_direct_s = <x_s, acc> ; dD partial = sum dy x
 // MP_DC     rows t: Rv=dy, Cv=x, V=B, mask as MP_FWD,               S=H_in^T[n][p], off e^{cs_t}
-//           per-head dC_t = acc ; rho_t = <C_t, acc>
+//           per-head dC_t = acc ; rho_t = <C_t, acc>   (= dy_t . (y_t - D x_t))
 // MP_DB     rows s: Rv=x, Cv=dy, V=C, mask=[t>=s] e^{cs_t-cs_s} dt_s, S=Gout^T[n][p], off dt_s e^{cs_last-cs_s}
-//           per-head dB_s = acc
+//           per-head dB_s = acc ; psi_s = <B_s, intra-chunk part>, psi2_s = <B_s, inter-chunk part>
+//           (psi + psi2 = dt_s ddt_direct_s, but psi is built from the same masked products as rho,
+//           so rho - psi cancels cleanly in the suffix sums of da)
 template <typename T, int NS, int MODE>
 __global__ void __launch_bounds__(256) k_masked_product_simt(SegParams p) {
     constexpr int KD = (MODE < 2) ? NS : 64;
@@ -382,6 +384,19 @@ __global__ void __launch_bounds__(256) k_masked_product_simt(SegParams p) {
         __syncthreads();
     }
 
+    // dB rows: psi_intra_s = <B_s, intra-chunk part of dB_s>, taken before the inter-chunk term is added
+    float dot_intra[4] = {0.f, 0.f, 0.f, 0.f};
+    if (MODE == MP_DB) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+#pragma unroll
+            for (int j = 0; j < NJ; ++j)
+                dot_intra[i] = fmaf(ldf(bc_base_B + (size_t)(r0 + ty * 4 + i) * GN + tx + 16 * j), acc[i][j], dot_intra[i]);
+#pragma unroll
+            for (int off = 8; off > 0; off >>= 1) dot_intra[i] += __shfl_xor_sync(0xffffffffu, dot_intra[i], off);
+        }
+    }
+
     // inter-chunk term
     const float *St = (MODE == MP_FWD || MODE == MP_DC) ? p.Hst + slot_off(p, b, c, h)
                                                         : p.Gst + slot_off(p, b, c + 1, h);
@@ -477,6 +492,7 @@ __global__ void __launch_bounds__(256) k_masked_product_simt(SegParams p) {
         }
     } else {
         // per-head partial dC / dB rows: [B, seg, G, nsl, N]
+        // (acc here already holds intra-chunk + inter-chunk parts; dot_intra was taken before)
         float *pb = (MODE == MP_DC) ? p.pC : p.pB;
         const int sl = (h % p.hpg) / (p.hpg / p.nsl);
         const size_t segcap = (size_t)p.ncs * Q;
@@ -490,12 +506,17 @@ __global__ void __launch_bounds__(256) k_masked_product_simt(SegParams p) {
             for (int j = 0; j < NJ; ++j) {
                 const int nn = tx + 16 * j;
                 row[nn] = acc[i][j];
-                if (MODE == MP_DC) dot = fmaf(ldf(bc_base_C + (size_t)r * GN + nn), acc[i][j], dot);
+                dot = fmaf(ldf((MODE == MP_DC ? bc_base_C : bc_base_B) + (size_t)r * GN + nn), acc[i][j], dot);
             }
-            if (MODE == MP_DC) {
 #pragma unroll
-                for (int off = 8; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
-                if (tx == 0) p.rho[vec_off(p, b, h, c) + r] = dot;
+            for (int off = 8; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+            if (tx == 0) {
+                if (MODE == MP_DC) {
+                    p.rho[vec_off(p, b, h, c) + r] = dot;
+                } else {
+                    p.psi[vec_off(p, b, h, c) + r] = dot_intra[i];
+                    p.psi2[vec_off(p, b, h, c) + r] = dot - dot_intra[i];
+                }
             }
         }
     }
@@ -532,9 +553,15 @@ cudaError_t launch_masked_product_simt(const SegParams &p, int dtype, int mode, 
 }
 
 // ------------------------------------------------------------------ a12 + a13: da, ddt, dA partial
-// One warp per (b, h, chunk).  da_t = sum_{t'>=t in chunk} (rho_t' - dt_t' ddt_direct_t') + <Gout,Hout>
-// (reverse scan: serial inside a lane, warp-shuffle across lanes), ddt = ddt_direct + A da,
-// dA partial = sum_t dt_t da_t.
+// One warp per (b, h, chunk).  With g_t = dLoss/dh_t and h_{t-1} split into their intra-chunk and
+// inter-chunk parts, da_t = exp(a_t) <g_t, h_{t-1}> is the sum of four terms, none of which
+// subtracts large numbers when the decay inside a chunk is strong:
+//   sum_{t'>=t} (rho_intra_t' - psi_t')     pairs (t' >= t > s) inside the chunk
+// + sum_{t'>=t} rho_inter_t'                outputs at/after t reading the chunk-entry state
+// + sum_{s<t}   psi2_s                      inputs before t feeding the chunk-exit gradient
+// + exp(cs_last) <Gout, H_in>
+// (rho = rho_intra + rho_inter is stored as one vector).  Suffix/prefix scans: serial inside a lane,
+// warp shuffles across lanes.  Then ddt = ddt_direct + A da, dA partial = sum_t dt_t da_t.
 __global__ void __launch_bounds__(128) k_bwd_finish(SegParams p) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int c = blockIdx.x * 4 + warp, h = blockIdx.y, b = blockIdx.z;
@@ -544,15 +571,14 @@ __global__ void __launch_bounds__(128) k_bwd_finish(SegParams p) {
     const int ngh = p.P * p.N / 1024;
     float gh = 0.f;
     for (int i = 0; i < ngh; ++i) gh += p.ghdot[((((size_t)b * p.H + h) * p.ncs + c) << 3) + i];
-    float v[8], dtv[8], dd[8], sfx[8];
+    float dtv[8], dd[8], sfx[8], pfx[8];
     float run = 0.f;
 #pragma unroll
     for (int j = 7; j >= 0; --j)
         if (j < per) {
             dtv[j] = p.dtT[vo + j];
             dd[j] = p.ddt_dir[vo + j];
-            v[j] = p.rho[vo + j] - dtv[j] * dd[j];
-            run += v[j];
+            run += p.rho[vo + j] - p.psi[vo + j];
             sfx[j] = run;
         }
     float incl = run;
@@ -563,13 +589,29 @@ __global__ void __launch_bounds__(128) k_bwd_finish(SegParams p) {
     }
     float excl = __shfl_down_sync(0xffffffffu, incl, 1);
     if (lane == 31) excl = 0.f;
+    // exclusive prefix of psi2
+    float prun = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        if (j < per) {
+            pfx[j] = prun;
+            prun += p.psi2[vo + j];
+        }
+    float pincl = prun;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const float t = __shfl_up_sync(0xffffffffu, pincl, off);
+        if (lane >= off) pincl += t;
+    }
+    float pexcl = __shfl_up_sync(0xffffffffu, pincl, 1);
+    if (lane == 0) pexcl = 0.f;
     const float Ah = __ldg(p.A + h);
     const size_t tok0 = (size_t)p.t0 + (size_t)c * Q + (size_t)lane * per;
     float sA = 0.f;
 #pragma unroll
     for (int j = 0; j < 8; ++j)
         if (j < per) {
-            const float da = (sfx[j] + excl) + gh;
+            const float da = ((sfx[j] + excl) + (pfx[j] + pexcl)) + gh;
             p.ddt[(size_t)b * p.dt_bs + (tok0 + j) * p.H + h] = fmaf(Ah, da, dd[j]);
             sA = fmaf(dtv[j], da, sA);
         }

@@ -72,13 +72,18 @@ def chunked_bwd(x, dt, A, Bm, Cm, D, h0, dy, dh_final, Q):
                 dx[b, sl, h] = D[h] * dyc + dtc[:, None] * u
                 ddt_direct = np.sum(xc * u, axis=1)
                 W = (dyc @ xc.T) * Lm * dtc[None, :]
-                dBh = W.T @ Cc + (dtc * wl)[:, None] * (xc @ Gout)
+                dB_intra, dB_inter = W.T @ Cc, (dtc * wl)[:, None] * (xc @ Gout)
                 dCh = W @ Bc + np.exp(cs)[:, None] * (dyc @ Hs[c])
-                dB[b, sl, g] += dBh
+                dB[b, sl, g] += dB_intra + dB_inter
                 dC[b, sl, g] += dCh
+                # da_t = exp(a_t) <g_t, h_{t-1}> split by intra-/inter-chunk parts of g_t and h_{t-1}:
+                # suffix sum of (rho - psi) [pairs t' >= t > s, and outputs reading the entry state],
+                # exclusive prefix sum of psi2 [inputs before t feeding Gout], plus e^{cs_last}<Gout,H_in>
                 rho = np.sum(Cc * dCh, axis=1)
-                beta = dtc * ddt_direct
-                da = np.cumsum((rho - beta)[::-1])[::-1] + np.sum(Gout * Hs[c + 1])
+                psi = np.sum(Bc * dB_intra, axis=1)
+                psi2 = np.sum(Bc * dB_inter, axis=1)
+                da = (np.cumsum((rho - psi)[::-1])[::-1] + (np.cumsum(psi2) - psi2)
+                      + np.exp(cs[-1]) * np.sum(Gout * Hs[c]))
                 ddt[b, sl, h] = ddt_direct + A[h] * da
                 dA[h] += np.sum(dtc * da)
                 dD[h] += np.sum(dyc * xc)
