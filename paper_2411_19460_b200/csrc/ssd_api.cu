@@ -87,7 +87,16 @@ static int make_plan(const ssd_shape_t *s, Plan &pl) {
         ((size_t)pl.x_bs * pl.esz) % 16 || ((size_t)pl.bc_bs * pl.esz) % 16)
         return SSD_EALIGN;
     pl.use_tc = tc_supported(s->dtype, s->flags, s->P, s->N, s->chunk, pl.hpg);
-    pl.nsl = pl.hpg;    // CUDA-core dB/dC kernels: one head per partial slice
+    // Partial slices of the dB/dC head sums.  CUDA-core kernels: one head per slice.  Tensor-core
+    // kernels: one slice per CTA head range of at most 16 heads.  A function of H/G only, so the
+    // summation order, and with it every bit of dB/dC, is the same for every segment length.
+    if (pl.use_tc) {
+        const int want = (pl.hpg + 15) / 16;
+        const int hps = (pl.hpg + want - 1) / want;
+        pl.nsl = (pl.hpg + hps - 1) / hps;
+    } else {
+        pl.nsl = pl.hpg;
+    }
     return SSD_OK;
 }
 
@@ -374,8 +383,13 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
         SSD_LAUNCH(KIND_STATE_PASS_BWD, launch_state_pass_bwd(sp, ginit, gleft, pl.use_tc, st));
         if (pl.use_tc) SSD_LAUNCH(KIND_BWD_DX, launch_scan_tc(sp, maps, SC_DX, st));
         else SSD_LAUNCH(KIND_BWD_DX, launch_masked_product_simt(sp, pl.dtype, MP_BWD_DX, st));
-        SSD_LAUNCH(KIND_BWD_DC, launch_masked_product_simt(sp, pl.dtype, MP_DC, st));
-        SSD_LAUNCH(KIND_BWD_DB, launch_masked_product_simt(sp, pl.dtype, MP_DB, st));
+        if (pl.use_tc) {
+            SSD_LAUNCH(KIND_BWD_DC, launch_grad_bc_tc(sp, maps, GB_DC, st));
+            SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_tc(sp, maps, GB_DB, st));
+        } else {
+            SSD_LAUNCH(KIND_BWD_DC, launch_masked_product_simt(sp, pl.dtype, MP_DC, st));
+            SSD_LAUNCH(KIND_BWD_DB, launch_masked_product_simt(sp, pl.dtype, MP_DB, st));
+        }
         SSD_LAUNCH(KIND_BWD_FINISH, launch_bwd_finish(sp, st));
         SSD_LAUNCH(KIND_REDUCE_DBDC, launch_reduce_dbdc(sp, pl.dtype, st));
     }

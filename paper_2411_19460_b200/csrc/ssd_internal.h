@@ -77,6 +77,9 @@ cudaError_t launch_chunk_state_tc(const SegParams &p, const TcMaps &m, int mode,
 // ssd_tc_scan.cu : y (SC_FWD) or dx, ddt_direct, dD partials (SC_DX)
 cudaError_t launch_scan_tc(const SegParams &p, const TcMaps &m, int mode, cudaStream_t st);
 enum { SC_FWD = 0, SC_DX = 1 };
+// ssd_tc_bc.cu : per-slice partial dC, rho (GB_DC) or partial dB, psi, psi2 (GB_DB)
+cudaError_t launch_grad_bc_tc(const SegParams &p, const TcMaps &m, int mode, cudaStream_t st);
+enum { GB_DC = 0, GB_DB = 1 };
 
 enum { STATE_MODE_FWD = 0, STATE_MODE_DSTATE = 1 };
 // kernel kinds, for the launch counter and the optional per-kind timing
