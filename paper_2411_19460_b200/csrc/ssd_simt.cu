@@ -30,55 +30,53 @@ __device__ __forceinline__ size_t vec_off(const SegParams &p, int b, int h, int 
 }
 
 // ------------------------------------------------------------------ a1: chunk cumsum
-// One CTA per (chunk, batch).  dt[b, t, :] rows are staged through shared memory 32 heads at a
-// time so global reads are coalesced; each warp then scans one head: a lane owns Q/32 consecutive
-// steps (serial prefix), lane totals are combined with a warp-shuffle scan.
+// One CTA per (chunk, block of 32 heads, batch).  The dt[b, t, h0..h0+31] rows (128 contiguous
+// bytes each) are staged through shared memory so global reads are coalesced; each warp then scans
+// four heads: a lane owns Q/32 consecutive steps (serial prefix), lane totals are combined with a
+// warp-shuffle scan.
 __global__ void __launch_bounds__(256) k_chunk_cumsum(SegParams p) {
     __shared__ float tile[256][33];
-    const int c = blockIdx.x, b = blockIdx.y;
+    const int c = blockIdx.x, h0 = blockIdx.y * 32, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int Q = p.Q, per = Q >> 5;
     const size_t tok0 = (size_t)p.t0 + (size_t)c * Q;
-    for (int h0 = 0; h0 < p.H; h0 += 32) {
-        const int nh = min(32, p.H - h0);
-        for (int idx = tid; idx < Q * 32; idx += 256) {
-            const int t = idx >> 5, hh = idx & 31;
-            if (hh < nh) tile[t][hh] = __ldg(p.dt + (size_t)b * p.dt_bs + (tok0 + t) * p.H + h0 + hh);
-        }
-        __syncthreads();
-        for (int hh = warp; hh < nh; hh += 8) {
-            const float Ah = __ldg(p.A + h0 + hh);
-            float a[8], d[8];
-            float run = 0.f;
+    const int nh = min(32, p.H - h0);
+    for (int idx = tid; idx < Q * 32; idx += 256) {
+        const int t = idx >> 5, hh = idx & 31;
+        if (hh < nh) tile[t][hh] = __ldg(p.dt + (size_t)b * p.dt_bs + (tok0 + t) * p.H + h0 + hh);
+    }
+    __syncthreads();
+    for (int hh = warp; hh < nh; hh += 8) {
+        const float Ah = __ldg(p.A + h0 + hh);
+        float a[8], d[8];
+        float run = 0.f;
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if (j < per) {
-                    d[j] = tile[lane * per + j][hh];
-                    run += d[j] * Ah;
-                    a[j] = run;
-                }
-            float incl = run;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const float v = __shfl_up_sync(0xffffffffu, incl, off);
-                if (lane >= off) incl += v;
+        for (int j = 0; j < 8; ++j)
+            if (j < per) {
+                d[j] = tile[lane * per + j][hh];
+                run += d[j] * Ah;
+                a[j] = run;
             }
-            float excl = __shfl_up_sync(0xffffffffu, incl, 1);
-            if (lane == 0) excl = 0.f;
-            const size_t o = vec_off(p, b, h0 + hh, c) + (size_t)lane * per;
+        float incl = run;
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if (j < per) {
-                    p.cs[o + j] = a[j] + excl;
-                    p.dtT[o + j] = d[j];
-                }
+        for (int off = 1; off < 32; off <<= 1) {
+            const float v = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += v;
         }
-        __syncthreads();
+        float excl = __shfl_up_sync(0xffffffffu, incl, 1);
+        if (lane == 0) excl = 0.f;
+        const size_t o = vec_off(p, b, h0 + hh, c) + (size_t)lane * per;
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (j < per) {
+                p.cs[o + j] = a[j] + excl;
+                p.dtT[o + j] = d[j];
+            }
     }
 }
 
 cudaError_t launch_chunk_cumsum(const SegParams &p, cudaStream_t st) {
-    k_chunk_cumsum<<<dim3(p.nc, p.B), 256, 0, st>>>(p);
+    k_chunk_cumsum<<<dim3(p.nc, (p.H + 31) / 32, p.B), 256, 0, st>>>(p);
     return cudaGetLastError();
 }
 

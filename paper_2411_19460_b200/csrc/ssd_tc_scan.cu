@@ -11,10 +11,12 @@
 // S = Rows * Cols^T (128 x up to 256, K = N) is computed ONCE with tcgen05.mma into TMEM and stays
 // there in fp32 for every head of the range.  Per head the CTA then runs a three-role pipeline:
 //   producer warp : TMA loads of the head's value rows (x or dy) and its bf16 chunk state
-//   MMA warp      : acc2 = Rows * State^T (K = N), acc1 = sum over 64-column pieces of M_piece * V
-//   4 mask warps  : read S from TMEM, apply the decay mask, round to bf16 and store the piece to
-//                   shared memory (A operand of the next MMA); then the epilogue of the previous
-//                   head from the double-buffered accumulators.
+//   MMA warp      : acc2 = Rows * State^T (K = N), acc1 = M * V (K = up to 256 columns)
+//   8 mask warps  : read S from TMEM, apply the decay mask, round to bf16 and store the masked
+//                   tile M to shared memory (A operand of the next MMA); then, while those MMAs run,
+//                   the epilogue of the previous head from the double-buffered accumulators.
+// One hand-off per head in each direction (mask -> MMA, MMA -> mask): a wait on an mbarrier costs
+// a few hundred cycles even when it is already complete, so the pipeline is kept coarse.
 // The decay mask is factored per 32 x 32 sub-tile: strictly off-diagonal sub-tiles use
 //   e^{cs_t-cs_s} = e^{cs_t-cs_i0} * e^{cs_i0-cs_j1} * e^{cs_j1-cs_s}      (i0 = first row of the row
 // sub-tile, j1 = last column of the column sub-tile), three factors that are each <= 1 because cs
@@ -29,14 +31,17 @@ using namespace sm100;
 
 namespace {
 
-constexpr int SC_THREADS = 192;
+constexpr int SC_THREADS = 320;          // warp 0 producer, warp 1 MMA, warps 2..9 mask + epilogue
 constexpr uint32_t OFF_ROWS = 0;          // 32 KB  [n-half][128 rows][128 B]
 constexpr uint32_t OFF_BX = 32768;        // 64 KB  score columns operand, then two value buffers
 constexpr uint32_t OFF_M = 98304;         // 64 KB  four 16 KB pieces of the masked tile
-constexpr uint32_t OFF_ST = 163840;       // 32 KB  two state buffers [n-half][64 rows][128 B]
-constexpr uint32_t OFF_VEC = 196608;      // per-head vectors, double buffered
+constexpr uint32_t OFF_ST = 163840;       // 16 KB  bf16 chunk state [n-half][64 rows][128 B]
+constexpr uint32_t OFF_OUT = 180224;      // 16 KB  output tile staged for the TMA store
+constexpr uint32_t OFF_XR = 196608;       // 16 KB  SC_DX: the head's x rows of this row block
+constexpr uint32_t OFF_VEC = 212992;      // per-head vectors, double buffered
 constexpr uint32_t VEC_FLOATS = 256 * 3 + 64;
-constexpr uint32_t SC_SMEM = OFF_VEC + 2 * VEC_FLOATS * 4 + 1024;
+constexpr uint32_t OFF_PART = OFF_VEC + 2 * VEC_FLOATS * 4;   // 2 x 136 floats: row halves, warp sums
+constexpr uint32_t SC_SMEM = OFF_PART + 2 * 136 * 4 + 1024;
 
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -45,7 +50,7 @@ __device__ __forceinline__ float ex2f(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ void bar_mask_warps() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void bar_mask_warps() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t *>(&v);
@@ -66,13 +71,13 @@ template <int MODE>
 __global__ void __launch_bounds__(SC_THREADS, 1)
 k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
           const __grid_constant__ CUtensorMap tmCol, const __grid_constant__ CUtensorMap tmV,
-          const __grid_constant__ CUtensorMap tmSt) {
+          const __grid_constant__ CUtensorMap tmSt, const __grid_constant__ CUtensorMap tmOut,
+          const __grid_constant__ CUtensorMap tmXr) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ uint64_t bar_ab, bar_s, xfull[2], hfull[2], xhempty[2], mfull[4], mempty[4], accfull[2],
+    __shared__ uint64_t bar_ab, bar_s, xfull[2], xempty[2], hfull, hempty, xrfull, xrempty, mfull, mempty, accfull[2],
         accempty[2];
     __shared__ uint32_t tmem_base, abort_flag;
-    __shared__ float dred[4];
 
     constexpr bool FWD = (MODE == SC_FWD);
     const int nc = p.nc;
@@ -96,15 +101,16 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
         mbar_init(&bar_s, 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(&xfull[i], 1);
-            mbar_init(&hfull[i], 1);
-            mbar_init(&xhempty[i], 1);
+            mbar_init(&xempty[i], 1 + 256);   // the MMAs (one commit) and the epilogue threads have read it
             mbar_init(&accfull[i], 1);
-            mbar_init(&accempty[i], 128);
+            mbar_init(&accempty[i], 256);
         }
-        for (int i = 0; i < 4; ++i) {
-            mbar_init(&mfull[i], 128);
-            mbar_init(&mempty[i], 1);
-        }
+        mbar_init(&mfull, 256);
+        mbar_init(&mempty, 1);
+        mbar_init(&hfull, 1);
+        mbar_init(&hempty, 1);
+        mbar_init(&xrfull, 1);
+        mbar_init(&xrempty, 256);
         abort_flag = 0;
         fence_barrier_init();
     }
@@ -127,24 +133,23 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                     tma_load_3d(smem + OFF_BX + nh * ncols * 128 + r0 * 128, &tmCol, &bar_ab, g * 128 + nh * 64,
                                 tok0 + colbase + r0, b);
             const int strow = (b * (p.ncs + 1) + slot) * p.H;
-            for (int hi = 0; hi < nheads && hi < 2; ++hi) {
-                mbar_arrive_expect_tx(&hfull[hi], 16384);
-                tma_load_3d(smem + OFF_ST + hi * 16384, &tmSt, &hfull[hi], 0, (strow + h_begin + hi) * 64, 0);
-                tma_load_3d(smem + OFF_ST + hi * 16384 + 8192, &tmSt, &hfull[hi], 64, (strow + h_begin + hi) * 64, 0);
-            }
-            mbar_wait(&bar_s, 0, abortp, p.status);   // score MMAs done: the column operand is dead
             for (int hi = 0; hi < nheads; ++hi) {
                 const int buf = hi & 1, h = h_begin + hi;
-                if (hi >= 2) {
-                    mbar_wait(&xhempty[buf], ((hi >> 1) - 1) & 1, abortp, p.status);
-                    mbar_arrive_expect_tx(&hfull[buf], 16384);
-                    tma_load_3d(smem + OFF_ST + buf * 16384, &tmSt, &hfull[buf], 0, (strow + h) * 64, 0);
-                    tma_load_3d(smem + OFF_ST + buf * 16384 + 8192, &tmSt, &hfull[buf], 64, (strow + h) * 64, 0);
-                }
+                if (hi >= 1) mbar_wait(&hempty, (hi - 1) & 1, abortp, p.status);
+                mbar_arrive_expect_tx(&hfull, 16384);
+                tma_load_3d(smem + OFF_ST, &tmSt, &hfull, 0, (strow + h) * 64, 0);
+                tma_load_3d(smem + OFF_ST + 8192, &tmSt, &hfull, 64, (strow + h) * 64, 0);
+                if (hi == 0) mbar_wait(&bar_s, 0, abortp, p.status);   // score MMAs done: the column operand is dead
+                if (hi >= 2) mbar_wait(&xempty[buf], ((hi >> 1) - 1) & 1, abortp, p.status);
                 mbar_arrive_expect_tx(&xfull[buf], (uint32_t)ncols * 128u);
                 for (int r0 = 0; r0 < ncols; r0 += 128)
                     tma_load_3d(smem + OFF_BX + buf * 32768 + r0 * 128, &tmV, &xfull[buf], h * 64,
                                 tok0 + colbase + r0, b);
+                if (!FWD) {
+                    if (hi >= 1) mbar_wait(&xrempty, (hi - 1) & 1, abortp, p.status);
+                    mbar_arrive_expect_tx(&xrfull, 16384);
+                    tma_load_3d(smem + OFF_XR, &tmXr, &xrfull, h * 64, tok0 + rb * 128, b);
+                }
             }
         }
     } else if (warp == 1) {
@@ -168,132 +173,151 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                 const int buf = hi & 1;
                 const uint32_t acc1 = tm + 256 + buf * 128, acc2 = acc1 + 64;
                 if (hi >= 2) mbar_wait(&accempty[buf], ((hi >> 1) - 1) & 1, abortp, p.status);
-                mbar_wait(&hfull[buf], (hi >> 1) & 1, abortp, p.status);
+                mbar_wait(&hfull, hi & 1, abortp, p.status);
                 tc_fence_after_sync();
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
                     const uint64_t ad = umma_desc_sw128(sRows + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024);
-                    const uint64_t bd = umma_desc_sw128(sSt + buf * 16384 + (kk >> 2) * 8192 + (kk & 3) * 32, 16, 1024);
+                    const uint64_t bd = umma_desc_sw128(sSt + (kk >> 2) * 8192 + (kk & 3) * 32, 16, 1024);
                     umma_bf16(acc2, ad, bd, id3, kk ? 1u : 0u);
                 }
+                umma_commit(&hempty);
                 mbar_wait(&xfull[buf], (hi >> 1) & 1, abortp, p.status);
+                mbar_wait(&mfull, hi & 1, abortp, p.status);
+                tc_fence_after_sync();
                 for (int jj = 0; jj < npieces; ++jj) {
-                    mbar_wait(&mfull[jj], hi & 1, abortp, p.status);
-                    tc_fence_after_sync();
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
                         const uint64_t ad = umma_desc_sw128(sM + jj * 16384 + k * 32, 16, 1024);
                         const uint64_t bd = umma_desc_sw128(sBX + buf * 32768 + (jj * 64 + k * 16) * 128, 8192, 1024);
                         umma_bf16(acc1, ad, bd, id2, (jj | k) ? 1u : 0u);
                     }
-                    umma_commit(&mempty[jj]);
                 }
+                umma_commit(&mempty);
                 umma_commit(&accfull[buf]);
-                umma_commit(&xhempty[buf]);
+                umma_commit(&xempty[buf]);
             }
         }
     } else {
         // ------------------------------------------------------------ mask + epilogue warps
-        const int q = warp & 3;                    // TMEM lane quarter this warp may access
-        const int mt = (warp - 2) * 32 + lane;     // 0..127 among the mask threads
+        // Two warps per TMEM lane quarter: warp (q, half) owns rows 32 q .. 32 q + 31 of the block and
+        // the 32-column sub-tile `half` of every 64-column piece / columns 32 half .. of the accumulators.
+        const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
+        const int mt = (warp - 2) * 32 + lane;     // 0..255 among the mask threads
         const int rl = q * 32 + lane;              // row inside the 128-row block
         const int r = rb * 128 + rl;               // row inside the chunk
         const int isub = r >> 5;
         const uint32_t tlane = (uint32_t)(q * 32) << 16;
         float *vec = reinterpret_cast<float *>(smem + OFF_VEC);
-        const size_t HP = (size_t)p.H * 64;
+        float *part = reinterpret_cast<float *>(smem + OFF_PART);
         float offs_prev = 0.f, dt_prev = 0.f;
 
+        // Epilogue of head hi.  The thread's x (and dy) row comes from the tiles TMA already brought to
+        // shared memory; the output tile is staged in shared memory (128-byte swizzle) and written with
+        // one TMA store, so no global access of this kernel is row-per-thread.
         auto epilogue = [&](int hi, float offs, float dtr) {
             const int buf = hi & 1, h = h_begin + hi;
+            uint4 xq[4], dyq[4];
+            mbar_wait(&xfull[buf], (hi >> 1) & 1, abortp, p.status);
+            if (FWD) {
+                const unsigned char *xrow = smem + OFF_BX + buf * 32768 + (rb * 128 + rl) * 128;
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    xq[k] = *reinterpret_cast<const uint4 *>(xrow + (((half * 4 + k) ^ (rl & 7)) << 4));
+            } else {
+                const unsigned char *dyrow = smem + OFF_BX + buf * 32768 + rl * 128;
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    dyq[k] = *reinterpret_cast<const uint4 *>(dyrow + (((half * 4 + k) ^ (rl & 7)) << 4));
+                mbar_wait(&xrfull, hi & 1, abortp, p.status);
+                const unsigned char *xrow = smem + OFF_XR + rl * 128;
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    xq[k] = *reinterpret_cast<const uint4 *>(xrow + (((half * 4 + k) ^ (rl & 7)) << 4));
+                mbar_arrive(&xrempty);
+            }
+            mbar_arrive(&xempty[buf]);
+            const float Dh = __ldg(p.D + h);
             mbar_wait(&accfull[buf], (hi >> 1) & 1, abortp, p.status);
             tc_fence_after_sync();
-            const float Dh = __ldg(p.D + h);
-            const size_t rowoff = (size_t)b * p.x_bs + (size_t)(tok0 + r) * HP + (size_t)h * 64;
-            const uint4 *xr = reinterpret_cast<const uint4 *>((const __nv_bfloat16 *)p.x + rowoff);
+            float a1[32], a2[32];
+            tmem_ld32_nowait(tm + tlane + 256 + buf * 128 + half * 32, a1);
+            tmem_ld32_nowait(tm + tlane + 320 + buf * 128 + half * 32, a2);
+            tmem_ld_wait32(a1);
+            tmem_ld_wait32(a2);
+            tc_fence_before_sync();
+            mbar_arrive(&accempty[buf]);             // both accumulators are in registers now
             float dd = 0.f, dsum = 0.f;
+            unsigned char *orow = smem + OFF_OUT + rl * 128;
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                float a1[32], a2[32];
-                tmem_ld32(tm + tlane + 256 + buf * 128 + half * 32, a1);
-                tmem_ld32(tm + tlane + 320 + buf * 128 + half * 32, a2);
-                if (FWD) {
-                    uint4 *yr = reinterpret_cast<uint4 *>((__nv_bfloat16 *)p.y + rowoff);
+            for (int k8 = 0; k8 < 4; ++k8) {
+                float xv[8], dyv[8];
+                unpack8(xq[k8], xv);
+                if (!FWD) unpack8(dyq[k8], dyv);
+                uint4 o;
+                uint32_t *ow = reinterpret_cast<uint32_t *>(&o);
 #pragma unroll
-                    for (int k8 = 0; k8 < 4; ++k8) {
-                        float xv[8];
-                        unpack8(__ldg(xr + half * 4 + k8), xv);
-                        uint4 o;
-                        uint32_t *ow = reinterpret_cast<uint32_t *>(&o);
-#pragma unroll
-                        for (int e = 0; e < 8; e += 2) {
-                            const int i = k8 * 8 + e;
-                            const float v0 = fmaf(Dh, xv[e], fmaf(offs, a2[i], a1[i]));
-                            const float v1 = fmaf(Dh, xv[e + 1], fmaf(offs, a2[i + 1], a1[i + 1]));
-                            ow[e >> 1] = pack2(v0, v1);
-                        }
-                        yr[half * 4 + k8] = o;
-                    }
-                } else {
-                    const uint4 *dyr = reinterpret_cast<const uint4 *>((const __nv_bfloat16 *)p.dy + rowoff);
-                    uint4 *dxr = reinterpret_cast<uint4 *>((__nv_bfloat16 *)p.dx + rowoff);
-#pragma unroll
-                    for (int k8 = 0; k8 < 4; ++k8) {
-                        float xv[8], dyv[8];
-                        unpack8(__ldg(xr + half * 4 + k8), xv);
-                        unpack8(__ldg(dyr + half * 4 + k8), dyv);
-                        uint4 o;
-                        uint32_t *ow = reinterpret_cast<uint32_t *>(&o);
-#pragma unroll
-                        for (int e = 0; e < 8; e += 2) {
-                            const int i = k8 * 8 + e;
-                            const float u0 = fmaf(offs, a2[i], a1[i]);
-                            const float u1 = fmaf(offs, a2[i + 1], a1[i + 1]);
-                            dd = fmaf(xv[e], u0, dd);
-                            dd = fmaf(xv[e + 1], u1, dd);
-                            dsum = fmaf(dyv[e], xv[e], dsum);
-                            dsum = fmaf(dyv[e + 1], xv[e + 1], dsum);
-                            ow[e >> 1] = pack2(fmaf(Dh, dyv[e], dtr * u0), fmaf(Dh, dyv[e + 1], dtr * u1));
-                        }
-                        dxr[half * 4 + k8] = o;
+                for (int e = 0; e < 8; e += 2) {
+                    const int i = k8 * 8 + e;
+                    const float u0 = fmaf(offs, a2[i], a1[i]);
+                    const float u1 = fmaf(offs, a2[i + 1], a1[i + 1]);
+                    if (FWD) {
+                        ow[e >> 1] = pack2(fmaf(Dh, xv[e], u0), fmaf(Dh, xv[e + 1], u1));
+                    } else {
+                        dd = fmaf(xv[e], u0, dd);
+                        dd = fmaf(xv[e + 1], u1, dd);
+                        dsum = fmaf(dyv[e], xv[e], dsum);
+                        dsum = fmaf(dyv[e + 1], xv[e + 1], dsum);
+                        ow[e >> 1] = pack2(fmaf(Dh, dyv[e], dtr * u0), fmaf(Dh, dyv[e + 1], dtr * u1));
                     }
                 }
+                *reinterpret_cast<uint4 *>(orow + (((half * 4 + k8) ^ (rl & 7)) << 4)) = o;
             }
-            tc_fence_before_sync();
-            mbar_arrive(&accempty[buf]);
+            float *pp = part + (hi & 1) * 136;
             if (!FWD) {
-                p.ddt_dir[((((size_t)b * p.H + h) * p.ncs + c) << 8) + r] = dd;
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, off);
-                if (lane == 0) dred[warp - 2] = dsum;
-                bar_mask_warps();
+                if (half == 1) pp[rl] = dd;
+                if (lane == 0) pp[128 + (warp - 2)] = dsum;
+            }
+            fence_proxy_async_smem();
+            bar_mask_warps();
+            if (mt == 0) {
+                tma_store_3d(&tmOut, smem + OFF_OUT, h * 64, tok0 + rb * 128, b);
+                tma_store_commit();
+            }
+            if (!FWD) {
+                // the two column halves of a row, and the eight warps' dy.x sums, in a fixed order
+                if (half == 0) p.ddt_dir[((((size_t)b * p.H + h) * p.ncs + c) << 8) + r] = dd + pp[rl];
                 if (mt == 0) {
-                    const float s = ((dred[0] + dred[1]) + dred[2]) + dred[3];
+                    float s = 0.f;
+#pragma unroll
+                    for (int w = 0; w < 8; ++w) s += pp[128 + w];
                     float *dst = p.dDp + (((((size_t)b * p.H + h) * p.nct + p.c0 + c) << 2) + rb * 2);
                     dst[0] = s;
                     dst[1] = 0.f;
                 }
-                bar_mask_warps();
             }
         };
 
+        // cs and dt of the head's 256 steps: one per thread, fetched one head ahead
+        float pre_cs, pre_dt;
+        auto fetch_vec = [&](int h) {
+            const size_t vo = (((size_t)b * p.H + h) * p.ncs + c) << 8;
+            pre_cs = __ldg(p.cs + vo + mt);
+            pre_dt = __ldg(p.dtT + vo + mt);
+        };
+        fetch_vec(h_begin);
+
         for (int hi = 0; hi < nheads; ++hi) {
-            const int h = h_begin + hi;
             float *cs2 = vec + (hi & 1) * VEC_FLOATS, *cf = cs2 + 256, *dtv = cs2 + 512, *blk = cs2 + 768;
-            // ---- per-head vectors
-            {
-                const size_t vo = (((size_t)b * p.H + h) * p.ncs + c) << 8;
-                cs2[mt] = p.cs[vo + mt] * kLog2e;
-                cs2[mt + 128] = p.cs[vo + mt + 128] * kLog2e;
-                dtv[mt] = p.dtT[vo + mt];
-                dtv[mt + 128] = p.dtT[vo + mt + 128];
-            }
+            cs2[mt] = pre_cs * kLog2e;
+            dtv[mt] = pre_dt;
+            if (hi + 1 < nheads) fetch_vec(h_begin + hi + 1);
+            if (mt == 0) tma_store_wait_read();   // the staged tile of the last store may be overwritten after the barrier
             bar_mask_warps();
-#pragma unroll
-            for (int w = 0; w < 2; ++w) {
-                const int t = mt + w * 128;
-                cf[t] = FWD ? ex2f(cs2[t | 31] - cs2[t]) * dtv[t] : ex2f(cs2[t] - cs2[t & ~31]);
-            }
+            cf[mt] = FWD ? ex2f(cs2[mt | 31] - cs2[mt]) * dtv[mt] : ex2f(cs2[mt] - cs2[mt & ~31]);
             if (mt < 64) {
                 const int i = mt >> 3, j = mt & 7;   // blk[i][j] = e^{cs[32 i] - cs[32 j + 31]}, j < i
                 blk[mt] = (j < i) ? ex2f(cs2[32 * i] - cs2[32 * j + 31]) : 0.f;
@@ -304,35 +328,43 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             const float offs = FWD ? ex2f(csr) : ex2f(cs2[255] - csr);
             const float dtr = dtv[r];
 
-            if (hi == 0) {
-                mbar_wait(&bar_s, 0, abortp, p.status);
-                tc_fence_after_sync();
-            }
-            // ---- masked pieces
-            for (int jj = 0; jj < npieces; ++jj) {
-                if (hi >= 1) mbar_wait(&mempty[jj], (hi - 1) & 1, abortp, p.status);
-                unsigned char *mrow = smem + OFF_M + jj * 16384 + rl * 128;
+            if (hi == 0) mbar_wait(&bar_s, 0, abortp, p.status);
+            else mbar_wait(&mempty, (hi - 1) & 1, abortp, p.status);   // MMAs of the previous head have read M
+            tc_fence_after_sync();
+            // ---- masked tile: this thread's 32-column sub-tile of two 64-column pieces at a time
+            for (int j0 = 0; j0 < npieces; j0 += 2) {
+                float v[2][32];
+                bool z[2];
 #pragma unroll
-                for (int sub = 0; sub < 2; ++sub) {
-                    const int cb = colbase + jj * 64 + sub * 32;   // first column of the sub-tile (in chunk)
+                for (int u = 0; u < 2; ++u) {
+                    const int jsub = ((colbase + (j0 + u) * 64) >> 5) + half;
+                    z[u] = FWD ? (jsub > isub) : (jsub < isub);
+                    if (!z[u]) tmem_ld32_nowait(tm + tlane + (j0 + u) * 64 + half * 32, v[u]);
+                }
+#pragma unroll
+                for (int u = 0; u < 2; ++u)
+                    if (!z[u]) tmem_ld_wait32(v[u]);
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int jj = j0 + u;
+                    const int cb = colbase + jj * 64 + half * 32;   // first column of the sub-tile (in chunk)
                     const int jsub = cb >> 5;
+                    unsigned char *mrow = smem + OFF_M + jj * 16384 + rl * 128;
                     uint32_t pk[16];
-                    const bool zero = FWD ? (jsub > isub) : (jsub < isub);
-                    if (zero) {
+                    if (z[u]) {
 #pragma unroll
                         for (int k = 0; k < 16; ++k) pk[k] = 0u;
                     } else {
-                        float v[32];
-                        tmem_ld32(tm + tlane + jj * 64 + sub * 32, v);
+                        float *vv = v[u];
                         if (jsub != isub) {
                             const float f = rowf * (FWD ? blk[isub * 8 + jsub] : blk[jsub * 8 + isub]);
 #pragma unroll
                             for (int k = 0; k < 32; k += 4) {
                                 const float4 cv = *reinterpret_cast<const float4 *>(cf + cb + k);
-                                v[k] *= cv.x * f;
-                                v[k + 1] *= cv.y * f;
-                                v[k + 2] *= cv.z * f;
-                                v[k + 3] *= cv.w * f;
+                                vv[k] *= cv.x * f;
+                                vv[k + 1] *= cv.y * f;
+                                vv[k + 2] *= cv.z * f;
+                                vv[k + 3] *= cv.w * f;
                             }
                         } else {
 #pragma unroll
@@ -349,29 +381,32 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                                     const int col = cb + k + e;
                                     const bool on = FWD ? (col <= r) : (col >= r);
                                     const float ex = FWD ? ex2f(csr - ccv[e]) * dv[e] : ex2f(ccv[e] - csr);
-                                    v[k + e] = on ? v[k + e] * ex : 0.f;
+                                    vv[k + e] = on ? vv[k + e] * ex : 0.f;
                                 }
                             }
                         }
 #pragma unroll
-                        for (int k = 0; k < 16; ++k) pk[k] = pack2(v[2 * k], v[2 * k + 1]);
+                        for (int k = 0; k < 16; ++k) pk[k] = pack2(vv[2 * k], vv[2 * k + 1]);
                     }
 #pragma unroll
                     for (int ch = 0; ch < 4; ++ch) {
-                        const int chunk16 = sub * 4 + ch;
+                        const int chunk16 = half * 4 + ch;
                         *reinterpret_cast<uint4 *>(mrow + ((chunk16 ^ (rl & 7)) << 4)) =
                             make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
                     }
                 }
-                tc_fence_before_sync();
-                fence_proxy_async_smem();
-                mbar_arrive(&mfull[jj]);
             }
+            tc_fence_before_sync();
+            fence_proxy_async_smem();
+            mbar_arrive(&mfull);
             if (hi >= 1) epilogue(hi - 1, offs_prev, dt_prev);
             offs_prev = offs;
             dt_prev = dtr;
         }
+        if (mt == 0) tma_store_wait_read();
+        bar_mask_warps();
         epilogue(nheads - 1, offs_prev, dt_prev);
+        if (mt == 0) tma_store_wait_all();
     }
 
     tc_fence_before_sync();
@@ -389,11 +424,11 @@ cudaError_t launch_scan_tc(const SegParams &p, const TcMaps &m, int mode, cudaSt
     if (mode == SC_FWD) {
         e = cudaFuncSetAttribute(k_scan_tc<SC_FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SC_SMEM);
         if (e != cudaSuccess) return e;
-        k_scan_tc<SC_FWD><<<grid, SC_THREADS, SC_SMEM, st>>>(p, nsplit, m.Cm, m.Bm, m.x, m.Hbf);
+        k_scan_tc<SC_FWD><<<grid, SC_THREADS, SC_SMEM, st>>>(p, nsplit, m.Cm, m.Bm, m.x, m.Hbf, m.y, m.x);
     } else {
         e = cudaFuncSetAttribute(k_scan_tc<SC_DX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SC_SMEM);
         if (e != cudaSuccess) return e;
-        k_scan_tc<SC_DX><<<grid, SC_THREADS, SC_SMEM, st>>>(p, nsplit, m.Bm, m.Cm, m.dy, m.Gbf);
+        k_scan_tc<SC_DX><<<grid, SC_THREADS, SC_SMEM, st>>>(p, nsplit, m.Bm, m.Cm, m.dy, m.Gbf, m.dx, m.x);
     }
     return cudaGetLastError();
 }
