@@ -44,7 +44,7 @@ static void prof_end(ProfEvent *ev, cudaStream_t st) {
 }
 
 struct Layout {
-    size_t status, cs, dtT, Hst, Hbf, hcarry, Gst, Gbf, gcarry, ghdot, ddt_dir, rho, psi, psi2, pB, pC, dAp, dDp;
+    size_t status, cs, dtT, Hst, Hbf, hcarry, Gst, Gbf, gcarry, ghdot, ddt_dir, rho, rho2, psi, psi2, pB, pC, dAp, dDp;
     size_t total;
 };
 
@@ -121,6 +121,7 @@ static void make_layout(const Plan &pl, int op, Layout &lo) {
         lo.ghdot = take(BH * pl.ncs * 8 * sizeof(float));
         lo.ddt_dir = take(vec);
         lo.rho = take(vec);
+        lo.rho2 = take(pl.use_tc ? vec : 0);
         lo.psi = take(vec);
         lo.psi2 = take(vec);
         const size_t part = (size_t)pl.B * pl.seg * pl.G * pl.nsl * pl.N * sizeof(float);
@@ -190,6 +191,7 @@ static void fill_params(const Plan &pl, const Layout &lo, void *ws, SegParams &s
     sp.ghdot = (float *)(w + lo.ghdot);
     sp.ddt_dir = (float *)(w + lo.ddt_dir);
     sp.rho = (float *)(w + lo.rho);
+    sp.rho2 = nullptr;   // set by the backward driver on the tensor-core path
     sp.psi = (float *)(w + lo.psi);
     sp.psi2 = (float *)(w + lo.psi2);
     sp.pB = (float *)(w + lo.pB);
@@ -363,6 +365,7 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
     fill_params(pl, lo, ws, sp);
     sp.x = x; sp.dt = dt; sp.A = A; sp.Bm = Bm; sp.Cm = Cm; sp.D = D; sp.dy = dy;
     sp.dx = dx; sp.ddt = ddt; sp.dB = dB; sp.dC = dC;
+    if (pl.use_tc) sp.rho2 = (float *)((char *)ws + lo.rho2);
     SSD_TRY(cudaMemsetAsync(sp.status, 0, 256, st));
     TcMaps maps;
     if (pl.use_tc && !tc_make_maps(sp, maps)) return SSD_ECUDA;

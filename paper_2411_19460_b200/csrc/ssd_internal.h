@@ -40,7 +40,9 @@ struct SegParams {
     float *gcarry;         // [B,H,P,N]     state gradient handed right-to-left (backward)
     float *ghdot;          // [B,H,ncs,8]   partial sums of exp(cs_last) <Gout_c, H_in,c>
     float *ddt_dir;        // [B,H,ncs,Q]   direct part of ddt
-    float *rho;            // [B,H,ncs,Q]   dy_t . (y_t - D x_t)   = C_t . dC_t of this head
+    float *rho;            // [B,H,ncs,Q]   C_t . dC_t of this head (CUDA-core path: all of it; tensor-core
+                           //               path: its intra-chunk part)
+    float *rho2;           // [B,H,ncs,Q]   tensor-core path: C_t . (inter-chunk part of this head's dC_t); else NULL
     float *psi;            // [B,H,ncs,Q]   B_t . (intra-chunk part of this head's dB_t)
     float *psi2;           // [B,H,ncs,Q]   B_t . (inter-chunk part of this head's dB_t)
     float *pB, *pC;        // [B,seg,G,nsl,N] per-head-slice partial dB / dC

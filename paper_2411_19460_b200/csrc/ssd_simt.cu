@@ -555,10 +555,10 @@ cudaError_t launch_masked_product_simt(const SegParams &p, int dtype, int mode, 
 // inter-chunk parts, da_t = exp(a_t) <g_t, h_{t-1}> is the sum of four terms, none of which
 // subtracts large numbers when the decay inside a chunk is strong:
 //   sum_{t'>=t} (rho_intra_t' - psi_t')     pairs (t' >= t > s) inside the chunk
-// + sum_{t'>=t} rho_inter_t'                outputs at/after t reading the chunk-entry state
+// + sum_{t'>=t} rho_inter_t'                outputs at/after t reading the chunk-entry state (rho2)
 // + sum_{s<t}   psi2_s                      inputs before t feeding the chunk-exit gradient
 // + exp(cs_last) <Gout, H_in>
-// (rho = rho_intra + rho_inter is stored as one vector).  Suffix/prefix scans: serial inside a lane,
+// (the CUDA-core kernels store rho = rho_intra + rho_inter as one vector and no rho2).  Suffix/prefix scans: serial inside a lane,
 // warp shuffles across lanes.  Then ddt = ddt_direct + A da, dA partial = sum_t dt_t da_t.
 __global__ void __launch_bounds__(128) k_bwd_finish(SegParams p) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -576,7 +576,7 @@ __global__ void __launch_bounds__(128) k_bwd_finish(SegParams p) {
         if (j < per) {
             dtv[j] = p.dtT[vo + j];
             dd[j] = p.ddt_dir[vo + j];
-            run += p.rho[vo + j] - p.psi[vo + j];
+            run += (p.rho[vo + j] - p.psi[vo + j]) + (p.rho2 ? p.rho2[vo + j] : 0.f);
             sfx[j] = run;
         }
     float incl = run;

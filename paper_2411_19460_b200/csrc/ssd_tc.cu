@@ -77,16 +77,22 @@ bool tc_make_maps(const SegParams &p, TcMaps &m) {
 // index).  The per-row weight is multiplied into the X tile in shared memory (it is uniform along
 // a row, so the swizzle does not matter), the two K halves are separate TMA transactions so the
 // second lands while the first is scaled and multiplied.
+//
+// Mode DSTATE also produces, per head, rho2_t = e^{cs_t} dy_t . (H_in C_t): the inter-chunk part of
+// C_t . dC_t that the decay gradient needs.  The C tile is already in shared memory (as rows of
+// time it is a K-major A operand), so it is one more product C (256 x N) * H_in^T (N x P) per head
+// into spare TMEM columns, and a row dot with the already scaled dy tile.
 constexpr int CS_THREADS = 128;
-constexpr int CS_SMEM = 2 * (2 * 16384 + 2 * 16384) + 1024;  // two K halves x (X pair 32 KB + V 32 KB) + align
+constexpr int CS_SMEM_BASE = 2 * (2 * 16384 + 2 * 16384);    // two K halves x (X pair 32 KB + V 32 KB)
+constexpr int CS_SMEM = CS_SMEM_BASE + 2 * 16384 + 1024;      // + two heads' bf16 entry states + align
 
 __global__ void __launch_bounds__(CS_THREADS)
 k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
-                 const __grid_constant__ CUtensorMap tmV) {
+                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmH) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     // [half][ X head0 16K | X head1 16K | V n0-63 16K | V n64-127 16K ]
-    __shared__ uint64_t bar_half[2], bar_mma;
+    __shared__ uint64_t bar_half[2], bar_mma, bar_h;
     __shared__ uint32_t tmem_base, abort_flag;
     __shared__ float wsm[2][256];
 
@@ -99,6 +105,7 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
         mbar_init(&bar_half[0], 1);
         mbar_init(&bar_half[1], 1);
         mbar_init(&bar_mma, 1);
+        mbar_init(&bar_h, 1);
         abort_flag = 0;
         fence_barrier_init();
         for (int half = 0; half < 2; ++half) {
@@ -109,8 +116,17 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
             tma_load_3d(st + 32768, &tmV, &bar_half[half], g * 128, tok0 + half * 128, b);
             tma_load_3d(st + 49152, &tmV, &bar_half[half], g * 128 + 64, tok0 + half * 128, b);
         }
+        if (mode == STATE_MODE_DSTATE) {
+            mbar_arrive_expect_tx(&bar_h, 32768);
+            for (int hh = 0; hh < 2; ++hh) {
+                const int row = ((b * (p.ncs + 1) + c) * p.H + h0 + hh) * 64;   // state entering chunk c
+                tma_load_3d(smem + CS_SMEM_BASE + hh * 16384, &tmH, &bar_h, 0, row, 0);
+                tma_load_3d(smem + CS_SMEM_BASE + hh * 16384 + 8192, &tmH, &bar_h, 64, row, 0);
+            }
+        }
     }
-    if (warp == 0) tmem_alloc(&tmem_base, 128);
+    const uint32_t ncol_tmem = (mode == STATE_MODE_DSTATE) ? 512u : 128u;
+    if (warp == 0) tmem_alloc(&tmem_base, ncol_tmem);
     // per-row weights of both heads
     for (int i = tid; i < 512; i += CS_THREADS) {
         const int hh = i >> 8, t = i & 255;
@@ -158,7 +174,26 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
                 const uint64_t bd = umma_desc_sw128(sb + ks * 2048, 16384, 1024);
                 umma_bf16(tm, ad, bd, idesc, (half | ks) ? 1u : 0u);
             }
-            if (half == 1) umma_commit(&bar_mma);
+            if (half == 1) {
+                if (mode == STATE_MODE_DSTATE) {
+                    // Yoff[t, p] = sum_n C[t, n] H_in[p, n] per head and 128-row time block
+                    mbar_wait(&bar_h, 0, &abort_flag, p.status);
+                    tc_fence_after_sync();
+                    const uint32_t idy = umma_idesc_bf16(128, 64, false, false);
+                    for (int hh = 0; hh < 2; ++hh)
+                        for (int tb = 0; tb < 2; ++tb) {
+                            const uint32_t sc = smem_u32(smem + tb * 65536 + 32768);
+                            const uint32_t sh = smem_u32(smem + CS_SMEM_BASE + hh * 16384);
+#pragma unroll
+                            for (int kk = 0; kk < 8; ++kk)
+                                umma_bf16(tm + 128 + (hh * 2 + tb) * 64,
+                                          umma_desc_sw128(sc + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024),
+                                          umma_desc_sw128(sh + (kk >> 2) * 8192 + (kk & 3) * 32, 16, 1024), idy,
+                                          kk ? 1u : 0u);
+                        }
+                }
+                umma_commit(&bar_mma);
+            }
         }
     }
     mbar_wait(&bar_mma, 0, &abort_flag, p.status);
@@ -177,17 +212,44 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
                 *reinterpret_cast<float4 *>(out + c0 + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
         }
     }
+    if (mode == STATE_MODE_DSTATE) {
+        // rho2_t = (e^{cs_t} dy_t) . Yoff_t with the scaled dy row read back from shared memory
+        for (int hh = 0; hh < 2; ++hh)
+            for (int tb = 0; tb < 2; ++tb) {
+                float y0[32], y1[32];
+                const uint32_t ta = tm + ((uint32_t)(warp * 32) << 16) + 128 + (hh * 2 + tb) * 64;
+                tmem_ld32_nowait(ta, y0);
+                tmem_ld32_nowait(ta + 32, y1);
+                tmem_ld_wait32(y0);
+                tmem_ld_wait32(y1);
+                const unsigned char *row = smem + tb * 65536 + hh * 16384 + tid * 128;
+                float acc = 0.f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint4 v = *reinterpret_cast<const uint4 *>(row + ((j ^ (tid & 7)) << 4));
+                    const __nv_bfloat162 *e = reinterpret_cast<const __nv_bfloat162 *>(&v);
+                    const float *yy = (j < 4) ? (y0 + j * 8) : (y1 + (j - 4) * 8);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float2 f = __bfloat1622float2(e[k]);
+                        acc = fmaf(f.x, yy[2 * k], acc);
+                        acc = fmaf(f.y, yy[2 * k + 1], acc);
+                    }
+                }
+                p.rho2[((((size_t)b * p.H + h0 + hh) * p.ncs + c) << 8) + tb * 128 + tid] = acc;
+            }
+    }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tm, 128);
+    if (warp == 0) tmem_dealloc(tm, ncol_tmem);
 }
 
 cudaError_t launch_chunk_state_tc(const SegParams &p, const TcMaps &m, int mode, cudaStream_t st) {
     cudaError_t e = cudaFuncSetAttribute(k_chunk_state_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, CS_SMEM);
     if (e != cudaSuccess) return e;
     dim3 grid(p.nc, p.H / 2, p.B);
-    if (mode == STATE_MODE_FWD) k_chunk_state_tc<<<grid, CS_THREADS, CS_SMEM, st>>>(p, mode, m.x, m.Bm);
-    else k_chunk_state_tc<<<grid, CS_THREADS, CS_SMEM, st>>>(p, mode, m.dy, m.Cm);
+    if (mode == STATE_MODE_FWD) k_chunk_state_tc<<<grid, CS_THREADS, CS_SMEM, st>>>(p, mode, m.x, m.Bm, m.Hbf);
+    else k_chunk_state_tc<<<grid, CS_THREADS, CS_SMEM, st>>>(p, mode, m.dy, m.Cm, m.Hbf);
     return cudaGetLastError();
 }
 

@@ -356,12 +356,10 @@ k_grad_bc_tc(SegParams p, const __grid_constant__ CUtensorMap tmRow,   // DC: dy
             if (half == 0) {
                 const size_t vo = ((((size_t)b * p.H + h) * p.ncs + c) << 8) + r;
                 const float e1 = d1 + pp[rl], e2 = d2 + pp[128 + rl];
-                if (DC) {
-                    p.rho[vo] = e1 + e2;
-                } else {
-                    p.psi[vo] = e1;
-                    p.psi2[vo] = e2;
-                }
+                // the inter-chunk parts (rho2, psi2) come from the dstate and dx kernels
+                if (DC) p.rho[vo] = e1;
+                else p.psi[vo] = e1;
+                (void)e2;
             }
         }
 

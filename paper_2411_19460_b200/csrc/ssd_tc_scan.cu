@@ -3,7 +3,8 @@
 //
 //   SC_FWD (a5+a6): y_t  = sum_{s<=t} (C_t.B_s) e^{cs_t-cs_s} dt_s x_s + e^{cs_t} C_t H_in + D x_t
 //   SC_DX  (a10)  : u_s  = sum_{t>=s} (B_s.C_t) e^{cs_t-cs_s} dy_t      + e^{cs_last-cs_s} B_s Gout
-//                   dx_s = D dy_s + dt_s u_s ;  ddt_direct_s = x_s . u_s ;  dD partial = sum dy.x
+//                   dx_s = D dy_s + dt_s u_s ;  ddt_direct_s = x_s . u_s ;  dD partial = sum dy.x ;
+//                   psi2_s = dt_s e^{cs_last-cs_s} x_s . (Gout B_s)   (inter-chunk part of B_s . dB_s)
 //
 // (Eq. 1 of the paper regrouped by chunks; cs = inclusive cumsum of dt*A inside the chunk.)
 //
@@ -40,8 +41,8 @@ constexpr uint32_t OFF_OUT = 180224;      // 16 KB  output tile staged for the T
 constexpr uint32_t OFF_XR = 196608;       // 16 KB  SC_DX: the head's x rows of this row block
 constexpr uint32_t OFF_VEC = 212992;      // per-head vectors, double buffered
 constexpr uint32_t VEC_FLOATS = 256 * 3 + 64;
-constexpr uint32_t OFF_PART = OFF_VEC + 2 * VEC_FLOATS * 4;   // 2 x 136 floats: row halves, warp sums
-constexpr uint32_t SC_SMEM = OFF_PART + 2 * 136 * 4 + 1024;
+constexpr uint32_t OFF_PART = OFF_VEC + 2 * VEC_FLOATS * 4;   // 2 x 264 floats: row halves (2 x 128), warp sums
+constexpr uint32_t SC_SMEM = OFF_PART + 2 * 264 * 4 + 1024;
 
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -248,7 +249,7 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             tmem_ld_wait32(a2);
             tc_fence_before_sync();
             mbar_arrive(&accempty[buf]);             // both accumulators are in registers now
-            float dd = 0.f, dsum = 0.f;
+            float dd = 0.f, dd2 = 0.f, dsum = 0.f;
             unsigned char *orow = smem + OFF_OUT + rl * 128;
 #pragma unroll
             for (int k8 = 0; k8 < 4; ++k8) {
@@ -267,6 +268,8 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                     } else {
                         dd = fmaf(xv[e], u0, dd);
                         dd = fmaf(xv[e + 1], u1, dd);
+                        dd2 = fmaf(xv[e], a2[i], dd2);
+                        dd2 = fmaf(xv[e + 1], a2[i + 1], dd2);
                         dsum = fmaf(dyv[e], xv[e], dsum);
                         dsum = fmaf(dyv[e + 1], xv[e + 1], dsum);
                         ow[e >> 1] = pack2(fmaf(Dh, dyv[e], dtr * u0), fmaf(Dh, dyv[e + 1], dtr * u1));
@@ -274,11 +277,14 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                 }
                 *reinterpret_cast<uint4 *>(orow + (((half * 4 + k8) ^ (rl & 7)) << 4)) = o;
             }
-            float *pp = part + (hi & 1) * 136;
+            float *pp = part + (hi & 1) * 264;
             if (!FWD) {
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, off);
-                if (half == 1) pp[rl] = dd;
+                if (half == 1) {
+                    pp[rl] = dd;
+                    pp[136 + rl] = dd2;
+                }
                 if (lane == 0) pp[128 + (warp - 2)] = dsum;
             }
             fence_proxy_async_smem();
@@ -289,7 +295,12 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             }
             if (!FWD) {
                 // the two column halves of a row, and the eight warps' dy.x sums, in a fixed order
-                if (half == 0) p.ddt_dir[((((size_t)b * p.H + h) * p.ncs + c) << 8) + r] = dd + pp[rl];
+                if (half == 0) {
+                    const size_t vo = ((((size_t)b * p.H + h) * p.ncs + c) << 8) + r;
+                    p.ddt_dir[vo] = dd + pp[rl];
+                    // psi2_s = B_s . (inter-chunk part of this head's dB_s) = dt_s e^{cs_last-cs_s} x_s . (Gout B_s)
+                    p.psi2[vo] = dtr * offs * (dd2 + pp[136 + rl]);
+                }
                 if (mt == 0) {
                     float s = 0.f;
 #pragma unroll
