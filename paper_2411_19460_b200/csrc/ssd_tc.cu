@@ -198,20 +198,6 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
     }
     mbar_wait(&bar_mma, 0, &abort_flag, p.status);
     tc_fence_after_sync();
-    {
-        const int hh = tid >> 6, pp = tid & 63;
-        const int slot = (mode == STATE_MODE_FWD) ? c + 1 : c;
-        float *base = (mode == STATE_MODE_FWD) ? p.Hst : p.Gst;
-        float *out = base + ((((size_t)b * (p.ncs + 1) + slot) * p.H + h0 + hh) * 64 + pp) * 128;
-#pragma unroll
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-            float v[32];
-            tmem_ld32(tm + ((uint32_t)(warp * 32) << 16) + c0, v);
-#pragma unroll
-            for (int i = 0; i < 32; i += 4)
-                *reinterpret_cast<float4 *>(out + c0 + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-        }
-    }
     if (mode == STATE_MODE_DSTATE) {
         // rho2_t = (e^{cs_t} dy_t) . Yoff_t with the scaled dy row read back from shared memory
         for (int hh = 0; hh < 2; ++hh)
@@ -238,6 +224,30 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
                 }
                 p.rho2[((((size_t)b * p.H + h0 + hh) * p.ncs + c) << 8) + tb * 128 + tid] = acc;
             }
+    }
+    // The CTA's 128 x 128 fp32 result (two heads x 64 rows) is one contiguous 64 KB block of the state
+    // buffer.  Row-per-thread stores would touch 32 different lines per instruction, so the tile goes
+    // through shared memory (operands are dead by now; rows padded to 132 floats) and leaves as whole rows.
+    __syncthreads();
+    {
+        float *stg = reinterpret_cast<float *>(smem);
+#pragma unroll
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+            float v[32];
+            tmem_ld32(tm + ((uint32_t)(warp * 32) << 16) + c0, v);
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+                *reinterpret_cast<float4 *>(stg + tid * 132 + c0 + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+        }
+        __syncthreads();
+        const int slot = (mode == STATE_MODE_FWD) ? c + 1 : c;
+        float *base = (mode == STATE_MODE_FWD) ? p.Hst : p.Gst;
+        float4 *out = reinterpret_cast<float4 *>(base + (((size_t)b * (p.ncs + 1) + slot) * p.H + h0) * 64 * 128);
+#pragma unroll 4
+        for (int it = 0; it < 32; ++it) {
+            const int idx = it * CS_THREADS + tid, row = idx >> 5, c4 = idx & 31;
+            out[idx] = *reinterpret_cast<const float4 *>(stg + row * 132 + c4 * 4);
+        }
     }
     tc_fence_before_sync();
     __syncthreads();
