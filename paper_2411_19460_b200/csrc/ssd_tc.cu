@@ -75,24 +75,23 @@ bool tc_make_maps(const SegParams &p, TcMaps &m) {
 //   mode DSTATE: X = dy, V = Cm, w_t = exp(cs_t)                 -> Gst slot c     (E_c)
 // Both operands are MN-major straight from the row-major tensors (rows = time = the contraction
 // index).  The per-row weight is multiplied into the X tile in shared memory (it is uniform along
-// a row, so the swizzle does not matter), the two K halves are separate TMA transactions so the
-// second lands while the first is scaled and multiplied.
+// a row, so the swizzle does not matter).  The kernel is bound by its loads, so a CTA keeps only
+// ONE 64 KB stage (half a chunk) and two to three CTAs share an SM: one CTA's load overlaps the
+// others' scaling, MMAs and epilogue.
 //
 // Mode DSTATE also produces, per head, rho2_t = e^{cs_t} dy_t . (H_in C_t): the inter-chunk part of
 // C_t . dC_t that the decay gradient needs.  The C tile is already in shared memory (as rows of
-// time it is a K-major A operand), so it is one more product C (256 x N) * H_in^T (N x P) per head
-// into spare TMEM columns, and a row dot with the already scaled dy tile.
+// time it is a K-major A operand), so it is one more product C (128 x N) * H_in^T (N x P) per head
+// and half into spare TMEM columns, and a row dot with the already scaled dy tile.
 constexpr int CS_THREADS = 128;
-constexpr int CS_SMEM_BASE = 2 * (2 * 16384 + 2 * 16384);    // two K halves x (X pair 32 KB + V 32 KB)
-constexpr int CS_SMEM = CS_SMEM_BASE + 2 * 16384 + 1024;      // + two heads' bf16 entry states + align
+constexpr int CS_STAGE = 65536;   // X head0 16K | X head1 16K | V n0-63 16K | V n64-127 16K   (128 time rows)
 
 __global__ void __launch_bounds__(CS_THREADS)
 k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmH) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    // [half][ X head0 16K | X head1 16K | V n0-63 16K | V n64-127 16K ]
-    __shared__ uint64_t bar_half[2], bar_mma, bar_h;
+    __shared__ uint64_t bar_ld, bar_mma, bar_h;
     __shared__ uint32_t tmem_base, abort_flag;
     __shared__ float wsm[2][256];
 
@@ -100,39 +99,40 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
     const int h0 = hp * 2, g = h0 / p.hpg;
     const int tid = threadIdx.x, warp = tid >> 5;
     const int tok0 = p.t0 + c * 256;
+    const bool dstate = (mode == STATE_MODE_DSTATE);
+
+    auto issue_stage = [&](int half) {
+        mbar_arrive_expect_tx(&bar_ld, CS_STAGE);
+        tma_load_3d(smem, &tmX, &bar_ld, h0 * 64, tok0 + half * 128, b);
+        tma_load_3d(smem + 16384, &tmX, &bar_ld, h0 * 64 + 64, tok0 + half * 128, b);
+        tma_load_3d(smem + 32768, &tmV, &bar_ld, g * 128, tok0 + half * 128, b);
+        tma_load_3d(smem + 49152, &tmV, &bar_ld, g * 128 + 64, tok0 + half * 128, b);
+    };
 
     if (tid == 0) {
-        mbar_init(&bar_half[0], 1);
-        mbar_init(&bar_half[1], 1);
+        mbar_init(&bar_ld, 1);
         mbar_init(&bar_mma, 1);
         mbar_init(&bar_h, 1);
         abort_flag = 0;
         fence_barrier_init();
-        for (int half = 0; half < 2; ++half) {
-            unsigned char *st = smem + half * 65536;
-            mbar_arrive_expect_tx(&bar_half[half], 65536);
-            tma_load_3d(st, &tmX, &bar_half[half], h0 * 64, tok0 + half * 128, b);
-            tma_load_3d(st + 16384, &tmX, &bar_half[half], h0 * 64 + 64, tok0 + half * 128, b);
-            tma_load_3d(st + 32768, &tmV, &bar_half[half], g * 128, tok0 + half * 128, b);
-            tma_load_3d(st + 49152, &tmV, &bar_half[half], g * 128 + 64, tok0 + half * 128, b);
-        }
-        if (mode == STATE_MODE_DSTATE) {
+        issue_stage(0);
+        if (dstate) {
             mbar_arrive_expect_tx(&bar_h, 32768);
             for (int hh = 0; hh < 2; ++hh) {
                 const int row = ((b * (p.ncs + 1) + c) * p.H + h0 + hh) * 64;   // state entering chunk c
-                tma_load_3d(smem + CS_SMEM_BASE + hh * 16384, &tmH, &bar_h, 0, row, 0);
-                tma_load_3d(smem + CS_SMEM_BASE + hh * 16384 + 8192, &tmH, &bar_h, 64, row, 0);
+                tma_load_3d(smem + CS_STAGE + hh * 16384, &tmH, &bar_h, 0, row, 0);
+                tma_load_3d(smem + CS_STAGE + hh * 16384 + 8192, &tmH, &bar_h, 64, row, 0);
             }
         }
     }
-    const uint32_t ncol_tmem = (mode == STATE_MODE_DSTATE) ? 512u : 128u;
+    const uint32_t ncol_tmem = dstate ? 256u : 128u;   // E or S: 128 columns; Yoff of two heads: 128 more
     if (warp == 0) tmem_alloc(&tmem_base, ncol_tmem);
     // per-row weights of both heads
     for (int i = tid; i < 512; i += CS_THREADS) {
         const int hh = i >> 8, t = i & 255;
         const float *csb = p.cs + ((((size_t)b * p.H + h0 + hh) * p.ncs + c) << 8);
         float w;
-        if (mode == STATE_MODE_FWD) {
+        if (!dstate) {
             const float *dtb = p.dtT + ((((size_t)b * p.H + h0 + hh) * p.ncs + c) << 8);
             w = __expf(fminf(csb[255] - csb[t], 0.f)) * dtb[t];
         } else {
@@ -147,13 +147,12 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
     const uint32_t idesc = umma_idesc_bf16(128, 128, true, true);
 
     for (int half = 0; half < 2; ++half) {
-        unsigned char *st = smem + half * 65536;
-        mbar_wait(&bar_half[half], 0, &abort_flag, p.status);
+        mbar_wait(&bar_ld, half, &abort_flag, p.status);
         // scale the X pair: 2 heads x 128 rows x 8 chunks of 16 B
         for (int q = tid; q < 2048; q += CS_THREADS) {
             const int hh = q >> 10, row = (q >> 3) & 127;
             const float w = wsm[hh][half * 128 + row];
-            uint4 *ptr = reinterpret_cast<uint4 *>(st + (size_t)q * 16);
+            uint4 *ptr = reinterpret_cast<uint4 *>(smem + (size_t)q * 16);
             uint4 v = *ptr;
             __nv_bfloat162 *e = reinterpret_cast<__nv_bfloat162 *>(&v);
 #pragma unroll
@@ -167,48 +166,40 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
         __syncthreads();
         if (tid == 0) {
             tc_fence_after_sync();
-            const uint32_t sa = smem_u32(st), sb = smem_u32(st + 32768);
+            const uint32_t sa = smem_u32(smem), sb = smem_u32(smem + 32768);
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                const uint64_t ad = umma_desc_sw128(sa + ks * 2048, 16384, 1024);
-                const uint64_t bd = umma_desc_sw128(sb + ks * 2048, 16384, 1024);
-                umma_bf16(tm, ad, bd, idesc, (half | ks) ? 1u : 0u);
-            }
-            if (half == 1) {
-                if (mode == STATE_MODE_DSTATE) {
-                    // Yoff[t, p] = sum_n C[t, n] H_in[p, n] per head and 128-row time block
+            for (int ks = 0; ks < 8; ++ks)
+                umma_bf16(tm, umma_desc_sw128(sa + ks * 2048, 16384, 1024), umma_desc_sw128(sb + ks * 2048, 16384, 1024),
+                          idesc, (half | ks) ? 1u : 0u);
+            if (dstate) {
+                // Yoff[t, p] = sum_n C[t, n] H_in[p, n] for the 128 time rows of this half, per head
+                if (half == 0) {
                     mbar_wait(&bar_h, 0, &abort_flag, p.status);
                     tc_fence_after_sync();
-                    const uint32_t idy = umma_idesc_bf16(128, 64, false, false);
-                    for (int hh = 0; hh < 2; ++hh)
-                        for (int tb = 0; tb < 2; ++tb) {
-                            const uint32_t sc = smem_u32(smem + tb * 65536 + 32768);
-                            const uint32_t sh = smem_u32(smem + CS_SMEM_BASE + hh * 16384);
-#pragma unroll
-                            for (int kk = 0; kk < 8; ++kk)
-                                umma_bf16(tm + 128 + (hh * 2 + tb) * 64,
-                                          umma_desc_sw128(sc + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024),
-                                          umma_desc_sw128(sh + (kk >> 2) * 8192 + (kk & 3) * 32, 16, 1024), idy,
-                                          kk ? 1u : 0u);
-                        }
                 }
-                umma_commit(&bar_mma);
+                const uint32_t idy = umma_idesc_bf16(128, 64, false, false);
+                for (int hh = 0; hh < 2; ++hh) {
+                    const uint32_t sh = smem_u32(smem + CS_STAGE + hh * 16384);
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        umma_bf16(tm + 128 + hh * 64, umma_desc_sw128(sb + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024),
+                                  umma_desc_sw128(sh + (kk >> 2) * 8192 + (kk & 3) * 32, 16, 1024), idy, kk ? 1u : 0u);
+                }
             }
+            umma_commit(&bar_mma);
         }
-    }
-    mbar_wait(&bar_mma, 0, &abort_flag, p.status);
-    tc_fence_after_sync();
-    if (mode == STATE_MODE_DSTATE) {
-        // rho2_t = (e^{cs_t} dy_t) . Yoff_t with the scaled dy row read back from shared memory
-        for (int hh = 0; hh < 2; ++hh)
-            for (int tb = 0; tb < 2; ++tb) {
+        mbar_wait(&bar_mma, half, &abort_flag, p.status);
+        tc_fence_after_sync();
+        if (dstate) {
+            // rho2_t = (e^{cs_t} dy_t) . Yoff_t with the scaled dy row read back from shared memory
+            for (int hh = 0; hh < 2; ++hh) {
                 float y0[32], y1[32];
-                const uint32_t ta = tm + ((uint32_t)(warp * 32) << 16) + 128 + (hh * 2 + tb) * 64;
+                const uint32_t ta = tm + ((uint32_t)(warp * 32) << 16) + 128 + hh * 64;
                 tmem_ld32_nowait(ta, y0);
                 tmem_ld32_nowait(ta + 32, y1);
                 tmem_ld_wait32(y0);
                 tmem_ld_wait32(y1);
-                const unsigned char *row = smem + tb * 65536 + hh * 16384 + tid * 128;
+                const unsigned char *row = smem + hh * 16384 + tid * 128;
                 float acc = 0.f;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -222,31 +213,37 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
                         acc = fmaf(f.y, yy[2 * k + 1], acc);
                     }
                 }
-                p.rho2[((((size_t)b * p.H + h0 + hh) * p.ncs + c) << 8) + tb * 128 + tid] = acc;
+                p.rho2[((((size_t)b * p.H + h0 + hh) * p.ncs + c) << 8) + half * 128 + tid] = acc;
             }
+        }
+        tc_fence_before_sync();
+        fence_proxy_async_smem();              // order this thread's accesses to the stage before the next TMA write
+        __syncthreads();                       // the stage (and the Yoff columns) may be overwritten now
+        if (half == 0 && tid == 0) issue_stage(1);
     }
+
     // The CTA's 128 x 128 fp32 result (two heads x 64 rows) is one contiguous 64 KB block of the state
     // buffer.  Row-per-thread stores would touch 32 different lines per instruction, so the tile goes
-    // through shared memory (operands are dead by now; rows padded to 132 floats) and leaves as whole rows.
-    __syncthreads();
+    // through the (now dead) stage: float4 (row, j) sits at slot j ^ (row & 31) of its row, which keeps
+    // both the row-per-thread writes and the row-per-warp reads free of bank conflicts.
     {
-        float *stg = reinterpret_cast<float *>(smem);
+        float4 *stg = reinterpret_cast<float4 *>(smem);
 #pragma unroll
         for (int c0 = 0; c0 < 128; c0 += 32) {
             float v[32];
             tmem_ld32(tm + ((uint32_t)(warp * 32) << 16) + c0, v);
 #pragma unroll
             for (int i = 0; i < 32; i += 4)
-                *reinterpret_cast<float4 *>(stg + tid * 132 + c0 + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                stg[tid * 32 + (((c0 + i) >> 2) ^ (tid & 31))] = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
         }
         __syncthreads();
-        const int slot = (mode == STATE_MODE_FWD) ? c + 1 : c;
-        float *base = (mode == STATE_MODE_FWD) ? p.Hst : p.Gst;
+        const int slot = dstate ? c : c + 1;
+        float *base = dstate ? p.Gst : p.Hst;
         float4 *out = reinterpret_cast<float4 *>(base + (((size_t)b * (p.ncs + 1) + slot) * p.H + h0) * 64 * 128);
 #pragma unroll 4
         for (int it = 0; it < 32; ++it) {
             const int idx = it * CS_THREADS + tid, row = idx >> 5, c4 = idx & 31;
-            out[idx] = *reinterpret_cast<const float4 *>(stg + row * 132 + c4 * 4);
+            out[idx] = stg[row * 32 + (c4 ^ (row & 31))];
         }
     }
     tc_fence_before_sync();
@@ -255,11 +252,13 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
 }
 
 cudaError_t launch_chunk_state_tc(const SegParams &p, const TcMaps &m, int mode, cudaStream_t st) {
-    cudaError_t e = cudaFuncSetAttribute(k_chunk_state_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, CS_SMEM);
+    const int smem = CS_STAGE + (mode == STATE_MODE_DSTATE ? 32768 : 0) + 1024;
+    cudaError_t e = cudaFuncSetAttribute(k_chunk_state_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         CS_STAGE + 32768 + 1024);
     if (e != cudaSuccess) return e;
     dim3 grid(p.nc, p.H / 2, p.B);
-    if (mode == STATE_MODE_FWD) k_chunk_state_tc<<<grid, CS_THREADS, CS_SMEM, st>>>(p, mode, m.x, m.Bm, m.Hbf);
-    else k_chunk_state_tc<<<grid, CS_THREADS, CS_SMEM, st>>>(p, mode, m.dy, m.Cm, m.Hbf);
+    if (mode == STATE_MODE_FWD) k_chunk_state_tc<<<grid, CS_THREADS, smem, st>>>(p, mode, m.x, m.Bm, m.Hbf);
+    else k_chunk_state_tc<<<grid, CS_THREADS, smem, st>>>(p, mode, m.dy, m.Cm, m.Hbf);
     return cudaGetLastError();
 }
 
