@@ -19,6 +19,7 @@ struct SegParams {
     int ncs;       // chunk capacity of the workspace (chunks of a full segment)
     int nct;       // chunks in the whole sequence (L / Q)
     int nsl;       // head slices per group in the dB/dC partial buffers
+    int ndd;          // partial sums of dD per (head, chunk) that the kernels of this path write (<= 16)
     int nsplit_scan;  // head ranges per group in the tensor-core scan kernels (no effect on results)
     int64_t x_bs, dt_bs, bc_bs;  // batch strides, elements
 
@@ -47,7 +48,7 @@ struct SegParams {
     float *psi2;           // [B,H,ncs,Q]   B_t . (inter-chunk part of this head's dB_t)
     float *pB, *pC;        // [B,seg,G,nsl,N] per-head-slice partial dB / dC
     float *dAp;            // [B,H,nct]     per-chunk partial of dA
-    float *dDp;            // [B,H,nct,4]   per-row-tile partial of dD
+    float *dDp;            // [B,H,nct,16]  partials of dD, the first ndd of each group of 16 in use
 };
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -71,7 +72,7 @@ cudaError_t launch_final_dAdD(const SegParams &p, float *dA, float *dD, cudaStre
 // ssd_tc.cu : tensor-core (tcgen05 / TMEM / TMA) kernels, bf16 I/O
 struct TcMaps {
     CUtensorMap x, dy, Bm, Cm;  // [B][L][H*64] / [B][L][G*128], box 64 x 128 rows
-    CUtensorMap y, dx;          // outputs, same geometry as x (TMA stores)
+    CUtensorMap y, dx;          // outputs, same geometry as x; box 32 columns x 32 rows, no swizzle (TMA stores)
     CUtensorMap Hbf, Gbf;       // bf16 chunk states as [rows][128], box 64 x 64 rows
 };
 bool tc_supported(int dtype, int flags, int P, int N, int Q, int hpg);

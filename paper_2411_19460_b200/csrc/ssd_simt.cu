@@ -486,7 +486,7 @@ __global__ void __launch_bounds__(256) k_masked_product_simt(SegParams p) {
             float s = 0.f;
 #pragma unroll
             for (int w = 0; w < 8; ++w) s += Mk[w];
-            p.dDp[((((size_t)b * p.H + h) * p.nct + p.c0 + c) << 2) + rt] = s;
+            p.dDp[((((size_t)b * p.H + h) * p.nct + p.c0 + c) << 4) + rt] = s;
         }
     } else {
         // per-head partial dC / dB rows: [B, seg, G, nsl, N]
@@ -660,13 +660,13 @@ cudaError_t launch_reduce_dbdc(const SegParams &p, int dtype, cudaStream_t st) {
 // One warp per head; lanes stride over the per-chunk partials in fp64, then a fixed shuffle tree.
 __global__ void __launch_bounds__(32) k_final_dAdD(SegParams p, float *dA, float *dD) {
     const int h = blockIdx.x, lane = threadIdx.x;
-    const int nrt = p.Q >> 6;
+    const int nrt = p.ndd;
     double sA = 0.0, sD = 0.0;
     for (int b = 0; b < p.B; ++b) {
         const size_t base = ((size_t)b * p.H + h) * p.nct;
         for (int c = lane; c < p.nct; c += 32) {
             sA += (double)p.dAp[base + c];
-            for (int r = 0; r < nrt; ++r) sD += (double)p.dDp[((base + c) << 2) + r];
+            for (int r = 0; r < nrt; ++r) sD += (double)p.dDp[((base + c) << 4) + r];
         }
     }
 #pragma unroll

@@ -32,18 +32,19 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// bf16 tensor [dim2][dim1][dim0] (dim0 contiguous), box {64, box_rows, 1}, 128-byte swizzle.
+// bf16 tensor [dim2][dim1][dim0] (dim0 contiguous), box {box_cols, box_rows, 1}; 128-byte swizzle for
+// 64-element (128-byte) box rows, none for narrower ones.
 static bool make_map3(CUtensorMap *m, const void *ptr, uint64_t dim0, uint64_t dim1, uint64_t dim2,
-                      uint64_t stride1_elems, uint64_t stride2_elems, uint32_t box_rows) {
+                      uint64_t stride1_elems, uint64_t stride2_elems, uint32_t box_rows, uint32_t box_cols = 64) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return false;
     cuuint64_t dims[3] = {dim0, dim1, dim2};
     cuuint64_t strides[2] = {stride1_elems * 2, stride2_elems * 2};
-    cuuint32_t box[3] = {64, box_rows, 1};
+    cuuint32_t box[3] = {box_cols, box_rows, 1};
     cuuint32_t es[3] = {1, 1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, es,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+               CU_TENSOR_MAP_INTERLEAVE_NONE, box_cols == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 bool tc_supported(int dtype, int flags, int P, int N, int Q, int hpg) {
@@ -58,8 +59,8 @@ bool tc_make_maps(const SegParams &p, TcMaps &m) {
     bool ok = true;
     if (p.x) ok = ok && make_map3(&m.x, p.x, HP, p.L, p.B, HP, p.x_bs, 128);
     if (p.dy) ok = ok && make_map3(&m.dy, p.dy, HP, p.L, p.B, HP, p.x_bs, 128);
-    if (p.y) ok = ok && make_map3(&m.y, p.y, HP, p.L, p.B, HP, p.x_bs, 128);
-    if (p.dx) ok = ok && make_map3(&m.dx, p.dx, HP, p.L, p.B, HP, p.x_bs, 128);
+    if (p.y) ok = ok && make_map3(&m.y, p.y, HP, p.L, p.B, HP, p.x_bs, 32, 32);
+    if (p.dx) ok = ok && make_map3(&m.dx, p.dx, HP, p.L, p.B, HP, p.x_bs, 32, 32);
     if (p.Bm) ok = ok && make_map3(&m.Bm, p.Bm, GN, p.L, p.B, GN, p.bc_bs, 128);
     if (p.Cm) ok = ok && make_map3(&m.Cm, p.Cm, GN, p.L, p.B, GN, p.bc_bs, 128);
     // bf16 state copies viewed as [B*(ncs+1)*H*64 rows][128]

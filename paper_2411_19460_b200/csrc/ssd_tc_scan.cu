@@ -13,6 +13,7 @@
 // there in fp32 for every head of the range.  Per head the CTA then runs a three-role pipeline:
 //   producer warp : TMA loads of the head's value rows (x or dy) and its bf16 chunk state
 //   MMA warp      : acc2 = Rows * State^T (K = N), acc1 = M * V (K = up to 256 columns)
+//   vector warp   : the head's cumulative sums, step sizes and mask factors, one head ahead
 //   8 mask warps  : read S from TMEM, apply the decay mask, round to bf16 and store the masked
 //                   tile M to shared memory (A operand of the next MMA); then, while those MMAs run,
 //                   the epilogue of the previous head from the double-buffered accumulators.
@@ -32,17 +33,17 @@ using namespace sm100;
 
 namespace {
 
-constexpr int SC_THREADS = 320;          // warp 0 producer, warp 1 MMA, warps 2..9 mask + epilogue
+constexpr int SC_THREADS = 352;          // warp 0 producer, warp 1 MMA, warps 2..9 mask + epilogue, warp 10 vectors
 constexpr uint32_t OFF_ROWS = 0;          // 32 KB  [n-half][128 rows][128 B]
 constexpr uint32_t OFF_BX = 32768;        // 64 KB  score columns operand, then two value buffers
 constexpr uint32_t OFF_M = 98304;         // 64 KB  four 16 KB pieces of the masked tile
 constexpr uint32_t OFF_ST = 163840;       // 16 KB  bf16 chunk state [n-half][64 rows][128 B]
-constexpr uint32_t OFF_OUT = 180224;      // 16 KB  output tile staged for the TMA store
+constexpr uint32_t OFF_OUT = 180224;      // 16 KB  eight 2 KB slabs (32 rows x 64 B), one per mask warp, staged for TMA stores
 constexpr uint32_t OFF_XR = 196608;       // 16 KB  SC_DX: the head's x rows of this row block
 constexpr uint32_t OFF_VEC = 212992;      // per-head vectors, double buffered
 constexpr uint32_t VEC_FLOATS = 256 * 3 + 64;
-constexpr uint32_t OFF_PART = OFF_VEC + 2 * VEC_FLOATS * 4;   // 2 x 264 floats: row halves (2 x 128), warp sums
-constexpr uint32_t SC_SMEM = OFF_PART + 2 * 264 * 4 + 1024;
+constexpr uint32_t OFF_PART = OFF_VEC + 2 * VEC_FLOATS * 4;   // 4 quarters x [head parity][dd | dd2][32] floats
+constexpr uint32_t SC_SMEM = OFF_PART + 4 * 128 * 4 + 1024;
 
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -51,7 +52,6 @@ __device__ __forceinline__ float ex2f(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ void bar_mask_warps() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t *>(&v);
@@ -77,7 +77,7 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     __shared__ uint64_t bar_ab, bar_s, xfull[2], xempty[2], hfull, hempty, xrfull, xrempty, mfull, mempty, accfull[2],
-        accempty[2];
+        accempty[2], vfull[2], vempty[2];
     __shared__ uint32_t tmem_base, abort_flag;
 
     constexpr bool FWD = (MODE == SC_FWD);
@@ -105,6 +105,8 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             mbar_init(&xempty[i], 1 + 256);   // the MMAs (one commit) and the epilogue threads have read it
             mbar_init(&accfull[i], 1);
             mbar_init(&accempty[i], 256);
+            mbar_init(&vfull[i], 32);
+            mbar_init(&vempty[i], 256);
         }
         mbar_init(&mfull, 256);
         mbar_init(&mempty, 1);
@@ -199,24 +201,60 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                 umma_commit(&xempty[buf]);
             }
         }
-    } else {
+    } else if (warp == 10) {
+        // ------------------------------------------------------------ vector warp
+        // Per head: the 256 cumulative sums (log2 units) and step sizes of the chunk, the column factor
+        // of the mask factorisation and the 8 x 8 table of sub-tile-to-sub-tile decays, written to a
+        // double-buffered area one head ahead of the mask warps.  Each lane owns 8 consecutive steps.
+        float *vec = reinterpret_cast<float *>(smem + OFF_VEC);
+        for (int hi = 0; hi < nheads; ++hi) {
+            const int buf = hi & 1, h = h_begin + hi;
+            const size_t vo = ((((size_t)b * p.H + h) * p.ncs + c) << 8) + lane * 8;
+            const float4 c0 = __ldg(reinterpret_cast<const float4 *>(p.cs + vo));
+            const float4 c1 = __ldg(reinterpret_cast<const float4 *>(p.cs + vo + 4));
+            const float4 d0 = __ldg(reinterpret_cast<const float4 *>(p.dtT + vo));
+            const float4 d1 = __ldg(reinterpret_cast<const float4 *>(p.dtT + vo + 4));
+            if (hi >= 2) mbar_wait(&vempty[buf], ((hi >> 1) - 1) & 1, abortp, p.status);
+            float *cs2 = vec + buf * VEC_FLOATS, *cf = cs2 + 256, *dtv = cs2 + 512, *blk = cs2 + 768;
+            const float cv[8] = {c0.x * kLog2e, c0.y * kLog2e, c0.z * kLog2e, c0.w * kLog2e,
+                                 c1.x * kLog2e, c1.y * kLog2e, c1.z * kLog2e, c1.w * kLog2e};
+            const float dv[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+            *reinterpret_cast<float4 *>(cs2 + lane * 8) = make_float4(cv[0], cv[1], cv[2], cv[3]);
+            *reinterpret_cast<float4 *>(cs2 + lane * 8 + 4) = make_float4(cv[4], cv[5], cv[6], cv[7]);
+            *reinterpret_cast<float4 *>(dtv + lane * 8) = d0;
+            *reinterpret_cast<float4 *>(dtv + lane * 8 + 4) = d1;
+            __syncwarp();
+            const float ref = FWD ? cs2[(lane * 8) | 31] : cs2[(lane * 8) & ~31];
+            float o[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) o[k] = FWD ? ex2f(ref - cv[k]) * dv[k] : ex2f(cv[k] - ref);
+            *reinterpret_cast<float4 *>(cf + lane * 8) = make_float4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<float4 *>(cf + lane * 8 + 4) = make_float4(o[4], o[5], o[6], o[7]);
+#pragma unroll
+            for (int w = 0; w < 2; ++w) {
+                const int idx = lane + 32 * w, i = idx >> 3, j = idx & 7;   // blk[i][j] = e^{cs[32 i] - cs[32 j + 31]}, j < i
+                blk[idx] = (j < i) ? ex2f(cs2[32 * i] - cs2[32 * j + 31]) : 0.f;
+            }
+            mbar_arrive(&vfull[buf]);
+        }
+    } else if (warp >= 2) {
         // ------------------------------------------------------------ mask + epilogue warps
         // Two warps per TMEM lane quarter: warp (q, half) owns rows 32 q .. 32 q + 31 of the block and
         // the 32-column sub-tile `half` of every 64-column piece / columns 32 half .. of the accumulators.
+        // The eight warps meet only through mbarriers (and, in SC_DX, pairwise), never as a block.
         const int q = warp & 3;
         const int half = (warp - 2) >> 2;
-        const int mt = (warp - 2) * 32 + lane;     // 0..255 among the mask threads
         const int rl = q * 32 + lane;              // row inside the 128-row block
         const int r = rb * 128 + rl;               // row inside the chunk
         const int isub = r >> 5;
         const uint32_t tlane = (uint32_t)(q * 32) << 16;
         float *vec = reinterpret_cast<float *>(smem + OFF_VEC);
-        float *part = reinterpret_cast<float *>(smem + OFF_PART);
+        float *pairbuf = reinterpret_cast<float *>(smem + OFF_PART) + q * 128;   // [head parity][dd | dd2][32]
+        unsigned char *slab = smem + OFF_OUT + (warp - 2) * 2048;                // 32 rows x 64 B, this warp's
         float offs_prev = 0.f, dt_prev = 0.f;
 
-        // Epilogue of head hi.  The thread's x (and dy) row comes from the tiles TMA already brought to
-        // shared memory; the output tile is staged in shared memory (128-byte swizzle) and written with
-        // one TMA store, so no global access of this kernel is row-per-thread.
+        // Epilogue of head hi: x (and dy) come from the tiles TMA already brought to shared memory; the
+        // warp's 32 x 32 output block is staged in shared memory and written with its own TMA store.
         auto epilogue = [&](int hi, float offs, float dtr) {
             const int buf = hi & 1, h = h_begin + hi;
             uint4 xq[4], dyq[4];
@@ -249,8 +287,9 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             tmem_ld_wait32(a2);
             tc_fence_before_sync();
             mbar_arrive(&accempty[buf]);             // both accumulators are in registers now
+            if (lane == 0) tma_store_wait_read();    // this warp's previous store has read the slab
+            __syncwarp();
             float dd = 0.f, dd2 = 0.f, dsum = 0.f;
-            unsigned char *orow = smem + OFF_OUT + rl * 128;
 #pragma unroll
             for (int k8 = 0; k8 < 4; ++k8) {
                 float xv[8], dyv[8];
@@ -275,65 +314,39 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                         ow[e >> 1] = pack2(fmaf(Dh, dyv[e], dtr * u0), fmaf(Dh, dyv[e + 1], dtr * u1));
                     }
                 }
-                *reinterpret_cast<uint4 *>(orow + (((half * 4 + k8) ^ (rl & 7)) << 4)) = o;
-            }
-            float *pp = part + (hi & 1) * 264;
-            if (!FWD) {
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, off);
-                if (half == 1) {
-                    pp[rl] = dd;
-                    pp[136 + rl] = dd2;
-                }
-                if (lane == 0) pp[128 + (warp - 2)] = dsum;
+                *reinterpret_cast<uint4 *>(slab + lane * 64 + k8 * 16) = o;
             }
             fence_proxy_async_smem();
-            bar_mask_warps();
-            if (mt == 0) {
-                tma_store_3d(&tmOut, smem + OFF_OUT, h * 64, tok0 + rb * 128, b);
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_3d(&tmOut, slab, h * 64 + half * 32, tok0 + rb * 128 + q * 32, b);
                 tma_store_commit();
             }
             if (!FWD) {
-                // the two column halves of a row, and the eight warps' dy.x sums, in a fixed order
+                // dy.x of this warp's 32 x 32 block: one of 16 partials per (head, chunk), summed later in order
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, off);
+                if (lane == 0)
+                    p.dDp[((((size_t)b * p.H + h) * p.nct + p.c0 + c) << 4) + rb * 8 + (warp - 2)] = dsum;
+                // the two column halves of a row meet through shared memory, pairwise
+                float *pp = pairbuf + (hi & 1) * 64;
+                if (half == 1) {
+                    pp[lane] = dd;
+                    pp[32 + lane] = dd2;
+                }
+                asm volatile("bar.sync %0, 64;" ::"r"(2 + q) : "memory");
                 if (half == 0) {
                     const size_t vo = ((((size_t)b * p.H + h) * p.ncs + c) << 8) + r;
-                    p.ddt_dir[vo] = dd + pp[rl];
+                    p.ddt_dir[vo] = dd + pp[lane];
                     // psi2_s = B_s . (inter-chunk part of this head's dB_s) = dt_s e^{cs_last-cs_s} x_s . (Gout B_s)
-                    p.psi2[vo] = dtr * offs * (dd2 + pp[136 + rl]);
-                }
-                if (mt == 0) {
-                    float s = 0.f;
-#pragma unroll
-                    for (int w = 0; w < 8; ++w) s += pp[128 + w];
-                    float *dst = p.dDp + (((((size_t)b * p.H + h) * p.nct + p.c0 + c) << 2) + rb * 2);
-                    dst[0] = s;
-                    dst[1] = 0.f;
+                    p.psi2[vo] = dtr * offs * (dd2 + pp[32 + lane]);
                 }
             }
         };
-
-        // cs and dt of the head's 256 steps: one per thread, fetched one head ahead
-        float pre_cs, pre_dt;
-        auto fetch_vec = [&](int h) {
-            const size_t vo = (((size_t)b * p.H + h) * p.ncs + c) << 8;
-            pre_cs = __ldg(p.cs + vo + mt);
-            pre_dt = __ldg(p.dtT + vo + mt);
-        };
-        fetch_vec(h_begin);
 
         for (int hi = 0; hi < nheads; ++hi) {
             float *cs2 = vec + (hi & 1) * VEC_FLOATS, *cf = cs2 + 256, *dtv = cs2 + 512, *blk = cs2 + 768;
-            cs2[mt] = pre_cs * kLog2e;
-            dtv[mt] = pre_dt;
-            if (hi + 1 < nheads) fetch_vec(h_begin + hi + 1);
-            if (mt == 0) tma_store_wait_read();   // the staged tile of the last store may be overwritten after the barrier
-            bar_mask_warps();
-            cf[mt] = FWD ? ex2f(cs2[mt | 31] - cs2[mt]) * dtv[mt] : ex2f(cs2[mt] - cs2[mt & ~31]);
-            if (mt < 64) {
-                const int i = mt >> 3, j = mt & 7;   // blk[i][j] = e^{cs[32 i] - cs[32 j + 31]}, j < i
-                blk[mt] = (j < i) ? ex2f(cs2[32 * i] - cs2[32 * j + 31]) : 0.f;
-            }
-            bar_mask_warps();
+            mbar_wait(&vfull[hi & 1], (hi >> 1) & 1, abortp, p.status);
             const float csr = cs2[r];
             const float rowf = FWD ? ex2f(csr - cs2[r & ~31]) : ex2f(cs2[r | 31] - csr);
             const float offs = FWD ? ex2f(csr) : ex2f(cs2[255] - csr);
@@ -410,14 +423,13 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             tc_fence_before_sync();
             fence_proxy_async_smem();
             mbar_arrive(&mfull);
+            mbar_arrive(&vempty[hi & 1]);      // the head's vectors are no longer needed (the epilogue uses registers)
             if (hi >= 1) epilogue(hi - 1, offs_prev, dt_prev);
             offs_prev = offs;
             dt_prev = dtr;
         }
-        if (mt == 0) tma_store_wait_read();
-        bar_mask_warps();
         epilogue(nheads - 1, offs_prev, dt_prev);
-        if (mt == 0) tma_store_wait_all();
+        if (lane == 0) tma_store_wait_all();
     }
 
     tc_fence_before_sync();
