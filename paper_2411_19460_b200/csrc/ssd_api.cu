@@ -177,7 +177,7 @@ static void fill_params(const Plan &pl, const Layout &lo, void *ws, SegParams &s
     memset(&sp, 0, sizeof(sp));
     sp.B = pl.B; sp.L = pl.L; sp.H = pl.H; sp.P = pl.P; sp.N = pl.N; sp.G = pl.G; sp.Q = pl.Q;
     sp.hpg = pl.hpg; sp.ncs = pl.ncs; sp.nct = pl.nct; sp.nsl = pl.nsl;
-    sp.ndd = pl.use_tc ? 16 : pl.Q / 64;
+    sp.ndd = pl.use_tc ? 8 : pl.Q / 64;
     sp.x_bs = pl.x_bs; sp.dt_bs = pl.dt_bs; sp.bc_bs = pl.bc_bs;
     char *w = (char *)ws;
     sp.status = (unsigned int *)(w + lo.status);

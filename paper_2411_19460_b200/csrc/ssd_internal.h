@@ -72,7 +72,7 @@ cudaError_t launch_final_dAdD(const SegParams &p, float *dA, float *dD, cudaStre
 // ssd_tc.cu : tensor-core (tcgen05 / TMEM / TMA) kernels, bf16 I/O
 struct TcMaps {
     CUtensorMap x, dy, Bm, Cm;  // [B][L][H*64] / [B][L][G*128], box 64 x 128 rows
-    CUtensorMap y, dx;          // outputs, same geometry as x; box 32 columns x 32 rows, no swizzle (TMA stores)
+    CUtensorMap y, dx;          // outputs, same geometry as x; box 64 columns x 32 rows (TMA stores)
     CUtensorMap Hbf, Gbf;       // bf16 chunk states as [rows][128], box 64 x 64 rows
 };
 bool tc_supported(int dtype, int flags, int P, int N, int Q, int hpg);

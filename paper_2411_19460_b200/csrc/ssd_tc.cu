@@ -59,8 +59,8 @@ bool tc_make_maps(const SegParams &p, TcMaps &m) {
     bool ok = true;
     if (p.x) ok = ok && make_map3(&m.x, p.x, HP, p.L, p.B, HP, p.x_bs, 128);
     if (p.dy) ok = ok && make_map3(&m.dy, p.dy, HP, p.L, p.B, HP, p.x_bs, 128);
-    if (p.y) ok = ok && make_map3(&m.y, p.y, HP, p.L, p.B, HP, p.x_bs, 32, 32);
-    if (p.dx) ok = ok && make_map3(&m.dx, p.dx, HP, p.L, p.B, HP, p.x_bs, 32, 32);
+    if (p.y) ok = ok && make_map3(&m.y, p.y, HP, p.L, p.B, HP, p.x_bs, 32);
+    if (p.dx) ok = ok && make_map3(&m.dx, p.dx, HP, p.L, p.B, HP, p.x_bs, 32);
     if (p.Bm) ok = ok && make_map3(&m.Bm, p.Bm, GN, p.L, p.B, GN, p.bc_bs, 128);
     if (p.Cm) ok = ok && make_map3(&m.Cm, p.Cm, GN, p.L, p.B, GN, p.bc_bs, 128);
     // bf16 state copies viewed as [B*(ncs+1)*H*64 rows][128]

@@ -10,15 +10,18 @@
 //
 // One CTA owns (chunk, 128-row block, group, a range of the group's heads).  The score tile
 // S = Rows * Cols^T (128 x up to 256, K = N) is computed ONCE with tcgen05.mma into TMEM and stays
-// there in fp32 for every head of the range.  Per head the CTA then runs a three-role pipeline:
-//   producer warp : TMA loads of the head's value rows (x or dy) and its bf16 chunk state
-//   MMA warp      : acc2 = Rows * State^T (K = N), acc1 = M * V (K = up to 256 columns)
-//   vector warp   : the head's cumulative sums, step sizes and mask factors, one head ahead
-//   8 mask warps  : read S from TMEM, apply the decay mask, round to bf16 and store the masked
-//                   tile M to shared memory (A operand of the next MMA); then, while those MMAs run,
-//                   the epilogue of the previous head from the double-buffered accumulators.
-// One hand-off per head in each direction (mask -> MMA, MMA -> mask): a wait on an mbarrier costs
-// a few hundred cycles even when it is already complete, so the pipeline is kept coarse.
+// there in fp32 for every head of the range.  Per head the CTA runs five roles that meet only
+// through mbarriers:
+//   producer warp   : TMA loads of the head's value rows (x or dy; three stages, so a load is issued
+//                     two heads before it is needed: a 32 KB tile takes about 3000 cycles to land)
+//                     and of its bf16 chunk state (two buffers)
+//   MMA warp        : acc2 = Rows * State^T (K = N); acc1 += M_piece * V per 64-column piece
+//   vector warp     : the head's cumulative sums, step sizes and mask factors, one head ahead
+//   8 mask warps    : read S from TMEM, apply the decay mask, round to bf16 and store the piece of M
+//                     to a two-slot ring in shared memory (A operand of the next MMAs)
+//   4 epilogue warps: the previous head's accumulators (double-buffered in TMEM) -> y or dx; x and dy
+//                     come from the value tile already in shared memory, the output overwrites it in
+//                     place and leaves by one TMA store per warp, which then releases the stage.
 // The decay mask is factored per 32 x 32 sub-tile: strictly off-diagonal sub-tiles use
 //   e^{cs_t-cs_s} = e^{cs_t-cs_i0} * e^{cs_i0-cs_j1} * e^{cs_j1-cs_s}      (i0 = first row of the row
 // sub-tile, j1 = last column of the column sub-tile), three factors that are each <= 1 because cs
@@ -33,17 +36,15 @@ using namespace sm100;
 
 namespace {
 
-constexpr int SC_THREADS = 352;          // warp 0 producer, warp 1 MMA, warps 2..9 mask + epilogue, warp 10 vectors
+constexpr int SC_THREADS = 480;           // warp 0 producer, 1 MMA, 2..9 mask, 10 vectors, 11..14 epilogue
 constexpr uint32_t OFF_ROWS = 0;          // 32 KB  [n-half][128 rows][128 B]
-constexpr uint32_t OFF_BX = 32768;        // 64 KB  score columns operand, then two value buffers
-constexpr uint32_t OFF_M = 98304;         // 64 KB  four 16 KB pieces of the masked tile
-constexpr uint32_t OFF_ST = 163840;       // 16 KB  bf16 chunk state [n-half][64 rows][128 B]
-constexpr uint32_t OFF_OUT = 180224;      // 16 KB  eight 2 KB slabs (32 rows x 64 B), one per mask warp, staged for TMA stores
+constexpr uint32_t OFF_X = 32768;         // 3 x 32 KB value stages; first the score-columns operand (<= 64 KB)
+constexpr uint32_t OFF_M = 131072;        // 2 x 16 KB ring of masked pieces
+constexpr uint32_t OFF_ST = 163840;       // 2 x 16 KB  bf16 chunk state [n-half][64 rows][128 B]
 constexpr uint32_t OFF_XR = 196608;       // 16 KB  SC_DX: the head's x rows of this row block
 constexpr uint32_t OFF_VEC = 212992;      // per-head vectors, double buffered
 constexpr uint32_t VEC_FLOATS = 256 * 3 + 64;
-constexpr uint32_t OFF_PART = OFF_VEC + 2 * VEC_FLOATS * 4;   // 4 quarters x [head parity][dd | dd2][32] floats
-constexpr uint32_t SC_SMEM = OFF_PART + 4 * 128 * 4 + 1024;
+constexpr uint32_t SC_SMEM = OFF_VEC + 2 * VEC_FLOATS * 4 + 1024;
 
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -76,8 +77,8 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
           const __grid_constant__ CUtensorMap tmXr) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ uint64_t bar_ab, bar_s, xfull[2], xempty[2], hfull, hempty, xrfull, xrempty, mfull, mempty, accfull[2],
-        accempty[2], vfull[2], vempty[2];
+    __shared__ uint64_t bar_ab, bar_s, xfull[3], xempty[3], hfull[2], hempty[2], xrfull, xrempty, mfull[2], mempty[2],
+        accfull[2], accempty[2], vfull[2], vempty[2];
     __shared__ uint32_t tmem_base, abort_flag;
 
     constexpr bool FWD = (MODE == SC_FWD);
@@ -100,20 +101,22 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
     if (tid == 0) {
         mbar_init(&bar_ab, 1);
         mbar_init(&bar_s, 1);
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < 3; ++i) {
             mbar_init(&xfull[i], 1);
-            mbar_init(&xempty[i], 1 + 256);   // the MMAs (one commit) and the epilogue threads have read it
-            mbar_init(&accfull[i], 1);
-            mbar_init(&accempty[i], 256);
-            mbar_init(&vfull[i], 32);
-            mbar_init(&vempty[i], 256);
+            mbar_init(&xempty[i], 1 + 4);     // the MMAs (one commit) and the four output stores staged in it
         }
-        mbar_init(&mfull, 256);
-        mbar_init(&mempty, 1);
-        mbar_init(&hfull, 1);
-        mbar_init(&hempty, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&hfull[i], 1);
+            mbar_init(&hempty[i], 1);
+            mbar_init(&mfull[i], 256);
+            mbar_init(&mempty[i], 1);
+            mbar_init(&accfull[i], 1);
+            mbar_init(&accempty[i], 128);
+            mbar_init(&vfull[i], 32);
+            mbar_init(&vempty[i], 256 + 128);
+        }
         mbar_init(&xrfull, 1);
-        mbar_init(&xrempty, 256);
+        mbar_init(&xrempty, 128);
         abort_flag = 0;
         fence_barrier_init();
     }
@@ -133,21 +136,20 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             tma_load_3d(smem + OFF_ROWS + 16384, &tmRow, &bar_ab, g * 128 + 64, tok0 + rb * 128, b);
             for (int nh = 0; nh < 2; ++nh)
                 for (int r0 = 0; r0 < ncols; r0 += 128)
-                    tma_load_3d(smem + OFF_BX + nh * ncols * 128 + r0 * 128, &tmCol, &bar_ab, g * 128 + nh * 64,
+                    tma_load_3d(smem + OFF_X + nh * ncols * 128 + r0 * 128, &tmCol, &bar_ab, g * 128 + nh * 64,
                                 tok0 + colbase + r0, b);
             const int strow = (b * (p.ncs + 1) + slot) * p.H;
             for (int hi = 0; hi < nheads; ++hi) {
-                const int buf = hi & 1, h = h_begin + hi;
-                if (hi >= 1) mbar_wait(&hempty, (hi - 1) & 1, abortp, p.status);
-                mbar_arrive_expect_tx(&hfull, 16384);
-                tma_load_3d(smem + OFF_ST, &tmSt, &hfull, 0, (strow + h) * 64, 0);
-                tma_load_3d(smem + OFF_ST + 8192, &tmSt, &hfull, 64, (strow + h) * 64, 0);
+                const int buf = hi & 1, xs = hi % 3, xuse = hi / 3, h = h_begin + hi;
+                if (hi >= 2) mbar_wait(&hempty[buf], ((hi >> 1) - 1) & 1, abortp, p.status);
+                mbar_arrive_expect_tx(&hfull[buf], 16384);
+                tma_load_3d(smem + OFF_ST + buf * 16384, &tmSt, &hfull[buf], 0, (strow + h) * 64, 0);
+                tma_load_3d(smem + OFF_ST + buf * 16384 + 8192, &tmSt, &hfull[buf], 64, (strow + h) * 64, 0);
                 if (hi == 0) mbar_wait(&bar_s, 0, abortp, p.status);   // score MMAs done: the column operand is dead
-                if (hi >= 2) mbar_wait(&xempty[buf], ((hi >> 1) - 1) & 1, abortp, p.status);
-                mbar_arrive_expect_tx(&xfull[buf], (uint32_t)ncols * 128u);
+                if (xuse >= 1) mbar_wait(&xempty[xs], (xuse - 1) & 1, abortp, p.status);
+                mbar_arrive_expect_tx(&xfull[xs], (uint32_t)ncols * 128u);
                 for (int r0 = 0; r0 < ncols; r0 += 128)
-                    tma_load_3d(smem + OFF_BX + buf * 32768 + r0 * 128, &tmV, &xfull[buf], h * 64,
-                                tok0 + colbase + r0, b);
+                    tma_load_3d(smem + OFF_X + xs * 32768 + r0 * 128, &tmV, &xfull[xs], h * 64, tok0 + colbase + r0, b);
                 if (!FWD) {
                     if (hi >= 1) mbar_wait(&xrempty, (hi - 1) & 1, abortp, p.status);
                     mbar_arrive_expect_tx(&xrfull, 16384);
@@ -158,7 +160,7 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const uint32_t sRows = smem_u32(smem + OFF_ROWS), sBX = smem_u32(smem + OFF_BX);
+            const uint32_t sRows = smem_u32(smem + OFF_ROWS), sX = smem_u32(smem + OFF_X);
             const uint32_t sM = smem_u32(smem + OFF_M), sSt = smem_u32(smem + OFF_ST);
             const uint32_t idS = umma_idesc_bf16(128, (uint32_t)ncols, false, false);
             const uint32_t id3 = umma_idesc_bf16(128, 64, false, false);
@@ -168,44 +170,47 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk) {
                 const uint64_t ad = umma_desc_sw128(sRows + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024);
-                const uint64_t bd = umma_desc_sw128(sBX + (kk >> 2) * (ncols * 128) + (kk & 3) * 32, 16, 1024);
+                const uint64_t bd = umma_desc_sw128(sX + (kk >> 2) * (ncols * 128) + (kk & 3) * 32, 16, 1024);
                 umma_bf16(tm, ad, bd, idS, kk ? 1u : 0u);
             }
             umma_commit(&bar_s);
+            uint32_t mcnt = 0;   // pieces of M consumed so far
             for (int hi = 0; hi < nheads; ++hi) {
-                const int buf = hi & 1;
+                const int buf = hi & 1, xs = hi % 3, xuse = hi / 3;
                 const uint32_t acc1 = tm + 256 + buf * 128, acc2 = acc1 + 64;
                 if (hi >= 2) mbar_wait(&accempty[buf], ((hi >> 1) - 1) & 1, abortp, p.status);
-                mbar_wait(&hfull, hi & 1, abortp, p.status);
+                mbar_wait(&hfull[buf], (hi >> 1) & 1, abortp, p.status);
                 tc_fence_after_sync();
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
                     const uint64_t ad = umma_desc_sw128(sRows + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024);
-                    const uint64_t bd = umma_desc_sw128(sSt + (kk >> 2) * 8192 + (kk & 3) * 32, 16, 1024);
+                    const uint64_t bd = umma_desc_sw128(sSt + buf * 16384 + (kk >> 2) * 8192 + (kk & 3) * 32, 16, 1024);
                     umma_bf16(acc2, ad, bd, id3, kk ? 1u : 0u);
                 }
-                umma_commit(&hempty);
-                mbar_wait(&xfull[buf], (hi >> 1) & 1, abortp, p.status);
-                mbar_wait(&mfull, hi & 1, abortp, p.status);
-                tc_fence_after_sync();
+                umma_commit(&hempty[buf]);
+                mbar_wait(&xfull[xs], xuse & 1, abortp, p.status);
                 for (int jj = 0; jj < npieces; ++jj) {
+                    const uint32_t ms = mcnt & 1;
+                    mbar_wait(&mfull[ms], (mcnt >> 1) & 1, abortp, p.status);
+                    ++mcnt;
+                    tc_fence_after_sync();
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
-                        const uint64_t ad = umma_desc_sw128(sM + jj * 16384 + k * 32, 16, 1024);
-                        const uint64_t bd = umma_desc_sw128(sBX + buf * 32768 + (jj * 64 + k * 16) * 128, 8192, 1024);
+                        const uint64_t ad = umma_desc_sw128(sM + ms * 16384 + k * 32, 16, 1024);
+                        const uint64_t bd = umma_desc_sw128(sX + xs * 32768 + (jj * 64 + k * 16) * 128, 8192, 1024);
                         umma_bf16(acc1, ad, bd, id2, (jj | k) ? 1u : 0u);
                     }
+                    umma_commit(&mempty[ms]);
                 }
-                umma_commit(&mempty);
                 umma_commit(&accfull[buf]);
-                umma_commit(&xempty[buf]);
+                umma_commit(&xempty[xs]);
             }
         }
     } else if (warp == 10) {
         // ------------------------------------------------------------ vector warp
         // Per head: the 256 cumulative sums (log2 units) and step sizes of the chunk, the column factor
         // of the mask factorisation and the 8 x 8 table of sub-tile-to-sub-tile decays, written to a
-        // double-buffered area one head ahead of the mask warps.  Each lane owns 8 consecutive steps.
+        // double-buffered area one head ahead of their readers.  Each lane owns 8 consecutive steps.
         float *vec = reinterpret_cast<float *>(smem + OFF_VEC);
         for (int hi = 0; hi < nheads; ++hi) {
             const int buf = hi & 1, h = h_begin + hi;
@@ -237,11 +242,10 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             }
             mbar_arrive(&vfull[buf]);
         }
-    } else if (warp >= 2) {
-        // ------------------------------------------------------------ mask + epilogue warps
+    } else if (warp >= 2 && warp < 10) {
+        // ------------------------------------------------------------ mask warps
         // Two warps per TMEM lane quarter: warp (q, half) owns rows 32 q .. 32 q + 31 of the block and
-        // the 32-column sub-tile `half` of every 64-column piece / columns 32 half .. of the accumulators.
-        // The eight warps meet only through mbarriers (and, in SC_DX, pairwise), never as a block.
+        // the 32-column sub-tile `half` of every 64-column piece.
         const int q = warp & 3;
         const int half = (warp - 2) >> 2;
         const int rl = q * 32 + lane;              // row inside the 128-row block
@@ -249,186 +253,159 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
         const int isub = r >> 5;
         const uint32_t tlane = (uint32_t)(q * 32) << 16;
         float *vec = reinterpret_cast<float *>(smem + OFF_VEC);
-        float *pairbuf = reinterpret_cast<float *>(smem + OFF_PART) + q * 128;   // [head parity][dd | dd2][32]
-        unsigned char *slab = smem + OFF_OUT + (warp - 2) * 2048;                // 32 rows x 64 B, this warp's
-        float offs_prev = 0.f, dt_prev = 0.f;
-
-        // Epilogue of head hi: x (and dy) come from the tiles TMA already brought to shared memory; the
-        // warp's 32 x 32 output block is staged in shared memory and written with its own TMA store.
-        auto epilogue = [&](int hi, float offs, float dtr) {
-            const int buf = hi & 1, h = h_begin + hi;
-            uint4 xq[4], dyq[4];
-            mbar_wait(&xfull[buf], (hi >> 1) & 1, abortp, p.status);
-            if (FWD) {
-                const unsigned char *xrow = smem + OFF_BX + buf * 32768 + (rb * 128 + rl) * 128;
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    xq[k] = *reinterpret_cast<const uint4 *>(xrow + (((half * 4 + k) ^ (rl & 7)) << 4));
-            } else {
-                const unsigned char *dyrow = smem + OFF_BX + buf * 32768 + rl * 128;
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    dyq[k] = *reinterpret_cast<const uint4 *>(dyrow + (((half * 4 + k) ^ (rl & 7)) << 4));
-                mbar_wait(&xrfull, hi & 1, abortp, p.status);
-                const unsigned char *xrow = smem + OFF_XR + rl * 128;
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    xq[k] = *reinterpret_cast<const uint4 *>(xrow + (((half * 4 + k) ^ (rl & 7)) << 4));
-                mbar_arrive(&xrempty);
-            }
-            mbar_arrive(&xempty[buf]);
-            const float Dh = __ldg(p.D + h);
-            mbar_wait(&accfull[buf], (hi >> 1) & 1, abortp, p.status);
-            tc_fence_after_sync();
-            float a1[32], a2[32];
-            tmem_ld32_nowait(tm + tlane + 256 + buf * 128 + half * 32, a1);
-            tmem_ld32_nowait(tm + tlane + 320 + buf * 128 + half * 32, a2);
-            tmem_ld_wait32(a1);
-            tmem_ld_wait32(a2);
-            tc_fence_before_sync();
-            mbar_arrive(&accempty[buf]);             // both accumulators are in registers now
-            if (lane == 0) tma_store_wait_read();    // this warp's previous store has read the slab
-            __syncwarp();
-            float dd = 0.f, dd2 = 0.f, dsum = 0.f;
-#pragma unroll
-            for (int k8 = 0; k8 < 4; ++k8) {
-                float xv[8], dyv[8];
-                unpack8(xq[k8], xv);
-                if (!FWD) unpack8(dyq[k8], dyv);
-                uint4 o;
-                uint32_t *ow = reinterpret_cast<uint32_t *>(&o);
-#pragma unroll
-                for (int e = 0; e < 8; e += 2) {
-                    const int i = k8 * 8 + e;
-                    const float u0 = fmaf(offs, a2[i], a1[i]);
-                    const float u1 = fmaf(offs, a2[i + 1], a1[i + 1]);
-                    if (FWD) {
-                        ow[e >> 1] = pack2(fmaf(Dh, xv[e], u0), fmaf(Dh, xv[e + 1], u1));
-                    } else {
-                        dd = fmaf(xv[e], u0, dd);
-                        dd = fmaf(xv[e + 1], u1, dd);
-                        dd2 = fmaf(xv[e], a2[i], dd2);
-                        dd2 = fmaf(xv[e + 1], a2[i + 1], dd2);
-                        dsum = fmaf(dyv[e], xv[e], dsum);
-                        dsum = fmaf(dyv[e + 1], xv[e + 1], dsum);
-                        ow[e >> 1] = pack2(fmaf(Dh, dyv[e], dtr * u0), fmaf(Dh, dyv[e + 1], dtr * u1));
-                    }
-                }
-                *reinterpret_cast<uint4 *>(slab + lane * 64 + k8 * 16) = o;
-            }
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) {
-                tma_store_3d(&tmOut, slab, h * 64 + half * 32, tok0 + rb * 128 + q * 32, b);
-                tma_store_commit();
-            }
-            if (!FWD) {
-                // dy.x of this warp's 32 x 32 block: one of 16 partials per (head, chunk), summed later in order
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, off);
-                if (lane == 0)
-                    p.dDp[((((size_t)b * p.H + h) * p.nct + p.c0 + c) << 4) + rb * 8 + (warp - 2)] = dsum;
-                // the two column halves of a row meet through shared memory, pairwise
-                float *pp = pairbuf + (hi & 1) * 64;
-                if (half == 1) {
-                    pp[lane] = dd;
-                    pp[32 + lane] = dd2;
-                }
-                asm volatile("bar.sync %0, 64;" ::"r"(2 + q) : "memory");
-                if (half == 0) {
-                    const size_t vo = ((((size_t)b * p.H + h) * p.ncs + c) << 8) + r;
-                    p.ddt_dir[vo] = dd + pp[lane];
-                    // psi2_s = B_s . (inter-chunk part of this head's dB_s) = dt_s e^{cs_last-cs_s} x_s . (Gout B_s)
-                    p.psi2[vo] = dtr * offs * (dd2 + pp[32 + lane]);
-                }
-            }
-        };
+        uint32_t mcnt = 0;   // pieces of M produced so far
 
         for (int hi = 0; hi < nheads; ++hi) {
             float *cs2 = vec + (hi & 1) * VEC_FLOATS, *cf = cs2 + 256, *dtv = cs2 + 512, *blk = cs2 + 768;
             mbar_wait(&vfull[hi & 1], (hi >> 1) & 1, abortp, p.status);
             const float csr = cs2[r];
             const float rowf = FWD ? ex2f(csr - cs2[r & ~31]) : ex2f(cs2[r | 31] - csr);
-            const float offs = FWD ? ex2f(csr) : ex2f(cs2[255] - csr);
-            const float dtr = dtv[r];
-
-            if (hi == 0) mbar_wait(&bar_s, 0, abortp, p.status);
-            else mbar_wait(&mempty, (hi - 1) & 1, abortp, p.status);   // MMAs of the previous head have read M
-            tc_fence_after_sync();
-            // ---- masked tile: this thread's 32-column sub-tile of two 64-column pieces at a time
-            for (int j0 = 0; j0 < npieces; j0 += 2) {
-                float v[2][32];
-                bool z[2];
+            if (hi == 0) {
+                mbar_wait(&bar_s, 0, abortp, p.status);
+                tc_fence_after_sync();
+            }
+            for (int jj = 0; jj < npieces; ++jj) {
+                const int cb = colbase + jj * 64 + half * 32;   // first column of this thread's sub-tile (in chunk)
+                const int jsub = cb >> 5;
+                const bool zero = FWD ? (jsub > isub) : (jsub < isub);
+                uint32_t pk[16];
+                if (zero) {
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int jsub = ((colbase + (j0 + u) * 64) >> 5) + half;
-                    z[u] = FWD ? (jsub > isub) : (jsub < isub);
-                    if (!z[u]) tmem_ld32_nowait(tm + tlane + (j0 + u) * 64 + half * 32, v[u]);
-                }
+                    for (int k = 0; k < 16; ++k) pk[k] = 0u;
+                } else {
+                    float v[32];
+                    tmem_ld32(tm + tlane + jj * 64 + half * 32, v);
+                    if (jsub != isub) {
+                        const float f = rowf * (FWD ? blk[isub * 8 + jsub] : blk[jsub * 8 + isub]);
 #pragma unroll
-                for (int u = 0; u < 2; ++u)
-                    if (!z[u]) tmem_ld_wait32(v[u]);
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int jj = j0 + u;
-                    const int cb = colbase + jj * 64 + half * 32;   // first column of the sub-tile (in chunk)
-                    const int jsub = cb >> 5;
-                    unsigned char *mrow = smem + OFF_M + jj * 16384 + rl * 128;
-                    uint32_t pk[16];
-                    if (z[u]) {
-#pragma unroll
-                        for (int k = 0; k < 16; ++k) pk[k] = 0u;
+                        for (int k = 0; k < 32; k += 4) {
+                            const float4 cv = *reinterpret_cast<const float4 *>(cf + cb + k);
+                            v[k] *= cv.x * f;
+                            v[k + 1] *= cv.y * f;
+                            v[k + 2] *= cv.z * f;
+                            v[k + 3] *= cv.w * f;
+                        }
                     } else {
-                        float *vv = v[u];
-                        if (jsub != isub) {
-                            const float f = rowf * (FWD ? blk[isub * 8 + jsub] : blk[jsub * 8 + isub]);
 #pragma unroll
-                            for (int k = 0; k < 32; k += 4) {
-                                const float4 cv = *reinterpret_cast<const float4 *>(cf + cb + k);
-                                vv[k] *= cv.x * f;
-                                vv[k + 1] *= cv.y * f;
-                                vv[k + 2] *= cv.z * f;
-                                vv[k + 3] *= cv.w * f;
+                        for (int k = 0; k < 32; k += 4) {
+                            const float4 cc = *reinterpret_cast<const float4 *>(cs2 + cb + k);
+                            const float ccv[4] = {cc.x, cc.y, cc.z, cc.w};
+                            float dv[4] = {1.f, 1.f, 1.f, 1.f};
+                            if (FWD) {
+                                const float4 d4 = *reinterpret_cast<const float4 *>(dtv + cb + k);
+                                dv[0] = d4.x; dv[1] = d4.y; dv[2] = d4.z; dv[3] = d4.w;
                             }
-                        } else {
 #pragma unroll
-                            for (int k = 0; k < 32; k += 4) {
-                                const float4 cc = *reinterpret_cast<const float4 *>(cs2 + cb + k);
-                                const float ccv[4] = {cc.x, cc.y, cc.z, cc.w};
-                                float dv[4] = {1.f, 1.f, 1.f, 1.f};
-                                if (FWD) {
-                                    const float4 d4 = *reinterpret_cast<const float4 *>(dtv + cb + k);
-                                    dv[0] = d4.x; dv[1] = d4.y; dv[2] = d4.z; dv[3] = d4.w;
-                                }
-#pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const int col = cb + k + e;
-                                    const bool on = FWD ? (col <= r) : (col >= r);
-                                    const float ex = FWD ? ex2f(csr - ccv[e]) * dv[e] : ex2f(ccv[e] - csr);
-                                    vv[k + e] = on ? vv[k + e] * ex : 0.f;
-                                }
+                            for (int e = 0; e < 4; ++e) {
+                                const int col = cb + k + e;
+                                const bool on = FWD ? (col <= r) : (col >= r);
+                                const float ex = FWD ? ex2f(csr - ccv[e]) * dv[e] : ex2f(ccv[e] - csr);
+                                v[k + e] = on ? v[k + e] * ex : 0.f;
                             }
                         }
-#pragma unroll
-                        for (int k = 0; k < 16; ++k) pk[k] = pack2(vv[2 * k], vv[2 * k + 1]);
                     }
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        const int chunk16 = half * 4 + ch;
-                        *reinterpret_cast<uint4 *>(mrow + ((chunk16 ^ (rl & 7)) << 4)) =
-                            make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+                    for (int k = 0; k < 16; ++k) pk[k] = pack2(v[2 * k], v[2 * k + 1]);
+                }
+                // the ring slot is free once the MMAs of the piece that last used it are done
+                const uint32_t ms = mcnt & 1;
+                if (mcnt >= 2) mbar_wait(&mempty[ms], ((mcnt >> 1) - 1) & 1, abortp, p.status);
+                ++mcnt;
+                unsigned char *mrow = smem + OFF_M + ms * 16384 + rl * 128;
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    const int chunk16 = half * 4 + ch;
+                    *reinterpret_cast<uint4 *>(mrow + ((chunk16 ^ (rl & 7)) << 4)) =
+                        make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+                }
+                tc_fence_before_sync();
+                fence_proxy_async_smem();
+                mbar_arrive(&mfull[ms]);
+            }
+            mbar_arrive(&vempty[hi & 1]);
+        }
+    } else if (warp >= 11) {
+        // ------------------------------------------------------------ epilogue warps (one per TMEM lane quarter)
+        // x (and dy) come from the tiles TMA already brought to shared memory; the output overwrites the
+        // rows just read, in place (the MMAs of the head are done with the stage), and leaves by one TMA
+        // store per warp (32 rows x 64 columns), after which the warp releases the stage.
+        const int q = warp & 3;
+        const int rl = q * 32 + lane;              // row inside the 128-row block
+        const int r = rb * 128 + rl;               // row inside the chunk
+        const uint32_t tlane = (uint32_t)(q * 32) << 16;
+        const float *vec = reinterpret_cast<const float *>(smem + OFF_VEC);
+        for (int hi = 0; hi < nheads; ++hi) {
+            const int buf = hi & 1, xs = hi % 3, xuse = hi / 3, h = h_begin + hi;
+            const float *cs2 = vec + buf * VEC_FLOATS, *dtv = cs2 + 512;
+            mbar_wait(&vfull[buf], (hi >> 1) & 1, abortp, p.status);
+            const float csr = cs2[r];
+            const float offs = FWD ? ex2f(csr) : ex2f(cs2[255] - csr);
+            const float dtr = dtv[r];
+            mbar_arrive(&vempty[buf]);
+            const float Dh = __ldg(p.D + h);
+            mbar_wait(&xfull[xs], xuse & 1, abortp, p.status);
+            if (!FWD) mbar_wait(&xrfull, hi & 1, abortp, p.status);
+            unsigned char *blockbase = smem + OFF_X + xs * 32768 + ((FWD ? rb * 128 : 0) + q * 32) * 128;
+            unsigned char *vrow = blockbase + lane * 128;                 // x row (SC_FWD) / dy row (SC_DX), then output
+            const unsigned char *xrow = smem + OFF_XR + rl * 128;         // SC_DX: x row
+            mbar_wait(&accfull[buf], (hi >> 1) & 1, abortp, p.status);
+            tc_fence_after_sync();
+            float dd = 0.f, dd2 = 0.f, dsum = 0.f;
+#pragma unroll
+            for (int pass = 0; pass < 4; ++pass) {
+                float a1[16], a2[16];
+                tmem_ld16(tm + tlane + 256 + buf * 128 + pass * 16, a1);
+                tmem_ld16(tm + tlane + 320 + buf * 128 + pass * 16, a2);
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2) {
+                    const uint32_t off = (uint32_t)((2 * pass + c2) ^ (rl & 7)) << 4;
+                    float vv[8], xv[8];
+                    unpack8(*reinterpret_cast<const uint4 *>(vrow + off), vv);
+                    if (!FWD) unpack8(*reinterpret_cast<const uint4 *>(xrow + off), xv);
+                    uint4 o;
+                    uint32_t *ow = reinterpret_cast<uint32_t *>(&o);
+#pragma unroll
+                    for (int e = 0; e < 8; e += 2) {
+                        const int i = c2 * 8 + e;
+                        const float u0 = fmaf(offs, a2[i], a1[i]);
+                        const float u1 = fmaf(offs, a2[i + 1], a1[i + 1]);
+                        if (FWD) {
+                            ow[e >> 1] = pack2(fmaf(Dh, vv[e], u0), fmaf(Dh, vv[e + 1], u1));
+                        } else {
+                            dd = fmaf(xv[e], u0, dd);
+                            dd = fmaf(xv[e + 1], u1, dd);
+                            dd2 = fmaf(xv[e], a2[i], dd2);
+                            dd2 = fmaf(xv[e + 1], a2[i + 1], dd2);
+                            dsum = fmaf(vv[e], xv[e], dsum);
+                            dsum = fmaf(vv[e + 1], xv[e + 1], dsum);
+                            ow[e >> 1] = pack2(fmaf(Dh, vv[e], dtr * u0), fmaf(Dh, vv[e + 1], dtr * u1));
+                        }
                     }
+                    *reinterpret_cast<uint4 *>(vrow + off) = o;
                 }
             }
             tc_fence_before_sync();
+            mbar_arrive(&accempty[buf]);
+            if (!FWD) mbar_arrive(&xrempty);
             fence_proxy_async_smem();
-            mbar_arrive(&mfull);
-            mbar_arrive(&vempty[hi & 1]);      // the head's vectors are no longer needed (the epilogue uses registers)
-            if (hi >= 1) epilogue(hi - 1, offs_prev, dt_prev);
-            offs_prev = offs;
-            dt_prev = dtr;
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_3d(&tmOut, blockbase, h * 64, tok0 + rb * 128 + q * 32, b);
+                tma_store_commit();
+                tma_store_wait_read();              // the store has read the block: the stage may be refilled
+                mbar_arrive(&xempty[xs]);
+            }
+            if (!FWD) {
+                const size_t vo = ((((size_t)b * p.H + h) * p.ncs + c) << 8) + r;
+                p.ddt_dir[vo] = dd;
+                // psi2_s = B_s . (inter-chunk part of this head's dB_s) = dt_s e^{cs_last-cs_s} x_s . (Gout B_s)
+                p.psi2[vo] = dtr * offs * dd2;
+                // dy.x of this warp's 32 rows: one of 8 partials per (head, chunk), summed later in a fixed order
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, off);
+                if (lane == 0) p.dDp[((((size_t)b * p.H + h) * p.nct + p.c0 + c) << 4) + rb * 4 + q] = dsum;
+            }
         }
-        epilogue(nheads - 1, offs_prev, dt_prev);
         if (lane == 0) tma_store_wait_all();
     }
 
