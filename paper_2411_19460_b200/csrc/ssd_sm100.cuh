@@ -203,6 +203,12 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr, uint32_t lbo
     return d;
 }
 
+// The same descriptor for a start address `bytes` further on (a multiple of 16; the address field is the
+// low 14 bits in units of 16 bytes and shared memory is smaller than 256 KB, so a plain add cannot carry out).
+__device__ __forceinline__ uint64_t umma_desc_advance(uint64_t desc, uint32_t bytes) {
+    return desc + (uint64_t)(bytes >> 4);
+}
+
 // Instruction descriptor for kind::f16 with bf16 A/B and fp32 accumulation.
 __device__ __forceinline__ uint32_t umma_idesc_bf16(uint32_t M, uint32_t N, bool a_mn_major, bool b_mn_major) {
     uint32_t d = 0;

@@ -175,6 +175,9 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             }
             umma_commit(&bar_s);
             uint32_t mcnt = 0;   // pieces of M consumed so far
+            // descriptors of the loop-invariant operands, advanced by plain adds inside the loops
+            const uint64_t dRows = umma_desc_sw128(sRows, 16, 1024), dSt = umma_desc_sw128(sSt, 16, 1024);
+            const uint64_t dM = umma_desc_sw128(sM, 16, 1024), dX = umma_desc_sw128(sX, 8192, 1024);
             for (int hi = 0; hi < nheads; ++hi) {
                 const int buf = hi & 1, xs = hi % 3, xuse = hi / 3;
                 const uint32_t acc1 = tm + 256 + buf * 128, acc2 = acc1 + 64;
@@ -183,9 +186,8 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                 tc_fence_after_sync();
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
-                    const uint64_t ad = umma_desc_sw128(sRows + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024);
-                    const uint64_t bd = umma_desc_sw128(sSt + buf * 16384 + (kk >> 2) * 8192 + (kk & 3) * 32, 16, 1024);
-                    umma_bf16(acc2, ad, bd, id3, kk ? 1u : 0u);
+                    umma_bf16(acc2, umma_desc_advance(dRows, (kk >> 2) * 16384 + (kk & 3) * 32),
+                              umma_desc_advance(dSt, buf * 16384 + (kk >> 2) * 8192 + (kk & 3) * 32), id3, kk ? 1u : 0u);
                 }
                 umma_commit(&hempty[buf]);
                 mbar_wait(&xfull[xs], xuse & 1, abortp, p.status);
@@ -196,9 +198,8 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                     tc_fence_after_sync();
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
-                        const uint64_t ad = umma_desc_sw128(sM + ms * 16384 + k * 32, 16, 1024);
-                        const uint64_t bd = umma_desc_sw128(sX + xs * 32768 + (jj * 64 + k * 16) * 128, 8192, 1024);
-                        umma_bf16(acc1, ad, bd, id2, (jj | k) ? 1u : 0u);
+                        umma_bf16(acc1, umma_desc_advance(dM, ms * 16384 + k * 32),
+                                  umma_desc_advance(dX, xs * 32768 + (jj * 64 + k * 16) * 128), id2, (jj | k) ? 1u : 0u);
                     }
                     umma_commit(&mempty[ms]);
                 }
