@@ -1,0 +1,75 @@
+"""GPU parity at the full benchmark sizes, in the launch configuration bench.py times (default path,
+the config's own segment length).  The oracle cannot run 80 heads x 10^5..10^6 steps in seconds, so
+it computes a few sampled heads end to end (every output that is per head: y, h_final, boundary, dx,
+ddt, dA, dD, dh0), and dB/dC, which sum over the heads of a group, are checked on a whole group of a
+shorter sequence with the same head/group structure.  The segment-invariance property (bit-exact
+gradients for any segment length) is checked at full length as well."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2411_19460_b200.inputs import CONFIGS, make_inputs, to_f64_numpy
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+PER_HEAD = ("y", "h_final", "boundary", "dx", "ddt", "dA", "dD", "dh0")
+
+
+def _slice_heads(name, t, heads):
+    hi = torch.as_tensor(heads, device=t.device)
+    if name in ("y", "dx"):
+        return t.index_select(2, hi)          # [B, L, H, P]
+    if name == "ddt":
+        return t.index_select(2, hi)          # [B, L, H]
+    if name in ("h_final", "dh0"):
+        return t.index_select(1, hi)          # [B, H, P, N]
+    if name == "boundary":
+        return t.index_select(2, hi)          # [B, nseg, H, P, N]
+    return t.index_select(0, hi)              # dA, dD
+
+
+def _sampled_head_parity(cfg, heads):
+    inp = make_inputs(cfg, "cuda")
+    gpu = pu.run_gpu(cfg, inp)
+    hpg = cfg.H // cfg.G
+    d = to_f64_numpy(inp, heads=heads, groups=[h // hpg for h in heads])
+    # each sampled head keeps its own copy of its group's B/C, so the oracle sees H' heads in H' groups
+    ref = pu.run_oracle(d, cfg.seg)
+    errs = {}
+    for k in PER_HEAD:
+        errs[k] = pu.relerr(_slice_heads(k, gpu[k], heads), ref[k])
+    bad = {k: v for k, v in errs.items() if not (v <= pu.TOL[cfg.dtype])}
+    assert not bad, "parity failure at full size: %s | all %s" % (bad, errs)
+    return errs
+
+
+def test_config2_full_size_sampled_heads():
+    print(_sampled_head_parity(CONFIGS[2], heads=[0, 37, 79]))
+
+
+def test_config1_full_size_all_outputs():
+    errs = pu.full_parity(CONFIGS[1])
+    print(errs)
+
+
+def test_config4_shape_group_sums_on_shorter_sequence():
+    """Config 4's head/group structure (H=80, G=8, stiff decays) on 32768 steps: every output, all heads."""
+    cfg = CONFIGS[4].scaled(L=32768)
+    errs = pu.full_parity(cfg)
+    print(errs)
+
+
+def test_config4_full_size_sampled_heads():
+    print(_sampled_head_parity(CONFIGS[4], heads=[3, 76]))
+
+
+def test_config2_full_size_segment_invariance():
+    cfg = CONFIGS[2]
+    inp = make_inputs(cfg, "cuda")
+    a = pu.run_gpu(cfg, inp, seg=cfg.seg)
+    keep = {k: a[k].clone() for k in ("y", "h_final", "dx", "ddt", "dA", "dB", "dC", "dD", "dh0")}
+    del a
+    b = pu.run_gpu(cfg, inp, seg=16384)
+    for k, v in keep.items():
+        assert torch.equal(v, b[k]), k
