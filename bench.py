@@ -85,6 +85,33 @@ def load_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
+# ----------------------------------------------------------------------------- DRAM traffic from ncu
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the `ncu --set full` capture summarised in
+# profiles/ncu_full_tc_kernels_cfg1.txt (config 1: one launch = 2048 tokens x 24 heads).  A figure is used
+# only while the kernel's source file still has the hash it had when the counters were taken; it is scaled
+# to the timed workload by tokens x heads per launch (the traffic of these kernels grows in proportion).
+NCU_TRAFFIC_CFG1 = {
+    # kernel kind: (bytes per launch, source file, sha256 of that file at capture time)
+}
+NCU_CFG1_UNITS = 2048 * 24
+
+
+def ncu_traffic(kind, tokens_per_launch, heads):
+    ent = NCU_TRAFFIC_CFG1.get(kind)
+    if not ent:
+        return None
+    import hashlib
+    nbytes, src, sha = ent
+    path = os.path.join(ROOT, "paper_2411_19460_b200", "csrc", src)
+    try:
+        cur = hashlib.sha256(open(path, "rb").read()).hexdigest()
+    except OSError:
+        return None
+    if cur != sha:
+        return None
+    return nbytes * (tokens_per_launch * heads) / NCU_CFG1_UNITS
+
+
 # ----------------------------------------------------------------------------- clocks sampling
 class ClockSampler:
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -144,14 +171,13 @@ class ClockSampler:
 def run_ours(args):
     from paper_2411_19460_b200 import libssd
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    from paper_2411_19460_b200.replicas import Replicas
+
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
+    rep = Replicas(backend="nccl", device=dev)
+    rank, world = rep.rank, rep.world
     cfg = CONFIGS[args.config]
     if cfg.layers != 1:
         raise SystemExit("config %d is the layer-stack sweep; it is not a bench line" % args.config)
@@ -183,17 +209,8 @@ def run_ours(args):
         libssd.ssd_bwd_segmented(s["x"], s["dt"], s["A"], s["Bm"], s["Cm"], s["D"], bd, s["dy"], None,
                                  chunk=cfg.chunk, seg=seg, flags=flags, out=out, ws=ws_b, stream=stream)
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def max_over_ranks(v):
-        if world == 1:
-            return v
-        t = torch.tensor([v], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    barrier = rep.barrier
+    max_over_ranks = rep.max_over_ranks
 
     # ---- device-resident timing
     for _ in range(max(args.warmup, 3)):
@@ -260,8 +277,7 @@ def run_ours(args):
         del host_in, host_out, dev_in
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        rep.close()
         return
 
     peaks = load_peaks()
@@ -282,7 +298,8 @@ def run_ours(args):
         peak = peaks["hbm_gbs"]
         unit = "GB/s"
     roofline = dict(kernel=dom, bound="tensor" if bound == "tensor" else "hbm", achieved=achieved, peak=peak,
-                    unit=unit, frac=achieved / peak, traffic=None, peak_source=peaks["source"],
+                    unit=unit, frac=achieved / peak, traffic=ncu_traffic(dom, tok_per_launch, H),
+                    peak_source=peaks["source"],
                     avg_launch_us=avg_s * 1e6, launches=dom_n, share_of_device_time=dom_ms / total_prof)
     fl, by = step_model(cfg, seg)
     t_roof = max(fl * tokens / (peaks["bf16_tflops"] * 1e12), by * tokens / (peaks["hbm_gbs"] * 1e9))
@@ -314,8 +331,7 @@ def run_ours(args):
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    rep.close()
 
 
 # ----------------------------------------------------------------------------- the CPU oracle legs
