@@ -15,7 +15,8 @@
 // Per head:
 //   MMA warp   : score units S = Rows * Cols^T (K = P, 128 columns) into a TMEM buffer;
 //                acc += W * V per finished unit; acc += (scaled Rows) * State.
-//   8 mask warps: S -> W (decay mask, same factorisation and same bf16 rounding in both modes, so
+//   vector warp : the head's cumulative sums, step sizes and mask factors, one head ahead
+//   16 mask warps: S -> W (decay mask, same factorisation and same bf16 rounding in both modes, so
 //                that rho and psi are built from identical W and rho - psi cancels cleanly), stored
 //                to shared memory as the A operand; the row sums of W o CB give rho / psi; then the
 //                head's row operand scaled by e^{cs_t} (or dt_s e^{cs_last-cs_s}) as one more
@@ -32,7 +33,7 @@ using namespace sm100;
 
 namespace {
 
-constexpr int GB_THREADS = 320;           // warp 0 producer, warp 1 MMA, warps 2..9 mask
+constexpr int GB_THREADS = 608;           // warp 0 producer, warp 1 MMA, warps 2..17 mask, warp 18 vectors
 constexpr uint32_t GB_OFF_V = 0;          // 64 KB  [n-half][ncols rows][128 B], kept for all heads
 constexpr uint32_t GB_OFF_R = 65536;      // 2 x 16 KB  the head's row operand (dy or x rows of the block)
 constexpr uint32_t GB_OFF_C = 98304;      // 32 KB  the head's column operand (x or dy rows of the column range)
@@ -40,8 +41,8 @@ constexpr uint32_t GB_OFF_ST = 131072;    // 16 KB  bf16 chunk state [n-half][64
 constexpr uint32_t GB_OFF_M = 147456;     // 2 x 32 KB  masked units (two 16 KB pieces each); first use: C/B rows for CB
 constexpr uint32_t GB_OFF_VEC = 212992;   // per-head vectors, double buffered
 constexpr uint32_t GB_VEC_FLOATS = 256 * 3 + 64;
-constexpr uint32_t GB_OFF_PART = GB_OFF_VEC + 2 * GB_VEC_FLOATS * 4;   // 2 x 128 floats
-constexpr uint32_t GB_SMEM = GB_OFF_PART + 2 * 128 * 4 + 1024;
+constexpr uint32_t GB_OFF_PART = GB_OFF_VEC + 2 * GB_VEC_FLOATS * 4;   // 2 x 3 x 128 floats
+constexpr uint32_t GB_SMEM = GB_OFF_PART + 2 * 384 * 4 + 1024;
 
 constexpr uint32_t TM_CB = 0, TM_S = 256, TM_ACC = 384;
 
@@ -52,7 +53,6 @@ __device__ __forceinline__ float ex2f(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ void bar_mask_warps() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t *>(&v);
@@ -73,7 +73,7 @@ k_grad_bc_tc(SegParams p, const __grid_constant__ CUtensorMap tmRow,   // DC: dy
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     __shared__ uint64_t bar_ld, bar_cb, rfull[2], rempty[2], cfull[2], cempty[2], stfull, stempty, sfull, sempty,
-        mfull[2], mempty[2], accfull;
+        mfull[2], mempty[2], accfull, vfull[2], vempty[2];
     __shared__ uint32_t tmem_base, abort_flag;
 
     constexpr bool DC = (MODE == GB_DC);
@@ -98,16 +98,18 @@ k_grad_bc_tc(SegParams p, const __grid_constant__ CUtensorMap tmRow,   // DC: dy
         mbar_init(&bar_cb, 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(&rfull[i], 1);
-            mbar_init(&rempty[i], 1 + 256);   // inter-chunk MMAs (one commit) + the mask threads that scaled it
+            mbar_init(&rempty[i], 1 + 512);   // inter-chunk MMAs (one commit) + the mask threads that scaled it
             mbar_init(&cfull[i], 1);
             mbar_init(&cempty[i], 1);
-            mbar_init(&mfull[i], 256);
+            mbar_init(&mfull[i], 512);
+            mbar_init(&vfull[i], 32);
+            mbar_init(&vempty[i], 512);
             mbar_init(&mempty[i], 1);
         }
         mbar_init(&stfull, 1);
         mbar_init(&stempty, 1);
         mbar_init(&sfull, 1);
-        mbar_init(&sempty, 256);
+        mbar_init(&sempty, 512);
         mbar_init(&accfull, 1);
         abort_flag = 0;
         fence_barrier_init();
@@ -226,80 +228,88 @@ k_grad_bc_tc(SegParams p, const __grid_constant__ CUtensorMap tmRow,   // DC: dy
             }
             umma_commit(&accfull);
         }
+    } else if (warp == 18) {
+        // ------------------------------------------------------------ vector warp
+        // Per head: the 256 cumulative sums (log2 units) and step sizes of the chunk, the column factor
+        // of the mask factorisation and the 8 x 8 table of sub-tile-to-sub-tile decays, written to a
+        // double-buffered area one head ahead of the mask warps.  Each lane owns 8 consecutive steps.
+        if (nheads > 0) {
+            float *vec = reinterpret_cast<float *>(smem + GB_OFF_VEC);
+            for (int hi = 0; hi < nheads; ++hi) {
+                const int buf = hi & 1, h = h_begin + hi;
+                const size_t vo = ((((size_t)b * p.H + h) * p.ncs + c) << 8) + lane * 8;
+                const float4 c0 = __ldg(reinterpret_cast<const float4 *>(p.cs + vo));
+                const float4 c1 = __ldg(reinterpret_cast<const float4 *>(p.cs + vo + 4));
+                const float4 d0 = __ldg(reinterpret_cast<const float4 *>(p.dtT + vo));
+                const float4 d1 = __ldg(reinterpret_cast<const float4 *>(p.dtT + vo + 4));
+                if (hi >= 2) mbar_wait(&vempty[buf], ((hi >> 1) - 1) & 1, abortp, p.status);
+                float *cs2 = vec + buf * GB_VEC_FLOATS, *cf = cs2 + 256, *dtv = cs2 + 512, *blk = cs2 + 768;
+                const float cv[8] = {c0.x * kLog2e, c0.y * kLog2e, c0.z * kLog2e, c0.w * kLog2e,
+                                     c1.x * kLog2e, c1.y * kLog2e, c1.z * kLog2e, c1.w * kLog2e};
+                const float dv[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+                *reinterpret_cast<float4 *>(cs2 + lane * 8) = make_float4(cv[0], cv[1], cv[2], cv[3]);
+                *reinterpret_cast<float4 *>(cs2 + lane * 8 + 4) = make_float4(cv[4], cv[5], cv[6], cv[7]);
+                *reinterpret_cast<float4 *>(dtv + lane * 8) = d0;
+                *reinterpret_cast<float4 *>(dtv + lane * 8 + 4) = d1;
+                __syncwarp();
+                // cf: DC  e^{cs[t|31] - cs[t]} dt_t ; DB  e^{cs[t] - cs[t&~31]}
+                const float ref = DC ? cs2[(lane * 8) | 31] : cs2[(lane * 8) & ~31];
+                float o[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) o[k] = DC ? ex2f(ref - cv[k]) * dv[k] : ex2f(cv[k] - ref);
+                *reinterpret_cast<float4 *>(cf + lane * 8) = make_float4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<float4 *>(cf + lane * 8 + 4) = make_float4(o[4], o[5], o[6], o[7]);
+#pragma unroll
+                for (int w = 0; w < 2; ++w) {
+                    const int idx = lane + 32 * w, i = idx >> 3, j = idx & 7;   // blk[i][j] = e^{cs[32 i] - cs[32 j + 31]}, j < i
+                    blk[idx] = (j < i) ? ex2f(cs2[32 * i] - cs2[32 * j + 31]) : 0.f;
+                }
+                mbar_arrive(&vfull[buf]);
+            }
+        }
     } else if (nheads > 0) {
         // ------------------------------------------------------------ mask warps
-        // Two warps per TMEM lane quarter: warp (q, half) owns rows 32 q .. 32 q + 31 of the block and
-        // the 32-column sub-tile `half` of every 64-column piece.
+        // Four warps per TMEM lane quarter: warp (q, quar) owns rows 32 q .. 32 q + 31 of the block and
+        // the 16-column slice `quar` of every 64-column piece (columns 32 quar .. of the accumulator).
         const int q = warp & 3;
-        const int half = (warp - 2) >> 2;
-        const int mt = (warp - 2) * 32 + lane;     // 0..255 among the mask threads
+        const int quar = (warp - 2) >> 2;
         const int rl = q * 32 + lane;              // row inside the 128-row block
         const int r = rb * 128 + rl;               // row inside the chunk
         const int isub = r >> 5;
         const uint32_t tlane = (uint32_t)(q * 32) << 16;
         float *vec = reinterpret_cast<float *>(smem + GB_OFF_VEC);
-        float *part = reinterpret_cast<float *>(smem + GB_OFF_PART);
+        float *part = reinterpret_cast<float *>(smem + GB_OFF_PART);   // [head parity][3][128]
         uint32_t job = 0, sidx = 0;
-
-        float pre_cs, pre_dt;
-        auto fetch_vec = [&](int h) {
-            const size_t vo = (((size_t)b * p.H + h) * p.ncs + c) << 8;
-            pre_cs = __ldg(p.cs + vo + mt);
-            pre_dt = __ldg(p.dtT + vo + mt);
-        };
-        fetch_vec(h_begin);
-        float d_prev = 0.f;   // this thread's share of rho / psi of the previous head
-
-        auto flush_prev = [&](int hi_prev) {   // after a barrier: add the two column halves, store
-            if (half == 0) {
-                const size_t vo = ((((size_t)b * p.H + h_begin + hi_prev) * p.ncs + c) << 8) + r;
-                const float e = d_prev + part[(hi_prev & 1) * 128 + rl];
-                if (DC) p.rho[vo] = e;
-                else p.psi[vo] = e;
-            }
-        };
 
         for (int hi = 0; hi < nheads; ++hi) {
             float *cs2 = vec + (hi & 1) * GB_VEC_FLOATS, *cf = cs2 + 256, *dtv = cs2 + 512, *blk = cs2 + 768;
-            cs2[mt] = pre_cs * kLog2e;
-            dtv[mt] = pre_dt;
-            if (hi + 1 < nheads) fetch_vec(h_begin + hi + 1);
-            if (hi >= 1 && half == 1) part[((hi - 1) & 1) * 128 + rl] = d_prev;
-            bar_mask_warps();
-            if (hi >= 1) flush_prev(hi - 1);
-            // cf: DC  e^{cs[t|31] - cs[t]} dt_t  (column factor) ; DB  e^{cs[t] - cs[t&~31]} (column factor)
-            cf[mt] = DC ? ex2f(cs2[mt | 31] - cs2[mt]) * dtv[mt] : ex2f(cs2[mt] - cs2[mt & ~31]);
-            if (mt < 64) {
-                const int i = mt >> 3, j = mt & 7;   // blk[i][j] = e^{cs[32 i] - cs[32 j + 31]}, j < i
-                blk[mt] = (j < i) ? ex2f(cs2[32 * i] - cs2[32 * j + 31]) : 0.f;
-            }
-            bar_mask_warps();
+            mbar_wait(&vfull[hi & 1], (hi >> 1) & 1, abortp, p.status);
             const float csr = cs2[r];
             const float dtr = dtv[r];
             // row factor: DC  e^{cs_r - cs[r&~31]} ; DB  e^{cs[r|31] - cs_r} dt_r
             const float rowf = DC ? ex2f(csr - cs2[r & ~31]) : ex2f(cs2[r | 31] - csr) * dtr;
             const float offs = DC ? ex2f(csr) : ex2f(cs2[255] - csr) * dtr;
-            float dsum = 0.f;
+            float2 dacc = make_float2(0.f, 0.f);
             if (hi == 0) {
                 mbar_wait(&bar_cb, 0, abortp, p.status);
                 tc_fence_after_sync();
             }
 
             for (int u = 0; u < nunits; ++u) {
-                // ---- copy this thread's two score sub-tiles of the unit out of TMEM
-                float v[2][32];
+                // ---- copy this thread's two 16-column score slices of the unit out of TMEM
+                float v[2][16];
                 bool z[2];
                 mbar_wait(&sfull, sidx & 1, abortp, p.status);
                 tc_fence_after_sync();
 #pragma unroll
                 for (int w = 0; w < 2; ++w) {
-                    const int jsub = ((colbase + u * 128 + w * 64) >> 5) + half;
+                    const int jsub = (colbase + u * 128 + w * 64 + quar * 16) >> 5;
                     z[w] = DC ? (jsub > isub) : (jsub < isub);
-                    if (!z[w]) tmem_ld32_nowait(tm + tlane + TM_S + w * 64 + half * 32, v[w]);
+                    if (!z[w]) tmem_ld16_nowait(tm + tlane + TM_S + w * 64 + quar * 16, v[w]);
                 }
 #pragma unroll
                 for (int w = 0; w < 2; ++w)
-                    if (!z[w]) tmem_ld_wait32(v[w]);
+                    if (!z[w]) tmem_ld_wait16(v[w]);
                 tc_fence_before_sync();
                 mbar_arrive(&sempty);
                 ++sidx;
@@ -308,42 +318,38 @@ k_grad_bc_tc(SegParams p, const __grid_constant__ CUtensorMap tmRow,   // DC: dy
                 ++job;
 #pragma unroll
                 for (int w = 0; w < 2; ++w) {
-                    const int cb = colbase + u * 128 + w * 64 + half * 32;   // first column of the sub-tile (in chunk)
+                    const int cb = colbase + u * 128 + w * 64 + quar * 16;   // first column of the slice (in chunk)
                     const int jsub = cb >> 5;
                     unsigned char *mrow = smem + GB_OFF_M + mb * 32768 + w * 16384 + rl * 128;
-                    uint32_t pk[16];
+                    uint32_t pk[8];
                     if (z[w]) {
 #pragma unroll
-                        for (int k = 0; k < 16; ++k) pk[k] = 0u;
+                        for (int k = 0; k < 8; ++k) pk[k] = 0u;
                     } else {
                         float *vv = v[w];
-                        float cbv[32];
-                        tmem_ld32_nowait(tm + tlane + TM_CB + u * 128 + w * 64 + half * 32, cbv);
+                        float cbv[16];
+                        tmem_ld16_nowait(tm + tlane + TM_CB + u * 128 + w * 64 + quar * 16, cbv);
                         if (jsub != isub) {
-                            if (DC) {
-                                const float f = rowf * blk[isub * 8 + jsub];
+                            // (packed fp32 pairs; DC: cf (rowf blk) ; DB: rowf (cf blk) -- the same two factors
+                            //  (dn dt) and (up blk) multiplied in the same order in both modes)
+                            const float s1 = DC ? rowf * blk[isub * 8 + jsub] : blk[jsub * 8 + isub];
+                            const float2 s1v = make_float2(s1, s1), rfv = make_float2(rowf, rowf);
 #pragma unroll
-                                for (int k = 0; k < 32; k += 4) {
-                                    const float4 cv = *reinterpret_cast<const float4 *>(cf + cb + k);
-                                    vv[k] *= cv.x * f;
-                                    vv[k + 1] *= cv.y * f;
-                                    vv[k + 2] *= cv.z * f;
-                                    vv[k + 3] *= cv.w * f;
+                            for (int k = 0; k < 16; k += 4) {
+                                const float4 cv = *reinterpret_cast<const float4 *>(cf + cb + k);
+                                float2 m0 = __fmul2_rn(make_float2(cv.x, cv.y), s1v);
+                                float2 m1 = __fmul2_rn(make_float2(cv.z, cv.w), s1v);
+                                if (!DC) {
+                                    m0 = __fmul2_rn(rfv, m0);
+                                    m1 = __fmul2_rn(rfv, m1);
                                 }
-                            } else {
-                                const float bl = blk[jsub * 8 + isub];
-#pragma unroll
-                                for (int k = 0; k < 32; k += 4) {
-                                    const float4 cv = *reinterpret_cast<const float4 *>(cf + cb + k);
-                                    vv[k] *= rowf * (cv.x * bl);
-                                    vv[k + 1] *= rowf * (cv.y * bl);
-                                    vv[k + 2] *= rowf * (cv.z * bl);
-                                    vv[k + 3] *= rowf * (cv.w * bl);
-                                }
+                                const float2 w0 = __fmul2_rn(make_float2(vv[k], vv[k + 1]), m0);
+                                const float2 w1 = __fmul2_rn(make_float2(vv[k + 2], vv[k + 3]), m1);
+                                vv[k] = w0.x; vv[k + 1] = w0.y; vv[k + 2] = w1.x; vv[k + 3] = w1.y;
                             }
                         } else {
 #pragma unroll
-                            for (int k = 0; k < 32; k += 4) {
+                            for (int k = 0; k < 16; k += 4) {
                                 const float4 cc = *reinterpret_cast<const float4 *>(cs2 + cb + k);
                                 const float ccv[4] = {cc.x, cc.y, cc.z, cc.w};
                                 float dv[4] = {dtr, dtr, dtr, dtr};
@@ -361,19 +367,17 @@ k_grad_bc_tc(SegParams p, const __grid_constant__ CUtensorMap tmRow,   // DC: dy
                             }
                         }
 #pragma unroll
-                        for (int k = 0; k < 16; ++k) pk[k] = pack2(vv[2 * k], vv[2 * k + 1]);
-                        // row sum of (rounded W) o CB
-                        tmem_ld_wait32(cbv);
+                        for (int k = 0; k < 8; ++k) pk[k] = pack2(vv[2 * k], vv[2 * k + 1]);
+                        // row sum of W o CB, in fp32 from the unrounded W: both modes form bit-identical
+                        // W and CB elements, so rho and psi are row and column sums of one matrix
+                        tmem_ld_wait16(cbv);
 #pragma unroll
-                        for (int k = 0; k < 16; ++k) {
-                            const float2 wv = unpack2(pk[k]);
-                            dsum = fmaf(wv.x, cbv[2 * k], dsum);
-                            dsum = fmaf(wv.y, cbv[2 * k + 1], dsum);
-                        }
+                        for (int k = 0; k < 16; k += 2)
+                            dacc = __ffma2_rn(make_float2(vv[k], vv[k + 1]), make_float2(cbv[k], cbv[k + 1]), dacc);
                     }
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        const int chunk16 = half * 4 + ch;
+                    for (int ch = 0; ch < 2; ++ch) {
+                        const int chunk16 = quar * 2 + ch;
                         *reinterpret_cast<uint4 *>(mrow + ((chunk16 ^ (rl & 7)) << 4)) =
                             make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
                     }
@@ -382,16 +386,17 @@ k_grad_bc_tc(SegParams p, const __grid_constant__ CUtensorMap tmRow,   // DC: dy
                 fence_proxy_async_smem();
                 mbar_arrive(&mfull[mb]);
             }
+            mbar_arrive(&vempty[hi & 1]);
 
-            // ---- inter-chunk piece: this thread's 32 values of its row of the head's row operand, scaled
+            // ---- inter-chunk piece: this thread's 16 values of its row of the head's row operand, scaled
             {
                 const int rbuf = hi & 1;
                 mbar_wait(&rfull[rbuf], (hi >> 1) & 1, abortp, p.status);
                 const unsigned char *rrow = smem + GB_OFF_R + rbuf * 16384 + rl * 128;
-                uint4 o[4];
+                uint4 o[2];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const uint4 qv = *reinterpret_cast<const uint4 *>(rrow + (((half * 4 + k) ^ (rl & 7)) << 4));
+                for (int k = 0; k < 2; ++k) {
+                    const uint4 qv = *reinterpret_cast<const uint4 *>(rrow + (((quar * 2 + k) ^ (rl & 7)) << 4));
                     const uint32_t *qw = reinterpret_cast<const uint32_t *>(&qv);
                     uint32_t *ow = reinterpret_cast<uint32_t *>(&o[k]);
 #pragma unroll
@@ -406,16 +411,26 @@ k_grad_bc_tc(SegParams p, const __grid_constant__ CUtensorMap tmRow,   // DC: dy
                 ++job;
                 unsigned char *mrow = smem + GB_OFF_M + mb * 32768 + rl * 128;
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    *reinterpret_cast<uint4 *>(mrow + (((half * 4 + k) ^ (rl & 7)) << 4)) = o[k];
+                for (int k = 0; k < 2; ++k)
+                    *reinterpret_cast<uint4 *>(mrow + (((quar * 2 + k) ^ (rl & 7)) << 4)) = o[k];
                 fence_proxy_async_smem();
                 mbar_arrive(&mfull[mb]);
             }
-            d_prev = dsum;
+
+            // ---- rho / psi of this head: the four column slices of a row meet through shared memory
+            {
+                const float dsum = dacc.x + dacc.y;
+                float *pp = part + (hi & 1) * 384;
+                if (quar > 0) pp[(quar - 1) * 128 + rl] = dsum;
+                asm volatile("bar.sync %0, 128;" ::"r"(2 + q) : "memory");
+                if (quar == 0) {
+                    const size_t vo = ((((size_t)b * p.H + h_begin + hi) * p.ncs + c) << 8) + r;
+                    const float e = ((dsum + pp[rl]) + pp[128 + rl]) + pp[256 + rl];
+                    if (DC) p.rho[vo] = e;
+                    else p.psi[vo] = e;
+                }
+            }
         }
-        if (half == 1) part[((nheads - 1) & 1) * 128 + rl] = d_prev;
-        bar_mask_warps();
-        flush_prev(nheads - 1);
 
         // ---- the CTA's partial slice of the group sum: [B, seg, G, nsl, N] fp32
         mbar_wait(&accfull, 0, abortp, p.status);
@@ -423,15 +438,12 @@ k_grad_bc_tc(SegParams p, const __grid_constant__ CUtensorMap tmRow,   // DC: dy
         {
             const size_t segcap = (size_t)p.ncs * 256;
             const size_t tl = (size_t)c * 256 + r;
-            float *dst = (DC ? p.pC : p.pB) + ((((size_t)b * segcap + tl) * p.G + g) * nsl + sl) * 128 + half * 64;
+            float *dst = (DC ? p.pC : p.pB) + ((((size_t)b * segcap + tl) * p.G + g) * nsl + sl) * 128 + quar * 32;
+            float a[32];
+            tmem_ld32(tm + tlane + TM_ACC + quar * 32, a);
 #pragma unroll
-            for (int blk32 = 0; blk32 < 2; ++blk32) {
-                float a[32];
-                tmem_ld32(tm + tlane + TM_ACC + half * 64 + blk32 * 32, a);
-#pragma unroll
-                for (int k = 0; k < 32; k += 4)
-                    *reinterpret_cast<float4 *>(dst + blk32 * 32 + k) = make_float4(a[k], a[k + 1], a[k + 2], a[k + 3]);
-            }
+            for (int k = 0; k < 32; k += 4)
+                *reinterpret_cast<float4 *>(dst + k) = make_float4(a[k], a[k + 1], a[k + 2], a[k + 3]);
         }
     }
 
