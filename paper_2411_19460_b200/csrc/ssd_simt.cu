@@ -30,53 +30,52 @@ __device__ __forceinline__ size_t vec_off(const SegParams &p, int b, int h, int 
 }
 
 // ------------------------------------------------------------------ a1: chunk cumsum
-// One CTA per (chunk, block of 32 heads, batch).  The dt[b, t, h0..h0+31] rows (128 contiguous
-// bytes each) are staged through shared memory so global reads are coalesced; each warp then scans
-// four heads: a lane owns Q/32 consecutive steps (serial prefix), lane totals are combined with a
-// warp-shuffle scan.
+// One CTA per (chunk, block of 8 heads, batch), one warp per head.  The dt[b, t, h0..h0+7] pieces
+// (32 contiguous bytes per step) are staged through shared memory; a lane owns Q/32 consecutive
+// steps (serial prefix), lane totals are combined with a warp-shuffle scan.
 __global__ void __launch_bounds__(256) k_chunk_cumsum(SegParams p) {
-    __shared__ float tile[256][33];
-    const int c = blockIdx.x, h0 = blockIdx.y * 32, b = blockIdx.z;
+    __shared__ float tile[256][9];
+    const int c = blockIdx.x, h0 = blockIdx.y * 8, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int Q = p.Q, per = Q >> 5;
     const size_t tok0 = (size_t)p.t0 + (size_t)c * Q;
-    const int nh = min(32, p.H - h0);
-    for (int idx = tid; idx < Q * 32; idx += 256) {
-        const int t = idx >> 5, hh = idx & 31;
+    const int nh = min(8, p.H - h0);
+    for (int idx = tid; idx < Q * 8; idx += 256) {
+        const int t = idx >> 3, hh = idx & 7;
         if (hh < nh) tile[t][hh] = __ldg(p.dt + (size_t)b * p.dt_bs + (tok0 + t) * p.H + h0 + hh);
     }
     __syncthreads();
-    for (int hh = warp; hh < nh; hh += 8) {
-        const float Ah = __ldg(p.A + h0 + hh);
-        float a[8], d[8];
-        float run = 0.f;
+    const int hh = warp;
+    if (hh >= nh) return;
+    const float Ah = __ldg(p.A + h0 + hh);
+    float a[8], d[8];
+    float run = 0.f;
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-            if (j < per) {
-                d[j] = tile[lane * per + j][hh];
-                run += d[j] * Ah;
-                a[j] = run;
-            }
-        float incl = run;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const float v = __shfl_up_sync(0xffffffffu, incl, off);
-            if (lane >= off) incl += v;
+    for (int j = 0; j < 8; ++j)
+        if (j < per) {
+            d[j] = tile[lane * per + j][hh];
+            run += d[j] * Ah;
+            a[j] = run;
         }
-        float excl = __shfl_up_sync(0xffffffffu, incl, 1);
-        if (lane == 0) excl = 0.f;
-        const size_t o = vec_off(p, b, h0 + hh, c) + (size_t)lane * per;
+    float incl = run;
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-            if (j < per) {
-                p.cs[o + j] = a[j] + excl;
-                p.dtT[o + j] = d[j];
-            }
+    for (int off = 1; off < 32; off <<= 1) {
+        const float v = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += v;
     }
+    float excl = __shfl_up_sync(0xffffffffu, incl, 1);
+    if (lane == 0) excl = 0.f;
+    const size_t o = vec_off(p, b, h0 + hh, c) + (size_t)lane * per;
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        if (j < per) {
+            p.cs[o + j] = a[j] + excl;
+            p.dtT[o + j] = d[j];
+        }
 }
 
 cudaError_t launch_chunk_cumsum(const SegParams &p, cudaStream_t st) {
-    k_chunk_cumsum<<<dim3(p.nc, (p.H + 31) / 32, p.B), 256, 0, st>>>(p);
+    k_chunk_cumsum<<<dim3(p.nc, (p.H + 7) / 8, p.B), 256, 0, st>>>(p);
     return cudaGetLastError();
 }
 
@@ -167,25 +166,42 @@ k_state_pass_fwd(SegParams p, const float *init, long long init_bs, float *bound
     if (boundary_out)
         *reinterpret_cast<float4 *>(boundary_out + (size_t)b * bnd_bs + (size_t)h * PN + e) = carry;
     const float *csl = p.cs + vec_off(p, b, h, 0) + (p.Q - 1);
-    for (int c = 0; c <= p.nc; ++c) {
-        const size_t so = slot_off(p, b, c, h) + e;
-        if (c > 0) {
-            const float decay = expf(csl[(size_t)(c - 1) * p.Q]);
-            const float4 s = *reinterpret_cast<const float4 *>(p.Hst + so);
-            carry.x = fmaf(decay, carry.x, s.x);
-            carry.y = fmaf(decay, carry.y, s.y);
-            carry.z = fmaf(decay, carry.z, s.z);
-            carry.w = fmaf(decay, carry.w, s.w);
-        }
-        *reinterpret_cast<float4 *>(p.Hst + so) = carry;
+    // tensor-core path: every later reader takes the bf16 copy, so the fp32 chunk-entry states are
+    // not written back (the fp32 carry still goes from segment to segment)
+    auto put = [&](size_t so, const float4 &v) {
+        if (!want_bf16) *reinterpret_cast<float4 *>(p.Hst + so) = v;
         if (want_bf16) {
-            __nv_bfloat162 lo = __floats2bfloat162_rn(carry.x, carry.y);
-            __nv_bfloat162 hi = __floats2bfloat162_rn(carry.z, carry.w);
+            __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
+            __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
             uint2 pk;
             pk.x = *reinterpret_cast<unsigned int *>(&lo);
             pk.y = *reinterpret_cast<unsigned int *>(&hi);
             *reinterpret_cast<uint2 *>(p.Hbf + so) = pk;
         }
+    };
+    put(slot_off(p, b, 0, h) + e, carry);
+    // The chunk sums and decays do not depend on the carry: fetch eight chunks ahead of the serial
+    // recurrence, so that a segment costs a few memory latencies instead of one per chunk.
+    constexpr int PF = 8;
+    for (int c0 = 1; c0 <= p.nc; c0 += PF) {
+        float4 sv[PF];
+        float dec[PF];
+#pragma unroll
+        for (int k = 0; k < PF; ++k)
+            if (c0 + k <= p.nc) {
+                sv[k] = *reinterpret_cast<const float4 *>(p.Hst + slot_off(p, b, c0 + k, h) + e);
+                dec[k] = csl[(size_t)(c0 + k - 1) * p.Q];
+            }
+#pragma unroll
+        for (int k = 0; k < PF; ++k)
+            if (c0 + k <= p.nc) {
+                const float decay = expf(dec[k]);
+                carry.x = fmaf(decay, carry.x, sv[k].x);
+                carry.y = fmaf(decay, carry.y, sv[k].y);
+                carry.z = fmaf(decay, carry.z, sv[k].z);
+                carry.w = fmaf(decay, carry.w, sv[k].w);
+                put(slot_off(p, b, c0 + k, h) + e, carry);
+            }
     }
     *reinterpret_cast<float4 *>(p.hcarry + bh) = carry;
     if (final_out) *reinterpret_cast<float4 *>(final_out + bh) = carry;
@@ -206,7 +222,7 @@ cudaError_t launch_state_pass_fwd(const SegParams &p, const float *init, long lo
 // the part of da_t that couples the gradient from the right with the state from the left.
 __global__ void __launch_bounds__(256)
 k_state_pass_bwd(SegParams p, const float *init, float *left_out, int want_bf16) {
-    __shared__ float red[2][8];
+    __shared__ float red[8][8];
     const int h = blockIdx.y, b = blockIdx.z;
     const int PN = p.P * p.N;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -215,41 +231,65 @@ k_state_pass_bwd(SegParams p, const float *init, float *left_out, int want_bf16)
     float4 carry = make_float4(0.f, 0.f, 0.f, 0.f);
     if (init) carry = *reinterpret_cast<const float4 *>(init + bh);
     const float *csl = p.cs + vec_off(p, b, h, 0) + (p.Q - 1);
-    for (int c = p.nc; c >= 0; --c) {
-        const size_t so = slot_off(p, b, c, h) + e;
-        if (c < p.nc) {
-            // carry is Gout of chunk c here (slot c+1); Hst slot c is the state entering chunk c
-            const float decay = expf(csl[(size_t)c * p.Q]);
-            const float4 hv = *reinterpret_cast<const float4 *>(p.Hst + so);
-            float part = carry.x * hv.x;
-            part = fmaf(carry.y, hv.y, part);
-            part = fmaf(carry.z, hv.z, part);
-            part = fmaf(carry.w, hv.w, part);
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
-            if (lane == 0) red[c & 1][warp] = part;
-            __syncthreads();
-            if (tid == 0) {
-                float s = 0.f;
-#pragma unroll
-                for (int w = 0; w < 8; ++w) s += red[c & 1][w];
-                p.ghdot[((((size_t)b * p.H + h) * p.ncs + c) << 3) + blockIdx.x] = decay * s;
-            }
-            const float4 ev = *reinterpret_cast<const float4 *>(p.Gst + so);
-            carry.x = fmaf(decay, carry.x, ev.x);
-            carry.y = fmaf(decay, carry.y, ev.y);
-            carry.z = fmaf(decay, carry.z, ev.z);
-            carry.w = fmaf(decay, carry.w, ev.w);
-        }
-        *reinterpret_cast<float4 *>(p.Gst + so) = carry;
+    auto put = [&](size_t so, const float4 &v) {
+        if (!want_bf16) *reinterpret_cast<float4 *>(p.Gst + so) = v;
         if (want_bf16) {
-            __nv_bfloat162 lo = __floats2bfloat162_rn(carry.x, carry.y);
-            __nv_bfloat162 hi = __floats2bfloat162_rn(carry.z, carry.w);
+            __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
+            __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
             uint2 pk;
             pk.x = *reinterpret_cast<unsigned int *>(&lo);
             pk.y = *reinterpret_cast<unsigned int *>(&hi);
             *reinterpret_cast<uint2 *>(p.Gbf + so) = pk;
         }
+    };
+    put(slot_off(p, b, p.nc, h) + e, carry);
+    // Eight chunks at a time: their E_c, entry states and decays are fetched ahead of the serial
+    // recurrence; the eight <Gout, H_in> partials of a batch share one block-wide reduction step.
+    constexpr int PF = 8;
+    for (int c0 = p.nc - 1; c0 >= 0; c0 -= PF) {
+        float4 ev[PF], hv[PF];
+        float dec[PF];
+#pragma unroll
+        for (int k = 0; k < PF; ++k)
+            if (c0 - k >= 0) {
+                const size_t so = slot_off(p, b, c0 - k, h) + e;
+                ev[k] = *reinterpret_cast<const float4 *>(p.Gst + so);
+                if (want_bf16) {   // entry state from its bf16 copy (the fp32 one was not kept)
+                    const uint2 pk = *reinterpret_cast<const uint2 *>(p.Hbf + so);
+                    const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&pk.x));
+                    const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&pk.y));
+                    hv[k] = make_float4(lo.x, lo.y, hi.x, hi.y);
+                } else {
+                    hv[k] = *reinterpret_cast<const float4 *>(p.Hst + so);
+                }
+                dec[k] = csl[(size_t)(c0 - k) * p.Q];
+            }
+#pragma unroll
+        for (int k = 0; k < PF; ++k)
+            if (c0 - k >= 0) {
+                // carry is Gout of chunk c = c0 - k here; hv[k] is the state entering chunk c
+                const float decay = expf(dec[k]);
+                float part = carry.x * hv[k].x;
+                part = fmaf(carry.y, hv[k].y, part);
+                part = fmaf(carry.z, hv[k].z, part);
+                part = fmaf(carry.w, hv[k].w, part);
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+                if (lane == 0) red[k][warp] = decay * part;
+                carry.x = fmaf(decay, carry.x, ev[k].x);
+                carry.y = fmaf(decay, carry.y, ev[k].y);
+                carry.z = fmaf(decay, carry.z, ev[k].z);
+                carry.w = fmaf(decay, carry.w, ev[k].w);
+                put(slot_off(p, b, c0 - k, h) + e, carry);
+            }
+        __syncthreads();
+        if (tid < PF && c0 - tid >= 0) {
+            float s = 0.f;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) s += red[tid][w];
+            p.ghdot[((((size_t)b * p.H + h) * p.ncs + (c0 - tid)) << 3) + blockIdx.x] = s;
+        }
+        __syncthreads();
     }
     *reinterpret_cast<float4 *>(left_out + bh) = carry;
 }
