@@ -55,6 +55,46 @@ struct Plan {
     size_t esz;
 };
 
+// How many head ranges per group for the tensor-core kernels whose CTAs are (chunk, 128-row block,
+// head range).  Half of the CTAs do about 1.8 times the work of the other half (causal structure) and
+// are launched first; one CTA per SM, kNumSMs SMs.  The split that minimises the makespan of a greedy
+// schedule is taken (cost of a CTA: one head-time of set-up plus its heads).
+static int best_head_split(int nchunks, int groups, int batch, int hpg, int max_split) {
+    const int kNumSMs = 148;
+    // the driver asks once per segment: remember the last few answers
+    struct Memo { int nchunks, groups, batch, hpg, max_split, answer; };
+    static thread_local Memo memo[4] = {};
+    static thread_local int memo_next = 0;
+    for (const Memo &m : memo)
+        if (m.answer > 0 && m.nchunks == nchunks && m.groups == groups && m.batch == batch && m.hpg == hpg &&
+            m.max_split == max_split)
+            return m.answer;
+    int best = 1;
+    double best_t = 1e300;
+    for (int ns = 1; ns <= max_split; ++ns) {
+        const int hps = (hpg + ns - 1) / ns;
+        if ((hpg + hps - 1) / hps != ns) continue;   // would leave an empty range
+        double sm[kNumSMs];
+        for (int i = 0; i < kNumSMs; ++i) sm[i] = 0.0;
+        double makespan = 0.0;
+        for (int pass = 0; pass < 2; ++pass)          // all long CTAs, then all short ones
+            for (int j = 0; j < nchunks * groups * batch; ++j)
+                for (int r = 0; r < ns; ++r) {
+                    const int heads = (r == ns - 1) ? hpg - hps * (ns - 1) : hps;
+                    const double cost = 1.0 + heads * (pass == 0 ? 1.0 : 0.55);
+                    int arg = 0;
+                    for (int i = 1; i < kNumSMs; ++i)
+                        if (sm[i] < sm[arg]) arg = i;
+                    sm[arg] += cost;
+                    if (sm[arg] > makespan) makespan = sm[arg];
+                }
+        if (makespan < best_t - 1e-9) { best_t = makespan; best = ns; }
+    }
+    memo[memo_next] = Memo{nchunks, groups, batch, hpg, max_split, best};
+    memo_next = (memo_next + 1) & 3;
+    return best;
+}
+
 static int make_plan(const ssd_shape_t *s, Plan &pl) {
     if (!s) return SSD_EINVAL;
     if (s->B <= 0 || s->L <= 0 || s->H <= 0 || s->P <= 0 || s->N <= 0 || s->G <= 0 || s->chunk <= 0 ||
@@ -88,12 +128,11 @@ static int make_plan(const ssd_shape_t *s, Plan &pl) {
         return SSD_EALIGN;
     pl.use_tc = tc_supported(s->dtype, s->flags, s->P, s->N, s->chunk, pl.hpg);
     // Partial slices of the dB/dC head sums.  CUDA-core kernels: one head per slice.  Tensor-core
-    // kernels: one slice per CTA head range of at most 16 heads.  A function of H/G only, so the
-    // summation order, and with it every bit of dB/dC, is the same for every segment length.
+    // kernels: one slice per CTA head range, chosen for a reference launch of 16 chunks (at least 4
+    // heads per range).  A function of H and G only, so the summation order, and with it every bit
+    // of dB/dC, is the same for every segment length.
     if (pl.use_tc) {
-        const int want = (pl.hpg + 15) / 16;
-        const int hps = (pl.hpg + want - 1) / want;
-        pl.nsl = (pl.hpg + hps - 1) / hps;
+        pl.nsl = best_head_split(16, pl.G, 1, pl.hpg, pl.hpg >= 4 ? pl.hpg / 4 : 1);
     } else {
         pl.nsl = pl.hpg;
     }
@@ -206,16 +245,9 @@ static void set_segment(const Plan &pl, int k, SegParams &sp) {
     const int len = (pl.L - sp.t0 < pl.seg) ? pl.L - sp.t0 : pl.seg;
     sp.nc = len / pl.Q;
     sp.c0 = sp.t0 / pl.Q;
-    // Head ranges per group for the scan kernels: enough CTAs for about two waves of the 148 SMs,
-    // at least two heads per CTA so the shared score tile is reused.  Their outputs are per head,
-    // so this choice cannot change any result bit.
-    const int base = sp.nc * 2 * pl.G * pl.B;
-    int want = (296 + base - 1) / base;
-    const int cap = pl.hpg >= 2 ? pl.hpg / 2 : 1;
-    if (want > cap) want = cap;
-    if (want < 1) want = 1;
-    const int hps = (pl.hpg + want - 1) / want;
-    sp.nsplit_scan = (pl.hpg + hps - 1) / hps;
+    // Head ranges per group for the scan kernels (at least two heads per CTA so the shared score tile
+    // is reused).  Their outputs are per head, so this choice cannot change any result bit.
+    sp.nsplit_scan = best_head_split(sp.nc, pl.G, pl.B, pl.hpg, pl.hpg >= 2 ? pl.hpg / 2 : 1);
 }
 
 static int forward_impl(const ssd_shape_t *shape, const void *x, const float *dt, const float *A,

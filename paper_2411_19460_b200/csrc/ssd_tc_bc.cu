@@ -77,10 +77,14 @@ k_grad_bc_tc(SegParams p, const __grid_constant__ CUtensorMap tmRow,   // DC: dy
     __shared__ uint32_t tmem_base, abort_flag;
 
     constexpr bool DC = (MODE == GB_DC);
-    const int nc = p.nc, nsl = p.nsl;
-    const int rb = DC ? 1 - (int)(blockIdx.x / nc) : (int)(blockIdx.x / nc);   // long CTAs first
-    const int c = blockIdx.x % nc, b = blockIdx.z;
-    const int g = blockIdx.y / nsl, sl = blockIdx.y % nsl;
+    // 1-D grid; the first half are the long CTAs (the row block with the larger column range), so the
+    // tail of the launch is filled with short ones
+    const int nc = p.nc, nsl = p.nsl, ny = nsl * p.G;
+    const int half_grid = (int)(gridDim.x >> 1), jid = (int)blockIdx.x % half_grid;
+    const bool is_long = (int)blockIdx.x < half_grid;
+    const int rb = DC ? (is_long ? 1 : 0) : (is_long ? 0 : 1);
+    const int c = jid % nc, yid = (jid / nc) % ny, b = jid / (nc * ny);
+    const int g = yid / nsl, sl = yid % nsl;
     const int hps = (p.hpg + nsl - 1) / nsl;
     const int h_begin = g * p.hpg + sl * hps;
     const int h_end = min(g * p.hpg + p.hpg, h_begin + hps);
@@ -456,7 +460,7 @@ k_grad_bc_tc(SegParams p, const __grid_constant__ CUtensorMap tmRow,   // DC: dy
 }
 
 cudaError_t launch_grad_bc_tc(const SegParams &p, const TcMaps &m, int mode, cudaStream_t st) {
-    dim3 grid(p.nc * 2, p.nsl * p.G, p.B);
+    dim3 grid(p.nc * 2 * p.nsl * p.G * p.B);
     cudaError_t e;
     if (mode == GB_DC) {
         e = cudaFuncSetAttribute(k_grad_bc_tc<GB_DC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GB_SMEM);

@@ -82,10 +82,14 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
     __shared__ uint32_t tmem_base, abort_flag;
 
     constexpr bool FWD = (MODE == SC_FWD);
-    const int nc = p.nc;
-    const int rb = FWD ? 1 - (int)(blockIdx.x / nc) : (int)(blockIdx.x / nc);  // long CTAs first
-    const int c = blockIdx.x % nc, b = blockIdx.z;
-    const int g = blockIdx.y / nsplit, sp = blockIdx.y % nsplit;
+    // 1-D grid; the first half are the long CTAs (the row block with the larger column range), so the
+    // tail of the launch is filled with short ones
+    const int nc = p.nc, ny = nsplit * p.G;
+    const int half_grid = (int)(gridDim.x >> 1), jid = (int)blockIdx.x % half_grid;
+    const bool is_long = (int)blockIdx.x < half_grid;
+    const int rb = FWD ? (is_long ? 1 : 0) : (is_long ? 0 : 1);
+    const int c = jid % nc, yid = (jid / nc) % ny, b = jid / (nc * ny);
+    const int g = yid / nsplit, sp = yid % nsplit;
     const int hps = (p.hpg + nsplit - 1) / nsplit;
     const int h_begin = g * p.hpg + sp * hps;
     const int h_end = min(g * p.hpg + p.hpg, h_begin + hps);
@@ -420,7 +424,7 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
 
 cudaError_t launch_scan_tc(const SegParams &p, const TcMaps &m, int mode, cudaStream_t st) {
     const int nsplit = p.nsplit_scan;
-    dim3 grid(p.nc * 2, nsplit * p.G, p.B);
+    dim3 grid(p.nc * 2 * nsplit * p.G * p.B);
     cudaError_t e;
     if (mode == SC_FWD) {
         e = cudaFuncSetAttribute(k_scan_tc<SC_FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SC_SMEM);
