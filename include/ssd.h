@@ -34,7 +34,7 @@
  *    CUDA code).
  *  - Deterministic: the same inputs give the same bits run to run, and the gradients of
  *    ssd_bwd_segmented do not depend on `seg` (seg == L is the unsegmented backward).
- *  - Gradient outputs are overwritten, not accumulated into.
+ *  - Gradient outputs are overwritten, not accumulated into (dA, dD: unless SSD_FLAG_ACCUM_PARAM_GRADS).
  */
 #ifndef SSD_H_
 #define SSD_H_
@@ -52,7 +52,9 @@ enum { SSD_DTYPE_F32 = 0, SSD_DTYPE_BF16 = 1 };
 
 /* shape.flags */
 enum {
-    SSD_FLAG_FORCE_SIMT = 1 /* bf16 I/O: use the CUDA-core kernels instead of the tensor-core ones */
+    SSD_FLAG_FORCE_SIMT = 1,       /* bf16 I/O: use the CUDA-core kernels instead of the tensor-core ones */
+    SSD_FLAG_ACCUM_PARAM_GRADS = 2 /* ssd_bwd_segmented: dA and dD are added to, not overwritten (a driver that
+                                      back-propagates one grid cell at a time sums them over the cells) */
 };
 
 /* `op` of ssd_workspace_bytes */
@@ -152,6 +154,21 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
                       const void *dy, const float *dh_final,
                       void *dx, float *ddt, float *dA, void *dB, void *dC, float *dD,
                       float *dh0, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Layer-axis glue for a stack of SSD layers (Algorithms 1 and 2 keep only each layer's input along the
+ * layer axis; the benchmark's stacked configuration feeds layer j+1 with x_{j+1} = W (y_j + x_j), W a fixed
+ * P x P row-major fp32 matrix applied per (batch, step, head)).  Tensors are [B, L, H, P] in the I/O dtype
+ * with batch stride x_bstride; only B, L, H, P, dtype and x_bstride of `shape` are read (P must be 64).
+ *   ssd_glue_fwd      : x_next = W (y + x)
+ *   ssd_glue_bwd      : dz = W^T g_next     (dz is the dy of the layer's SSD backward)
+ *   ssd_glue_residual : dx += dz            (the skip branch; call after ssd_bwd_segmented wrote dx)
+ * Device pointers, enqueued on `stream`, no scratch.  Returns SSD_OK or SSD_EINVAL / SSD_EUNSUPPORTED /
+ * SSD_EALIGN / SSD_ECUDA.
+ */
+int ssd_glue_fwd(const ssd_shape_t *shape, const void *x, const void *y, const float *W, void *x_next, void *stream);
+int ssd_glue_bwd(const ssd_shape_t *shape, const void *g_next, const float *W, void *dz, void *stream);
+int ssd_glue_residual(const ssd_shape_t *shape, void *dx, const void *dz, void *stream);
 
 /*
  * Reads the status word at the start of `ws` (device memory) with a blocking copy: call it after

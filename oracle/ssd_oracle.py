@@ -83,3 +83,15 @@ def ssd_bwd(x, dt, A, Bm, Cm, D, h0, dy, dh_final=None, blk=256):
     if rc != 0:
         raise RuntimeError("ssd_oracle_bwd failed: %d" % rc)
     return out
+
+
+def glue_fwd(x, y, W):
+    """Hand-over between two stacked layers: x_next[b,t,h,:] = W (y + x)[b,t,h,:] (fp64)."""
+    x, y, W = map(_f64, (x, y, W))
+    return np.einsum("ij,bthj->bthi", W, y + x)
+
+
+def glue_bwd(g_next, W):
+    """dz = W^T g_next: gradient of (y + x) given the gradient of x_next (fp64)."""
+    g_next, W = map(_f64, (g_next, W))
+    return np.einsum("ij,bthi->bthj", W, g_next)

@@ -24,7 +24,7 @@ static size_t g_prof_used = 0;
 
 static const char *const kKindNames[KIND_COUNT] = {
     "chunk_cumsum", "chunk_state", "state_pass_fwd", "chunk_scan_fwd", "dstate_contrib",
-    "state_pass_bwd", "bwd_dx", "bwd_dC", "bwd_dB", "bwd_finish", "reduce_dBdC", "final_dAdD"};
+    "state_pass_bwd", "bwd_dx", "bwd_dC", "bwd_dB", "bwd_finish", "reduce_dBdC", "final_dAdD", "glue"};
 
 static ProfEvent *prof_begin(int kind, cudaStream_t st) {
     if (!g_prof_on) return nullptr;
@@ -429,7 +429,50 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
         SSD_LAUNCH(KIND_BWD_FINISH, launch_bwd_finish(sp, st));
         SSD_LAUNCH(KIND_REDUCE_DBDC, launch_reduce_dbdc(sp, pl.dtype, st));
     }
-    SSD_LAUNCH(KIND_FINAL, launch_final_dAdD(sp, dA, dD, st));
+    SSD_LAUNCH(KIND_FINAL, launch_final_dAdD(sp, dA, dD, (shape->flags & SSD_FLAG_ACCUM_PARAM_GRADS) != 0, st));
+    return SSD_OK;
+}
+
+static int glue_check(const ssd_shape_t *s, const void *a, const void *b, size_t &esz, long long &bs) {
+    if (!s || !a || !b) return SSD_EINVAL;
+    if (s->B <= 0 || s->L <= 0 || s->H <= 0) return SSD_EINVAL;
+    if (s->P != 64) return SSD_EUNSUPPORTED;
+    if (s->dtype != SSD_DTYPE_F32 && s->dtype != SSD_DTYPE_BF16) return SSD_EUNSUPPORTED;
+    esz = s->dtype == SSD_DTYPE_BF16 ? 2 : 4;
+    bs = s->x_bstride ? s->x_bstride : (long long)s->L * s->H * s->P;
+    if (bs < (long long)s->L * s->H * s->P) return SSD_EINVAL;
+    if (misaligned(a) || misaligned(b) || ((size_t)bs * esz) % 16) return SSD_EALIGN;
+    return SSD_OK;
+}
+
+int ssd_glue_fwd(const ssd_shape_t *shape, const void *x, const void *y, const float *W, void *x_next, void *stream) {
+    size_t esz; long long bs;
+    int rc = glue_check(shape, x, y, esz, bs);
+    if (rc) return rc;
+    if (!W || !x_next) return SSD_EINVAL;
+    if (misaligned(W) || misaligned(x_next)) return SSD_EALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    SSD_LAUNCH(KIND_GLUE, launch_glue(shape->dtype, false, x, y, W, x_next, (long long)shape->L * shape->H, bs, shape->B, st));
+    return SSD_OK;
+}
+
+int ssd_glue_bwd(const ssd_shape_t *shape, const void *g_next, const float *W, void *dz, void *stream) {
+    size_t esz; long long bs;
+    int rc = glue_check(shape, g_next, dz, esz, bs);
+    if (rc) return rc;
+    if (!W) return SSD_EINVAL;
+    if (misaligned(W)) return SSD_EALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    SSD_LAUNCH(KIND_GLUE, launch_glue(shape->dtype, true, g_next, nullptr, W, dz, (long long)shape->L * shape->H, bs, shape->B, st));
+    return SSD_OK;
+}
+
+int ssd_glue_residual(const ssd_shape_t *shape, void *dx, const void *dz, void *stream) {
+    size_t esz; long long bs;
+    int rc = glue_check(shape, dx, dz, esz, bs);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    SSD_LAUNCH(KIND_GLUE, launch_residual(shape->dtype, dx, dz, (long long)shape->L * shape->H * shape->P, bs, shape->B, st));
     return SSD_OK;
 }
 

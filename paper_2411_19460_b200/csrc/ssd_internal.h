@@ -67,7 +67,12 @@ cudaError_t launch_state_pass_bwd(const SegParams &p, const float *init, float *
 cudaError_t launch_masked_product_simt(const SegParams &p, int dtype, int mode, cudaStream_t st);
 cudaError_t launch_bwd_finish(const SegParams &p, cudaStream_t st);
 cudaError_t launch_reduce_dbdc(const SegParams &p, int dtype, cudaStream_t st);
-cudaError_t launch_final_dAdD(const SegParams &p, float *dA, float *dD, cudaStream_t st);
+cudaError_t launch_final_dAdD(const SegParams &p, float *dA, float *dD, bool accumulate, cudaStream_t st);
+// ssd_glue.cu : layer-axis glue of a layer stack
+cudaError_t launch_glue(int dtype, bool transpose, const void *a, const void *b, const float *W, void *out,
+                        long long rows_per_batch, long long bstride, int B, cudaStream_t st);
+cudaError_t launch_residual(int dtype, void *dst, const void *src, long long n_per_batch, long long bstride, int B,
+                            cudaStream_t st);
 
 // ssd_tc.cu : tensor-core (tcgen05 / TMEM / TMA) kernels, bf16 I/O
 struct TcMaps {
@@ -90,7 +95,7 @@ enum { STATE_MODE_FWD = 0, STATE_MODE_DSTATE = 1 };
 enum {
     KIND_CUMSUM = 0, KIND_CHUNK_STATE, KIND_STATE_PASS_FWD, KIND_SCAN_FWD, KIND_DSTATE,
     KIND_STATE_PASS_BWD, KIND_BWD_DX, KIND_BWD_DC, KIND_BWD_DB, KIND_BWD_FINISH, KIND_REDUCE_DBDC,
-    KIND_FINAL, KIND_COUNT
+    KIND_FINAL, KIND_GLUE, KIND_COUNT
 };
 enum { MP_FWD = 0, MP_BWD_DX = 1, MP_DC = 2, MP_DB = 3 };
 

@@ -698,7 +698,7 @@ cudaError_t launch_reduce_dbdc(const SegParams &p, int dtype, cudaStream_t st) {
 
 // ------------------------------------------------------------------ a13 tail: dA, dD over (batch, chunks)
 // One warp per head; lanes stride over the per-chunk partials in fp64, then a fixed shuffle tree.
-__global__ void __launch_bounds__(32) k_final_dAdD(SegParams p, float *dA, float *dD) {
+__global__ void __launch_bounds__(32) k_final_dAdD(SegParams p, float *dA, float *dD, int accumulate) {
     const int h = blockIdx.x, lane = threadIdx.x;
     const int nrt = p.ndd;
     double sA = 0.0, sD = 0.0;
@@ -715,13 +715,13 @@ __global__ void __launch_bounds__(32) k_final_dAdD(SegParams p, float *dA, float
         sD += __shfl_xor_sync(0xffffffffu, sD, off);
     }
     if (lane == 0) {
-        dA[h] = (float)sA;
-        dD[h] = (float)sD;
+        dA[h] = accumulate ? dA[h] + (float)sA : (float)sA;
+        dD[h] = accumulate ? dD[h] + (float)sD : (float)sD;
     }
 }
 
-cudaError_t launch_final_dAdD(const SegParams &p, float *dA, float *dD, cudaStream_t st) {
-    k_final_dAdD<<<p.H, 32, 0, st>>>(p, dA, dD);
+cudaError_t launch_final_dAdD(const SegParams &p, float *dA, float *dD, bool accumulate, cudaStream_t st) {
+    k_final_dAdD<<<p.H, 32, 0, st>>>(p, dA, dD, accumulate ? 1 : 0);
     return cudaGetLastError();
 }
 

@@ -116,3 +116,24 @@ def to_f64_numpy(inp, heads=None, groups=None):
         dh_final=None if inp["dh_final"] is None else cv(inp["dh_final"].index_select(1, hi)),
     )
     return {k: (None if v is None else np.ascontiguousarray(v)) for k, v in out.items()}
+
+
+def make_stack_params(cfg: SSDConfig, device="cpu", scale=None):
+    """Per-layer A, D (seed + layer) and the fixed mixing matrix W of the stacked configuration.
+
+    W = scale * Q0 with Q0 the orthogonal factor of a seeded Gaussian P x P matrix, rounded to bf16
+    so that both sides use the same numbers; `scale` defaults to 0.5, which keeps the RMS of the layer
+    inputs of order one over 64 layers for D ~ N(0,1) (y + x has about (1 + D_h^2)^(1/2) times the RMS
+    of x).  B, C and dt are shared by all layers (those of make_inputs)."""
+    dev = torch.device(device)
+    g = torch.Generator(device="cpu")
+    g.manual_seed(cfg.seed + 7919)
+    q0, _ = torch.linalg.qr(torch.randn(cfg.P, cfg.P, generator=g, dtype=torch.float64))
+    W = ((0.5 if scale is None else scale) * q0).to(torch.bfloat16).to(torch.float32).to(dev)
+    A, D = [], []
+    for layer in range(cfg.layers):
+        gl = torch.Generator(device="cpu")
+        gl.manual_seed(cfg.seed + 1 + layer)
+        A.append((-torch.exp(torch.rand(cfg.H, generator=gl) * math.log(cfg.a_max))).to(dev))
+        D.append(torch.randn(cfg.H, generator=gl).to(dev))
+    return dict(W=W.contiguous(), A=A, D=D)

@@ -12,6 +12,7 @@ LIB_PATH = os.path.join(_HERE, "lib", "libssd.so")
 
 SSD_DTYPE_F32, SSD_DTYPE_BF16 = 0, 1
 SSD_FLAG_FORCE_SIMT = 1
+SSD_FLAG_ACCUM_PARAM_GRADS = 2
 SSD_OP_FWD, SSD_OP_FWD_SEG, SSD_OP_BWD_SEG = 0, 1, 2
 SSD_OK, SSD_EINVAL, SSD_EUNSUPPORTED, SSD_EALIGN = 0, -1, -2, -3
 SSD_EWORKSPACE, SSD_EDEVICE, SSD_ECUDA, SSD_ETIMEOUT = -4, -5, -6, -7
@@ -21,7 +22,8 @@ SSD_STATIC_WS_BYTES = 8 * 1024 * 1024
 EXPORTS = ["ssd_workspace_bytes", "ssd_boundary_bytes", "ssd_fwd", "ssd_fwd_segmented",
            "ssd_bwd_segmented", "ssd_poll_status", "ssd_strerror", "ssd_version",
            "ssd_last_cuda_error", "ssd_launch_count", "ssd_kernel_kinds", "ssd_kernel_name",
-           "ssd_profile", "ssd_profile_read", "ssd_fwd_static_ws"]
+           "ssd_profile", "ssd_profile_read", "ssd_fwd_static_ws", "ssd_glue_fwd", "ssd_glue_bwd",
+           "ssd_glue_residual"]
 
 
 class SSDShape(ctypes.Structure):
@@ -64,6 +66,12 @@ def lib():
         L.ssd_bwd_segmented.restype = ctypes.c_int
         L.ssd_bwd_segmented.argtypes = [sp, vp, fp, fp, vp, vp, fp, fp, vp, fp,
                                         vp, fp, fp, vp, vp, fp, fp, vp, ctypes.c_size_t, vp]
+        L.ssd_glue_fwd.restype = ctypes.c_int
+        L.ssd_glue_fwd.argtypes = [sp, vp, vp, fp, vp, vp]
+        L.ssd_glue_bwd.restype = ctypes.c_int
+        L.ssd_glue_bwd.argtypes = [sp, vp, fp, vp, vp]
+        L.ssd_glue_residual.restype = ctypes.c_int
+        L.ssd_glue_residual.argtypes = [sp, vp, vp, vp]
         L.ssd_poll_status.restype = ctypes.c_int
         L.ssd_poll_status.argtypes = [vp]
         L.ssd_strerror.restype = ctypes.c_char_p
@@ -233,3 +241,40 @@ def ssd_bwd_segmented(x, dt, A, Bm, Cm, D, boundary, dy, dh_final=None, *, chunk
     if rc != SSD_OK:
         raise SSDError(rc, "ssd_bwd_segmented")
     return out
+
+
+def _glue_shape(t):
+    B, L, H, P = t.shape
+    if t.dtype == torch.bfloat16:
+        dt = SSD_DTYPE_BF16
+    elif t.dtype == torch.float32:
+        dt = SSD_DTYPE_F32
+    else:
+        raise TypeError("tensor must be float32 or bfloat16")
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("tensor must be a contiguous CUDA tensor")
+    return SSDShape(B, L, H, P, 1, 1, 64, 0, dt, 0, 0, 0, 0)
+
+
+def ssd_glue_fwd(x, y, W, x_next, stream=None):
+    """x_next = W (y + x) per (batch, step, head): the hand-over between two stacked layers."""
+    rc = lib().ssd_glue_fwd(ctypes.byref(_glue_shape(x)), _ptr(x), _ptr(y), _ptr(W), _ptr(x_next), _stream(stream))
+    if rc != SSD_OK:
+        raise SSDError(rc, "ssd_glue_fwd")
+    return x_next
+
+
+def ssd_glue_bwd(g_next, W, dz, stream=None):
+    """dz = W^T g_next: the gradient of the layer's output (its dy) and of the skip branch."""
+    rc = lib().ssd_glue_bwd(ctypes.byref(_glue_shape(g_next)), _ptr(g_next), _ptr(W), _ptr(dz), _stream(stream))
+    if rc != SSD_OK:
+        raise SSDError(rc, "ssd_glue_bwd")
+    return dz
+
+
+def ssd_glue_residual(dx, dz, stream=None):
+    """dx += dz (the skip branch of the layer's input gradient)."""
+    rc = lib().ssd_glue_residual(ctypes.byref(_glue_shape(dx)), _ptr(dx), _ptr(dz), _stream(stream))
+    if rc != SSD_OK:
+        raise SSDError(rc, "ssd_glue_residual")
+    return dx

@@ -1,0 +1,87 @@
+"""Layer stack under MA-GC (Algorithms 1 and 2, layer interval 1): the glue of the oracle is pinned on
+the CPU; the GPU driver is checked layer by layer, teacher-forced (the oracle's layer j is fed the
+layer input, and in the backward the output gradient, that the GPU path itself stored), because
+bf16 rounding compounds over the layers."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ssd_oracle as orc
+from paper_2411_19460_b200.inputs import CONFIGS, make_inputs, make_stack_params
+
+
+def test_oracle_glue_is_a_matrix_product_and_its_adjoint():
+    rng = np.random.default_rng(0)
+    W = rng.standard_normal((5, 5))
+    x = rng.standard_normal((2, 3, 4, 5))
+    y = rng.standard_normal((2, 3, 4, 5))
+    g = rng.standard_normal((2, 3, 4, 5))
+    out = orc.glue_fwd(x, y, W)
+    for b in range(2):
+        for t in range(3):
+            for h in range(4):
+                ref = [sum(W[i, j] * (x[b, t, h, j] + y[b, t, h, j]) for j in range(5)) for i in range(5)]
+                assert np.allclose(out[b, t, h], ref, rtol=0, atol=1e-13)
+    dz = orc.glue_bwd(g, W)
+    assert abs(np.sum(out * g) - np.sum((x + y) * dz)) < 1e-10      # <W z, g> = <z, W^T g>
+
+
+def test_stack_parameters_are_seeded_and_bf16_representable():
+    cfg = CONFIGS[3].scaled(layers=3)
+    a, b = make_stack_params(cfg), make_stack_params(cfg)
+    assert torch.equal(a["W"], b["W"]) and all(torch.equal(x, y) for x, y in zip(a["A"], b["A"]))
+    assert torch.equal(a["W"], a["W"].to(torch.bfloat16).to(torch.float32))
+    q = (a["W"].double() / 0.5)
+    assert torch.allclose(q @ q.T, torch.eye(cfg.P, dtype=torch.float64), atol=2e-2)
+    assert not torch.equal(a["A"][0], a["A"][1])
+
+
+@pytest.mark.gpu
+def test_stack_matches_oracle_layer_by_layer():
+    from paper_2411_19460_b200.stack import LayerStack
+    from tests.parity_util import TOL, relerr
+
+    cfg = CONFIGS[3].scaled(L=1024, H=4, seg=512, layers=3, dh_std=0.0)
+    tol = TOL[cfg.dtype]
+    inp = make_inputs(cfg, "cuda")
+    sp = make_stack_params(cfg, "cuda")
+    st = LayerStack(inp["x"], inp["dt"], inp["Bm"], inp["Cm"], sp["A"], sp["D"], sp["W"], chunk=cfg.chunk, seg=cfg.seg)
+    h0 = [torch.randn(cfg.B, cfg.H, cfg.P, cfg.N, device="cuda") * 0.1 for _ in range(cfg.layers)]
+    for j in range(cfg.layers):
+        st.set_h0(j, h0[j])
+    st.forward()
+    torch.cuda.synchronize()
+
+    f64 = lambda t: t.detach().double().cpu().numpy()
+    dt, Bm, Cm, W = f64(inp["dt"]), f64(inp["Bm"]), f64(inp["Cm"]), f64(sp["W"])
+    for j in range(cfg.layers):
+        xj = f64(st.x[j])
+        y, hf, bd = orc.ssd_fwd(xj, dt, f64(sp["A"][j]), Bm, Cm, f64(sp["D"][j]), f64(h0[j]), seg=cfg.seg)
+        assert relerr(st.x[j + 1], orc.glue_fwd(xj, y, W)) <= tol, j
+        assert relerr(st.bnd[j, st.nseg], hf) <= tol, j
+        assert relerr(st.bnd[j, 1], bd[:, 1]) <= tol, j
+
+    # backward, collecting the per-cell outputs into per-layer tensors
+    keep = {k: [torch.zeros_like(inp[src]) for _ in range(cfg.layers)]
+            for k, src in (("dx", "x"), ("dy", "x"), ("ddt", "dt"), ("dB", "Bm"), ("dC", "Cm"))}
+
+    def on_cell(j, k, cell):
+        sl = slice(k * cfg.seg, (k + 1) * cfg.seg)
+        for name in keep:
+            keep[name][j][:, sl].copy_(cell[name])
+
+    g_top = inp["dy"]
+    out = st.backward(g_top, on_cell=on_cell)
+    torch.cuda.synchronize()
+    for j in range(cfg.layers - 1, -1, -1):
+        g_next = f64(g_top) if j == cfg.layers - 1 else f64(keep["dx"][j + 1])
+        dz = orc.glue_bwd(g_next, W)
+        assert relerr(keep["dy"][j], dz) <= tol, j
+        ref = orc.ssd_bwd(f64(st.x[j]), dt, f64(sp["A"][j]), Bm, Cm, f64(sp["D"][j]), f64(h0[j]), f64(keep["dy"][j]), None)
+        errs = dict(dx=relerr(keep["dx"][j], ref["dx"] + f64(keep["dy"][j])), ddt=relerr(keep["ddt"][j], ref["ddt"]),
+                    dB=relerr(keep["dB"][j], ref["dB"]), dC=relerr(keep["dC"][j], ref["dC"]),
+                    dA=relerr(out["dA"][j], ref["dA"]), dD=relerr(out["dD"][j], ref["dD"]),
+                    dh0=relerr(out["dh0"][j], ref["dh0"]))
+        bad = {k: v for k, v in errs.items() if not (v <= tol)}
+        assert not bad, (j, bad, errs)
+    assert torch.equal(out["dx0"], keep["dx"][0])
