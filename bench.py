@@ -180,7 +180,7 @@ def run_ours(args):
     rank, world = rep.rank, rep.world
     cfg = CONFIGS[args.config]
     if cfg.layers != 1:
-        raise SystemExit("config %d is the layer-stack sweep; it is not a bench line" % args.config)
+        return run_stack(args, rep, dev)
     seg = args.seg or cfg.seg
     flags = libssd.SSD_FLAG_FORCE_SIMT if args.simt else 0
     inp = make_inputs(cfg, dev, seed=cfg.seed + rank)
@@ -334,6 +334,72 @@ def run_ours(args):
     rep.close()
 
 
+# ----------------------------------------------------------------------------- the stacked configuration
+def run_stack(args, rep, dev):
+    """Config 3: 64 stacked layers under MA-GC (layer inputs + segment-boundary states kept), one step =
+    Algorithm 1 forward + Algorithm 2 backward of the whole stack.  The literal L = 262144 needs 175 GB of
+    layer inputs alone, so the sequence is run at --stack-len (default 131072) and the figure says so."""
+    from paper_2411_19460_b200 import libssd
+    from paper_2411_19460_b200.inputs import make_stack_params
+    from paper_2411_19460_b200.stack import LayerStack
+
+    base = CONFIGS[args.config]
+    L = args.stack_len or 131072
+    cfg = base.scaled(L=L, seg=args.seg or base.seg, layers=args.layers or base.layers)
+    inp = make_inputs(cfg, dev, seed=cfg.seed + rep.rank)
+    sp = make_stack_params(cfg, dev)
+    st = LayerStack(inp["x"], inp["dt"], inp["Bm"], inp["Cm"], sp["A"], sp["D"], sp["W"], chunk=cfg.chunk, seg=cfg.seg)
+    out = dict(dx0=torch.empty_like(inp["x"]), dA=torch.zeros(cfg.layers, cfg.H, device=dev),
+               dD=torch.zeros(cfg.layers, cfg.H, device=dev))
+    stream = torch.cuda.current_stream()
+
+    def step():
+        out["dA"].zero_()
+        out["dD"].zero_()
+        st.forward()
+        st.backward(inp["dy"], out=out)
+
+    for _ in range(max(args.warmup, 1)):
+        step()
+    rep.barrier()
+    torch.cuda.reset_peak_memory_stats(dev)
+    sampler = ClockSampler(dev) if rep.rank == 0 else None
+    n0 = libssd.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rep.barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    rep.barrier()
+    ms = rep.max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    launches = libssd.launch_count() - n0
+    clocks = sampler.stop() if sampler else None
+    peak_mem = torch.cuda.max_memory_allocated(dev)
+    if rep.rank != 0:
+        rep.close()
+        return
+    peaks = load_peaks()
+    fl, by = step_model(cfg, cfg.seg)
+    glue_bytes = 2 * (3 + 3) * cfg.H * cfg.P              # forward x, y -> x_next; backward g -> dz, dx += dz
+    t_roof = cfg.layers * cfg.L * max(fl / (peaks["bf16_tflops"] * 1e12), (by + glue_bytes) / (peaks["hbm_gbs"] * 1e9))
+    value = rep.world * cfg.L / (ms * 1e-3)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": rep.world, "steps": args.steps,
+        "warmup": max(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "impl": "ours",
+        "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "L_in_definition": base.L, "layers": cfg.layers,
+                   "H": cfg.H, "P": cfg.P, "N": cfg.N, "G": cfg.G, "chunk": cfg.chunk, "seg": cfg.seg,
+                   "layer_tokens_per_s": value * cfg.layers, "l2": "inputs larger than L2",
+                   "parallelism": "replicas" if rep.world > 1 else "single"},
+        "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+        "step_roofline": {"roofline_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms},
+        "memory": dict(peak_allocated_bytes=int(peak_mem), **st.checkpoint_bytes()),
+    }
+    print(json.dumps(line))
+    rep.close()
+
+
 # ----------------------------------------------------------------------------- the CPU oracle legs
 def _oracle_sample(cfg, inp, sample_tokens):
     """fp64 host copies of the first `sample_tokens` tokens (all heads) of the workload."""
@@ -400,6 +466,8 @@ def main():
                     "Mamba-2-2.7B-dim layer, L=131072)")
     ap.add_argument("--seg", type=int, default=0, help="override the segment length")
     ap.add_argument("--simt", action="store_true", help="force the CUDA-core kernels")
+    ap.add_argument("--stack-len", type=int, default=0, help="config 3: sequence length (default 131072)")
+    ap.add_argument("--layers", type=int, default=0, help="config 3: number of layers (default 64)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-tokens", type=int, default=32768, help="tokens in the cpu_baseline sample")

@@ -40,6 +40,13 @@ class LayerStack:
         self.ws_f = libssd.alloc_workspace(cell, libssd.SSD_OP_FWD, dev)
         self.ws_b = libssd.alloc_workspace(cell, libssd.SSD_OP_BWD_SEG, dev)
         self.dh = torch.zeros(self.layers, 2, B, H, P, N, dtype=torch.float32, device=dev)
+        # the slices every cell call takes (views; made once, the loops below are launch-bound otherwise)
+        ns = self.nseg
+        self._xs = [[self._sl(t, k) for k in range(ns)] for t in self.x]
+        self._dts = [self._sl(dt, k) for k in range(ns)]
+        self._Bs = [self._sl(Bm, k) for k in range(ns)]
+        self._Cs = [self._sl(Cm, k) for k in range(ns)]
+        self._bin = [[self.bnd[j, k:k + 1].reshape(B, 1, H, P, N) for k in range(ns)] for j in range(self.layers)]
 
     def set_h0(self, layer, h0):
         self.bnd[layer, 0].copy_(h0)
@@ -51,11 +58,11 @@ class LayerStack:
         """Algorithm 1.  Returns the stack output x[layers] (a kept buffer)."""
         for k in range(self.nseg):
             for j in range(self.layers):
-                xs = self._sl(self.x[j], k)
-                libssd.ssd_fwd(xs, self._sl(self.dt, k), self.A[j], self._sl(self.Bm, k), self._sl(self.Cm, k),
+                xs = self._xs[j][k]
+                libssd.ssd_fwd(xs, self._dts[k], self.A[j], self._Bs[k], self._Cs[k],
                                self.D[j], self.bnd[j, k], chunk=self.chunk, seg=self.seg, flags=self.flags,
                                y=self.y, h_final=self.bnd[j, k + 1], ws=self.ws_f)
-                libssd.ssd_glue_fwd(xs, self.y, self.W, self._sl(self.x[j + 1], k))
+                libssd.ssd_glue_fwd(xs, self.y, self.W, self._xs[j + 1][k])
         return self.x[self.layers]
 
     def backward(self, g_top, dh_final=None, out=None, on_cell=None):
@@ -83,13 +90,12 @@ class LayerStack:
             cur = (self.nseg - 1 - k) & 1              # dh[j, cur] enters from the right, dh[j, 1-cur] leaves
             g_in = self._sl(g_top, k)
             for j in range(self.layers - 1, -1, -1):
-                xs = self._sl(self.x[j], k)
+                xs = self._xs[j][k]
                 libssd.ssd_glue_bwd(g_in, self.W, self.dz)
                 dx = self._sl(out["dx0"], k) if j == 0 else self.g[j & 1]
                 cell = dict(dx=dx, ddt=ddt, dA=out["dA"][j], dB=dB, dC=dC, dD=out["dD"][j], dh0=self.dh[j, 1 - cur])
-                libssd.ssd_bwd_segmented(xs, self._sl(self.dt, k), self.A[j], self._sl(self.Bm, k),
-                                         self._sl(self.Cm, k), self.D[j], self.bnd[j, k:k + 1].reshape(
-                                             self.B, 1, H, self.P, self.N), self.dz, self.dh[j, cur],
+                libssd.ssd_bwd_segmented(xs, self._dts[k], self.A[j], self._Bs[k],
+                                         self._Cs[k], self.D[j], self._bin[j][k], self.dz, self.dh[j, cur],
                                          chunk=self.chunk, seg=self.seg, flags=flags, out=cell, ws=self.ws_b)
                 libssd.ssd_glue_residual(dx, self.dz)
                 if on_cell is not None:
