@@ -92,6 +92,11 @@ def load_peaks():
 # to the timed workload by tokens x heads per launch (the traffic of these kernels grows in proportion).
 NCU_TRAFFIC_CFG1 = {
     # kernel kind: (bytes per launch, source file, sha256 of that file at capture time)
+    "bwd_dB": (17.22e6, "ssd_tc_bc.cu", "800395a98e29fa540b7f78cc9bd182ba6d9e044247f9fdbe3071ce2aa2e6c65e"),
+    "bwd_dC": (17.22e6, "ssd_tc_bc.cu", "800395a98e29fa540b7f78cc9bd182ba6d9e044247f9fdbe3071ce2aa2e6c65e"),
+    "bwd_dx": (17.22e6, "ssd_tc_scan.cu", "8c6e27020dadacba65067e5da6ee0d4454197329a58427ad979106ad1b61fb80"),
+    "chunk_state": (7.24e6, "ssd_tc.cu", "08ba9e297121e0bc3fe4bd835ce929e0578a9936620712ece7868ec0a7d6f316"),
+    "dstate_contrib": (7.24e6, "ssd_tc.cu", "08ba9e297121e0bc3fe4bd835ce929e0578a9936620712ece7868ec0a7d6f316"),
 }
 NCU_CFG1_UNITS = 2048 * 24
 
