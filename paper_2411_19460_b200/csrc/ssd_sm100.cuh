@@ -51,21 +51,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 // given up, later waits only poll briefly (so copies still in flight get a last chance to land)
 // and the kernel runs to its normal end, frees its TMEM and returns; `status` is the global word
 // the host reads back.
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
-constexpr unsigned long long kWaitAbortedNs = 2000000ull;   // 2 ms once aborted
+constexpr long long kWaitLimitClk = 4000000000ll;   // about 2 s at 2 GHz
+constexpr long long kWaitAbortedClk = 4000000ll;     // about 2 ms once aborted
 
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
                                           unsigned int *status) {
     if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long start = globaltimer_ns();
-    const unsigned long long limit = (*abort_flag) ? kWaitAbortedNs : kWaitLimitNs;
+    // Not complete yet: poll with a short sleep in between, so that the waiting warps of a CTA do not
+    // flood the shared-memory pipe (every poll is a shared-memory access) that the MMAs read from.
+    const long long start = clock64();
+    const long long limit = (*abort_flag) ? kWaitAbortedClk : kWaitLimitClk;
     uint32_t it = 0;
     while (true) {
+        __nanosleep(20);
         if (mbar_try_wait(bar, parity)) return true;
-        if ((++it & 63u) == 0) {
-            if (globaltimer_ns() - start > limit) break;
-            __nanosleep(32);
-        }
+        if ((++it & 255u) == 0 && clock64() - start > limit) break;
     }
     *abort_flag = 1u;
     atomicExch(status, 1u);
