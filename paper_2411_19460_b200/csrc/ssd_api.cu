@@ -279,9 +279,12 @@ static int forward_impl(const ssd_shape_t *shape, const void *x, const float *dt
     const long long PN = (long long)pl.P * pl.N;
     for (int k = 0; k < pl.nseg; ++k) {
         set_segment(pl, k, sp);
-        SSD_LAUNCH(KIND_CUMSUM, launch_chunk_cumsum(sp, st));
-        if (pl.use_tc) SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_tc(sp, maps, STATE_MODE_FWD, st));
-        else SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
+        if (pl.use_tc) {   // the tensor-core chunk-state kernel computes the chunk cumsum itself
+            SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_tc(sp, maps, STATE_MODE_FWD, st));
+        } else {
+            SSD_LAUNCH(KIND_CUMSUM, launch_chunk_cumsum(sp, st));
+            SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
+        }
         const float *init = (k == 0) ? h0 : sp.hcarry;
         float *bnd = boundary ? boundary + (size_t)k * pl.H * PN : nullptr;
         SSD_LAUNCH(KIND_STATE_PASS_FWD, launch_state_pass_fwd(sp, init, (long long)pl.H * PN, bnd, (long long)pl.nseg * pl.H * PN,
@@ -406,9 +409,12 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
     for (int k = pl.nseg - 1; k >= 0; --k) {
         set_segment(pl, k, sp);
         // Recompute_Forward: chunk-entry states of segment k from the stored boundary state
-        SSD_LAUNCH(KIND_CUMSUM, launch_chunk_cumsum(sp, st));
-        if (pl.use_tc) SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_tc(sp, maps, STATE_MODE_FWD, st));
-        else SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
+        if (pl.use_tc) {   // the tensor-core chunk-state kernel computes the chunk cumsum itself
+            SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_tc(sp, maps, STATE_MODE_FWD, st));
+        } else {
+            SSD_LAUNCH(KIND_CUMSUM, launch_chunk_cumsum(sp, st));
+            SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
+        }
         SSD_LAUNCH(KIND_STATE_PASS_FWD, launch_state_pass_fwd(sp, boundary + (size_t)k * pl.H * PN, (long long)pl.nseg * pl.H * PN,
                                       nullptr, 0, nullptr, pl.use_tc, st));
         // Backward through the segment; dh enters from the right, leaves to the left

@@ -80,7 +80,8 @@ bool tc_make_maps(const SegParams &p, TcMaps &m) {
 // ONE 64 KB stage (half a chunk) and two to three CTAs share an SM: one CTA's load overlaps the
 // others' scaling, MMAs and epilogue.
 //
-// Mode DSTATE also produces, per head, rho2_t = e^{cs_t} dy_t . (H_in C_t): the inter-chunk part of
+// Mode FWD also computes the chunk cumsum of dt*A (a1) for its two heads and leaves cs / dtT for the
+// later kernels of the segment.  Mode DSTATE also produces, per head, rho2_t = e^{cs_t} dy_t . (H_in C_t): the inter-chunk part of
 // C_t . dC_t that the decay gradient needs.  The C tile is already in shared memory (as rows of
 // time it is a K-major A operand), so it is one more product C (128 x N) * H_in^T (N x P) per head
 // and half into spare TMEM columns, and a row dot with the already scaled dy tile.
@@ -128,18 +129,51 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
     }
     const uint32_t ncol_tmem = dstate ? 256u : 128u;   // E or S: 128 columns; Yoff of two heads: 128 more
     if (warp == 0) tmem_alloc(&tmem_base, ncol_tmem);
-    // per-row weights of both heads
-    for (int i = tid; i < 512; i += CS_THREADS) {
-        const int hh = i >> 8, t = i & 255;
-        const float *csb = p.cs + ((((size_t)b * p.H + h0 + hh) * p.ncs + c) << 8);
-        float w;
-        if (!dstate) {
-            const float *dtb = p.dtT + ((((size_t)b * p.H + h0 + hh) * p.ncs + c) << 8);
-            w = __expf(fminf(csb[255] - csb[t], 0.f)) * dtb[t];
-        } else {
-            w = __expf(csb[t]);
+    if (!dstate) {
+        // a1 fused in: the chunk's cumulative sums of dt*A for the two heads (warp hh scans head hh: a
+        // lane owns 8 consecutive steps, lane totals meet in a warp-shuffle scan), kept for every later
+        // kernel of the segment in cs / dtT, and turned into the per-row weights right here.
+        if (warp < 2) {
+            const int hh = warp, lane = tid & 31, h = h0 + hh;
+            const float Ah = __ldg(p.A + h);
+            const float *dtp = p.dt + (size_t)b * p.dt_bs + (size_t)(tok0 + lane * 8) * p.H + h;
+            float d[8], a[8], run = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) d[j] = __ldg(dtp + (size_t)j * p.H);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                run += d[j] * Ah;
+                a[j] = run;
+            }
+            float incl = run;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const float v = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += v;
+            }
+            float excl = __shfl_up_sync(0xffffffffu, incl, 1);
+            if (lane == 0) excl = 0.f;
+            const float last = __shfl_sync(0xffffffffu, incl, 31);
+            float *cso = p.cs + ((((size_t)b * p.H + h) * p.ncs + c) << 8) + lane * 8;
+            float *dto = p.dtT + ((((size_t)b * p.H + h) * p.ncs + c) << 8) + lane * 8;
+            float cv[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                cv[j] = a[j] + excl;
+                wsm[hh][lane * 8 + j] = __expf(fminf(last - cv[j], 0.f)) * d[j];
+            }
+            *reinterpret_cast<float4 *>(cso) = make_float4(cv[0], cv[1], cv[2], cv[3]);
+            *reinterpret_cast<float4 *>(cso + 4) = make_float4(cv[4], cv[5], cv[6], cv[7]);
+            *reinterpret_cast<float4 *>(dto) = make_float4(d[0], d[1], d[2], d[3]);
+            *reinterpret_cast<float4 *>(dto + 4) = make_float4(d[4], d[5], d[6], d[7]);
         }
-        wsm[hh][t] = w;
+    } else {
+        // per-row weights of both heads from the cumulative sums the forward-mode launch left
+        for (int i = tid; i < 512; i += CS_THREADS) {
+            const int hh = i >> 8, t = i & 255;
+            const float *csb = p.cs + ((((size_t)b * p.H + h0 + hh) * p.ncs + c) << 8);
+            wsm[hh][t] = __expf(csb[t]);
+        }
     }
     tc_fence_before_sync();
     __syncthreads();
