@@ -114,6 +114,14 @@ __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.b
 // all earlier stores of this thread are complete
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
+// Untiled bulk store shared -> global: `bytes` contiguous bytes (a multiple of 16, both addresses 16-byte
+// aligned), in the bulk async group of the issuing thread.
+__device__ __forceinline__ void bulk_store(void *gdst, const void *ssrc, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(reinterpret_cast<uint64_t>(gdst)),
+                 "r"(smem_u32(ssrc)), "r"(bytes)
+                 : "memory");
+}
+
 // ---------------------------------------------------------------- TMEM
 // Allocation is done by one full warp; the base address is written to *dst_smem.
 __device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t ncols) {

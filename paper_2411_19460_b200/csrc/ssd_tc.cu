@@ -85,10 +85,11 @@ bool tc_make_maps(const SegParams &p, TcMaps &m) {
 // C_t . dC_t that the decay gradient needs.  The C tile is already in shared memory (as rows of
 // time it is a K-major A operand), so it is one more product C (128 x N) * H_in^T (N x P) per head
 // and half into spare TMEM columns, and a row dot with the already scaled dy tile.
-constexpr int CS_THREADS = 128;
+constexpr int CS_THREADS = 256;
+constexpr int CS_OUT_STAGE = 128 * 528;   // result tile staged as 128 rows of 512 B, 16 B of padding each
 constexpr int CS_STAGE = 65536;   // X head0 16K | X head1 16K | V n0-63 16K | V n64-127 16K   (128 time rows)
 
-__global__ void __launch_bounds__(CS_THREADS)
+__global__ void __launch_bounds__(CS_THREADS, 3)
 k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmH) {
     extern __shared__ unsigned char smem_raw[];
@@ -100,6 +101,8 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
     const int c = blockIdx.x, hp = blockIdx.y, b = blockIdx.z;
     const int h0 = hp * 2, g = h0 / p.hpg;
     const int tid = threadIdx.x, warp = tid >> 5;
+    const int qrow = (warp & 3) * 32 + (tid & 31);   // row of the accumulator this thread can read (TMEM lane)
+    const int chalf = warp >> 2;                      // which half of the work of that row it takes
     const int tok0 = p.t0 + c * 256;
     const bool dstate = (mode == STATE_MODE_DSTATE);
 
@@ -227,18 +230,19 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
         tc_fence_after_sync();
         if (dstate) {
             // rho2_t = (e^{cs_t} dy_t) . Yoff_t with the scaled dy row read back from shared memory
-            for (int hh = 0; hh < 2; ++hh) {
+            {
+                const int hh = chalf;
                 float y0[32], y1[32];
-                const uint32_t ta = tm + ((uint32_t)(warp * 32) << 16) + 128 + hh * 64;
+                const uint32_t ta = tm + ((uint32_t)((warp & 3) * 32) << 16) + 128 + hh * 64;
                 tmem_ld32_nowait(ta, y0);
                 tmem_ld32_nowait(ta + 32, y1);
                 tmem_ld_wait32(y0);
                 tmem_ld_wait32(y1);
-                const unsigned char *row = smem + hh * 16384 + tid * 128;
+                const unsigned char *row = smem + hh * 16384 + qrow * 128;
                 float acc = 0.f;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    const uint4 v = *reinterpret_cast<const uint4 *>(row + ((j ^ (tid & 7)) << 4));
+                    const uint4 v = *reinterpret_cast<const uint4 *>(row + ((j ^ (qrow & 7)) << 4));
                     const __nv_bfloat162 *e = reinterpret_cast<const __nv_bfloat162 *>(&v);
                     const float *yy = (j < 4) ? (y0 + j * 8) : (y1 + (j - 4) * 8);
 #pragma unroll
@@ -248,7 +252,7 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
                         acc = fmaf(f.y, yy[2 * k + 1], acc);
                     }
                 }
-                p.rho2[((((size_t)b * p.H + h0 + hh) * p.ncs + c) << 8) + half * 128 + tid] = acc;
+                p.rho2[((((size_t)b * p.H + h0 + hh) * p.ncs + c) << 8) + half * 128 + qrow] = acc;
             }
         }
         tc_fence_before_sync();
@@ -258,27 +262,28 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
     }
 
     // The CTA's 128 x 128 fp32 result (two heads x 64 rows) is one contiguous 64 KB block of the state
-    // buffer.  Row-per-thread stores would touch 32 different lines per instruction, so the tile goes
-    // through the (now dead) stage: float4 (row, j) sits at slot j ^ (row & 31) of its row, which keeps
-    // both the row-per-thread writes and the row-per-warp reads free of bank conflicts.
+    // buffer.  Row-per-thread global stores would touch 32 different lines per instruction, so the tile is
+    // staged in the (now dead) stage, rows padded to 528 bytes (conflict-free row-per-thread writes), and
+    // every row leaves as one 512-byte bulk copy.
     {
-        float4 *stg = reinterpret_cast<float4 *>(smem);
+        float *stg = reinterpret_cast<float *>(smem);
 #pragma unroll
-        for (int c0 = 0; c0 < 128; c0 += 32) {
+        for (int c0 = 0; c0 < 64; c0 += 32) {
             float v[32];
-            tmem_ld32(tm + ((uint32_t)(warp * 32) << 16) + c0, v);
+            tmem_ld32(tm + ((uint32_t)((warp & 3) * 32) << 16) + chalf * 64 + c0, v);
 #pragma unroll
             for (int i = 0; i < 32; i += 4)
-                stg[tid * 32 + (((c0 + i) >> 2) ^ (tid & 31))] = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                *reinterpret_cast<float4 *>(stg + qrow * 132 + chalf * 64 + c0 + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
         }
+        fence_proxy_async_smem();
         __syncthreads();
-        const int slot = dstate ? c : c + 1;
-        float *base = dstate ? p.Gst : p.Hst;
-        float4 *out = reinterpret_cast<float4 *>(base + (((size_t)b * (p.ncs + 1) + slot) * p.H + h0) * 64 * 128);
-#pragma unroll 4
-        for (int it = 0; it < 32; ++it) {
-            const int idx = it * CS_THREADS + tid, row = idx >> 5, c4 = idx & 31;
-            out[idx] = stg[row * 32 + (c4 ^ (row & 31))];
+        if (tid < 128) {
+            const int slot = dstate ? c : c + 1;
+            float *base = dstate ? p.Gst : p.Hst;
+            float *out = base + ((((size_t)b * (p.ncs + 1) + slot) * p.H + h0) * 64 + tid) * 128;
+            bulk_store(out, stg + tid * 132, 512);
+            tma_store_commit();
+            tma_store_wait_read();
         }
     }
     tc_fence_before_sync();
@@ -287,7 +292,8 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
 }
 
 cudaError_t launch_chunk_state_tc(const SegParams &p, const TcMaps &m, int mode, cudaStream_t st) {
-    const int smem = CS_STAGE + (mode == STATE_MODE_DSTATE ? 32768 : 0) + 1024;
+    // forward mode: the stage, reused (and slightly outgrown) by the padded result tile
+    const int smem = (mode == STATE_MODE_DSTATE ? CS_STAGE + 32768 : CS_OUT_STAGE) + 1024;
     cudaError_t e = cudaFuncSetAttribute(k_chunk_state_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          CS_STAGE + 32768 + 1024);
     if (e != cudaSuccess) return e;
