@@ -221,6 +221,30 @@ def run_ours(args):
     for _ in range(max(args.warmup, 3)):
         step()
     barrier()
+    run_step = step
+    graph = None
+    if args.graph:
+        # the whole step (several hundred launches) captured once and replayed: the library only enqueues
+        # on the caller's stream, so it can be captured as it is
+        side = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(side):
+            stream_g = torch.cuda.current_stream()
+            def step_on_side():
+                libssd.ssd_fwd_segmented(inp["x"], inp["dt"], inp["A"], inp["Bm"], inp["Cm"], inp["D"], inp["h0"],
+                                         chunk=cfg.chunk, seg=seg, flags=flags, y=y, h_final=hf, boundary=bd,
+                                         ws=ws_f, stream=stream_g)
+                libssd.ssd_bwd_segmented(inp["x"], inp["dt"], inp["A"], inp["Bm"], inp["Cm"], inp["D"], bd, inp["dy"],
+                                         None, chunk=cfg.chunk, seg=seg, flags=flags, out=out, ws=ws_b, stream=stream_g)
+            step_on_side()
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                step_on_side()
+        torch.cuda.synchronize()
+        run_step = graph.replay
+        for _ in range(3):
+            run_step()
+        barrier()
     torch.cuda.reset_peak_memory_stats(dev)
     sampler = ClockSampler(dev) if rank == 0 else None
     n0 = libssd.launch_count()
@@ -228,7 +252,7 @@ def run_ours(args):
     barrier()
     e0.record(stream)
     for _ in range(args.steps):
-        step()
+        run_step()
     e1.record(stream)
     barrier()
     ms_total = max_over_ranks(e0.elapsed_time(e1))
@@ -327,6 +351,7 @@ def run_ours(args):
         "config": {"workload": cfg.name, "B": B, "L": L, "H": H, "P": P, "N": N, "G": cfg.G,
                    "chunk": cfg.chunk, "seg": seg, "nseg": nseg, "l2": "inputs larger than L2",
                    "path": "simt" if (args.simt or cfg.dtype == "fp32") else "default",
+                   "launch": "cuda graph replay" if args.graph else "stream launches",
                    "parallelism": "replicas" if world > 1 else "single"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline, "step_roofline": step_roof, "kernels": kinds,
@@ -473,6 +498,7 @@ def main():
     ap.add_argument("--simt", action="store_true", help="force the CUDA-core kernels")
     ap.add_argument("--stack-len", type=int, default=0, help="config 3: sequence length (default 131072)")
     ap.add_argument("--layers", type=int, default=0, help="config 3: number of layers (default 64)")
+    ap.add_argument("--graph", action="store_true", help="capture the step in a CUDA graph and time its replay")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-tokens", type=int, default=32768, help="tokens in the cpu_baseline sample")
