@@ -238,8 +238,10 @@ def run_ours(args):
             step_on_side()
             torch.cuda.synchronize()
             graph = torch.cuda.CUDAGraph()
+            nc0 = libssd.launch_count()
             with torch.cuda.graph(graph, stream=side):
                 step_on_side()
+            launches_per_replay = libssd.launch_count() - nc0      # kernel nodes of the captured step
         torch.cuda.synchronize()
         run_step = graph.replay
         for _ in range(3):
@@ -257,6 +259,8 @@ def run_ours(args):
     barrier()
     ms_total = max_over_ranks(e0.elapsed_time(e1))
     launches = libssd.launch_count() - n0
+    if graph is not None:
+        launches = launches_per_replay * args.steps
     clocks = sampler.stop() if sampler else None
     peak_mem = torch.cuda.max_memory_allocated(dev)
     assert libssd.poll_status(ws_f) == 0 and libssd.poll_status(ws_b) == 0, "device-side wait timed out"
