@@ -371,18 +371,20 @@ def run_ours(args):
 # ----------------------------------------------------------------------------- the stacked configuration
 def run_stack(args, rep, dev):
     """Config 3: 64 stacked layers under MA-GC (layer inputs + segment-boundary states kept), one step =
-    Algorithm 1 forward + Algorithm 2 backward of the whole stack.  The literal L = 262144 needs 175 GB of
-    layer inputs alone, so the sequence is run at --stack-len (default 131072) and the figure says so."""
+    Algorithm 1 forward + Algorithm 2 backward of the whole stack.  At layer interval 1 the literal
+    L = 262144 needs 175 GB of layer inputs alone, so it is run at --stack-len (default 131072) and the line
+    says so; with --layer-interval 2 or more (Eq. 4's l) the literal length fits and is the default."""
     from paper_2411_19460_b200 import libssd
     from paper_2411_19460_b200.inputs import make_stack_params
     from paper_2411_19460_b200.stack import LayerStack
 
     base = CONFIGS[args.config]
-    L = args.stack_len or 131072
+    L = args.stack_len or (131072 if args.layer_interval == 1 else base.L)
     cfg = base.scaled(L=L, seg=args.seg or base.seg, layers=args.layers or base.layers)
     inp = make_inputs(cfg, dev, seed=cfg.seed + rep.rank)
     sp = make_stack_params(cfg, dev)
-    st = LayerStack(inp["x"], inp["dt"], inp["Bm"], inp["Cm"], sp["A"], sp["D"], sp["W"], chunk=cfg.chunk, seg=cfg.seg)
+    st = LayerStack(inp["x"], inp["dt"], inp["Bm"], inp["Cm"], sp["A"], sp["D"], sp["W"], chunk=cfg.chunk, seg=cfg.seg,
+                    layer_interval=args.layer_interval)
     out = dict(dx0=torch.empty_like(inp["x"]), dA=torch.zeros(cfg.layers, cfg.H, device=dev),
                dD=torch.zeros(cfg.layers, cfg.H, device=dev))
     stream = torch.cuda.current_stream()
@@ -423,7 +425,7 @@ def run_stack(args, rep, dev):
         "warmup": max(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "impl": "ours",
         "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "L_in_definition": base.L, "layers": cfg.layers,
-                   "H": cfg.H, "P": cfg.P, "N": cfg.N, "G": cfg.G, "chunk": cfg.chunk, "seg": cfg.seg,
+                   "H": cfg.H, "P": cfg.P, "N": cfg.N, "G": cfg.G, "chunk": cfg.chunk, "seg": cfg.seg, "layer_interval": args.layer_interval,
                    "layer_tokens_per_s": value * cfg.layers, "l2": "inputs larger than L2",
                    "parallelism": "replicas" if rep.world > 1 else "single"},
         "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
@@ -500,9 +502,11 @@ def main():
                     "Mamba-2-2.7B-dim layer, L=131072)")
     ap.add_argument("--seg", type=int, default=0, help="override the segment length")
     ap.add_argument("--simt", action="store_true", help="force the CUDA-core kernels")
-    ap.add_argument("--stack-len", type=int, default=0, help="config 3: sequence length (default 131072)")
+    ap.add_argument("--layer-interval", type=int, default=1, help="config 3: keep the input of every l-th layer")
+    ap.add_argument("--stack-len", type=int, default=0, help="config 3: sequence length (default 131072 at layer interval 1, else the configuration's own)")
     ap.add_argument("--layers", type=int, default=0, help="config 3: number of layers (default 64)")
-    ap.add_argument("--graph", action="store_true", help="capture the step in a CUDA graph and time its replay")
+    ap.add_argument("--no-graph", dest="graph", action="store_false",
+                    help="time plain stream launches instead of the replay of the step captured in a CUDA graph")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-tokens", type=int, default=32768, help="tokens in the cpu_baseline sample")

@@ -1,10 +1,12 @@
-"""Driver for a stack of SSD layers under Multi-Axis Gradient Checkpointing, layer interval 1.
+"""Driver for a stack of SSD layers under Multi-Axis Gradient Checkpointing.
 
-Algorithm 1 (forward): segments outer, layers inner; along the layer axis only every layer's INPUT
-x_j is kept (L_ckpt), along the sequence axis only the state entering every segment of every layer
-(S_ckpt).  Algorithm 2 (backward): segments right to left (outer), layers top to bottom (inner); each
-grid cell (one layer x one segment) is restored from (x_j slice, state entering it), back-propagated,
-and hands dx down the layer stack and dh to the segment on its left.
+Algorithm 1 (forward): segments outer, layers inner; along the layer axis only the INPUT x_j of every
+`layer_interval`-th layer is kept (L_ckpt), along the sequence axis the state entering every segment
+of every layer (S_ckpt).  Algorithm 2 (backward): segments right to left (outer), blocks of
+`layer_interval` layers top to bottom (inner); each grid cell (one block x one segment) is restored
+from (x_j slice of its lowest layer, the states entering it): the inputs of its upper layers are
+recomputed into `layer_interval - 1` segment-long buffers (the l*s term of Eq. 4), then the cell is
+back-propagated layer by layer and hands dx down the stack and dh to the segment on its left.
 
 Layer j: y_j = SSD_j(x_j), x_{j+1} = W (y_j + x_j).  B, C, dt are shared by the layers; A, D are per layer.
 This module only marshals: every arithmetic step is a libssd call (ssd_fwd, ssd_bwd_segmented with
@@ -16,8 +18,10 @@ from . import libssd
 
 
 class LayerStack:
-    def __init__(self, x0, dt, Bm, Cm, A_list, D_list, W, *, chunk, seg, flags=0):
+    def __init__(self, x0, dt, Bm, Cm, A_list, D_list, W, *, chunk, seg, flags=0, layer_interval=1):
         self.layers = len(A_list)
+        self.interval = int(layer_interval)
+        assert 1 <= self.interval <= self.layers
         self.dt, self.Bm, self.Cm, self.A, self.D, self.W = dt, Bm, Cm, A_list, D_list, W
         self.chunk, self.seg, self.flags = int(chunk), int(seg), int(flags)
         B, L, H, P = x0.shape
@@ -27,14 +31,20 @@ class LayerStack:
         self.B, self.L, self.H, self.P, self.N = B, L, H, P, N
         self.nseg = L // self.seg
         dev = x0.device
-        # layer checkpoints: the input of every layer (x[0] is the caller's), plus the stack output
-        self.x = [x0] + [torch.empty_like(x0) for _ in range(self.layers)]
+        # layer checkpoints: the input of every `interval`-th layer (x[0] is the caller's) and the stack
+        # output; None for the layers whose input is recomputed inside a cell
+        self.x = [x0] + [torch.empty_like(x0) if (j % self.interval == 0 or j == self.layers) else None
+                         for j in range(1, self.layers + 1)]
         # sequence checkpoints: state entering segment k of layer j at [j][k]; [j][nseg] = final state
         self.bnd = torch.zeros(self.layers, self.nseg + 1, B, H, P, N, dtype=torch.float32, device=dev)
         # per-cell scratch
         self.y = torch.empty(B, self.seg, H, P, dtype=x0.dtype, device=dev)
         self.g = [torch.empty(B, self.seg, H, P, dtype=x0.dtype, device=dev) for _ in range(2)]
         self.dz = torch.empty(B, self.seg, H, P, dtype=x0.dtype, device=dev)
+        # inputs of the upper layers of a block, one segment long: forward passes through them, the
+        # backward recomputes them per cell
+        self.cx = [torch.empty(B, self.seg, H, P, dtype=x0.dtype, device=dev) for _ in range(self.interval - 1)]
+        self.h_scratch = torch.empty(B, H, P, N, dtype=torch.float32, device=dev) if self.interval > 1 else None
         cell = libssd.SSDShape(B, self.seg, H, P, N, Bm.shape[2], self.chunk, self.seg, libssd.SSD_DTYPE_BF16
                                if x0.dtype == torch.bfloat16 else libssd.SSD_DTYPE_F32, self.flags, 0, 0, 0)
         self.ws_f = libssd.alloc_workspace(cell, libssd.SSD_OP_FWD, dev)
@@ -42,7 +52,8 @@ class LayerStack:
         self.dh = torch.zeros(self.layers, 2, B, H, P, N, dtype=torch.float32, device=dev)
         # the slices every cell call takes (views; made once, the loops below are launch-bound otherwise)
         ns = self.nseg
-        self._xs = [[self._sl(t, k) for k in range(ns)] for t in self.x]
+        self._xs = [[self._sl(t, k) if t is not None else self.cx[j % self.interval - 1] for k in range(ns)]
+                    for j, t in enumerate(self.x)]
         self._dts = [self._sl(dt, k) for k in range(ns)]
         self._Bs = [self._sl(Bm, k) for k in range(ns)]
         self._Cs = [self._sl(Cm, k) for k in range(ns)]
@@ -90,6 +101,8 @@ class LayerStack:
             cur = (self.nseg - 1 - k) & 1              # dh[j, cur] enters from the right, dh[j, 1-cur] leaves
             g_in = self._sl(g_top, k)
             for j in range(self.layers - 1, -1, -1):
+                if self.interval > 1 and (j % self.interval == self.interval - 1 or j == self.layers - 1):
+                    self._restore_cell(j - j % self.interval, j, k)
                 xs = self._xs[j][k]
                 libssd.ssd_glue_bwd(g_in, self.W, self.dz)
                 dx = self._sl(out["dx0"], k) if j == 0 else self.g[j & 1]
@@ -105,9 +118,18 @@ class LayerStack:
         out["dh0"] = [self.dh[j, last] for j in range(self.layers)]
         return out
 
+    def _restore_cell(self, j0, j1, k):
+        """Recompute the inputs of layers j0+1..j1 on segment k from the kept x[j0] and the stored states."""
+        for j in range(j0, j1):
+            xs = self._xs[j][k]
+            libssd.ssd_fwd(xs, self._dts[k], self.A[j], self._Bs[k], self._Cs[k], self.D[j], self.bnd[j, k],
+                           chunk=self.chunk, seg=self.seg, flags=self.flags, y=self.y, h_final=self.h_scratch,
+                           ws=self.ws_f)
+            libssd.ssd_glue_fwd(xs, self.y, self.W, self._xs[j + 1][k])
+
     def checkpoint_bytes(self):
-        layer_inputs = sum(t.numel() * t.element_size() for t in self.x)
+        layer_inputs = sum(t.numel() * t.element_size() for t in self.x if t is not None)
         boundary = self.bnd.numel() * 4
         scratch = self.ws_f.numel() + self.ws_b.numel() + sum(
-            t.numel() * t.element_size() for t in (self.y, self.dz, self.g[0], self.g[1]))
+            t.numel() * t.element_size() for t in [self.y, self.dz, self.g[0], self.g[1]] + self.cx)
         return dict(layer_inputs=layer_inputs, boundary_states=boundary, per_cell_scratch=scratch)

@@ -85,3 +85,47 @@ def test_stack_matches_oracle_layer_by_layer():
         bad = {k: v for k, v in errs.items() if not (v <= tol)}
         assert not bad, (j, bad, errs)
     assert torch.equal(out["dx0"], keep["dx"][0])
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("interval", [2, 3])
+def test_layer_interval_changes_no_bit(interval):
+    """Algorithms 1/2 with a layer checkpoint every `interval` layers: the inputs of the layers in between
+    are recomputed per cell by the same kernels from the same operands, so every output equals the
+    interval-1 run (itself checked against the oracle above) bit for bit, while fewer layer inputs are kept.
+    4 layers: interval 3 leaves a partial block on top."""
+    from paper_2411_19460_b200.stack import LayerStack
+
+    cfg = CONFIGS[3].scaled(L=1024, H=4, seg=256, layers=4, dh_std=0.0)
+    inp = make_inputs(cfg, "cuda")
+    sp = make_stack_params(cfg, "cuda")
+    h0 = [torch.randn(cfg.B, cfg.H, cfg.P, cfg.N, device="cuda") * 0.1 for _ in range(cfg.layers)]
+
+    def run(l):
+        st = LayerStack(inp["x"], inp["dt"], inp["Bm"], inp["Cm"], sp["A"], sp["D"], sp["W"], chunk=cfg.chunk,
+                        seg=cfg.seg, layer_interval=l)
+        for j in range(cfg.layers):
+            st.set_h0(j, h0[j])
+        top = st.forward().clone()
+        cells = {}
+
+        def on_cell(j, k, cell):
+            cells[(j, k)] = {n: cell[n].clone() for n in ("dx", "ddt", "dB", "dC", "dy")}
+
+        out = st.backward(inp["dy"], on_cell=on_cell)
+        torch.cuda.synchronize()
+        res = dict(top=top, bnd=st.bnd.clone(), dx0=out["dx0"].clone(), dA=out["dA"].clone(), dD=out["dD"].clone(),
+                   dh0=torch.stack(out["dh0"]).clone())
+        return res, cells, st.checkpoint_bytes()
+
+    ref, ref_cells, ref_mem = run(1)
+    got, got_cells, mem = run(interval)
+    for name in ref:
+        assert torch.equal(ref[name], got[name]), name
+    assert ref_cells.keys() == got_cells.keys()
+    for key in ref_cells:
+        for name in ref_cells[key]:
+            assert torch.equal(ref_cells[key][name], got_cells[key][name]), (key, name)
+    kept = 1 + len([j for j in range(1, cfg.layers + 1) if j % interval == 0 or j == cfg.layers])
+    one = inp["x"].numel() * inp["x"].element_size()
+    assert mem["layer_inputs"] == kept * one < ref_mem["layer_inputs"] == (cfg.layers + 1) * one
