@@ -377,6 +377,7 @@ def run_stack(args, rep, dev):
     from paper_2411_19460_b200 import libssd
     from paper_2411_19460_b200.inputs import make_stack_params
     from paper_2411_19460_b200.stack import LayerStack
+    from paper_2411_19460_b200.memory_model import layer_stack_bytes
 
     base = CONFIGS[args.config]
     L = args.stack_len or (131072 if args.layer_interval == 1 else base.L)
@@ -431,6 +432,7 @@ def run_stack(args, rep, dev):
         "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
         "step_roofline": {"roofline_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms},
         "memory": dict(peak_allocated_bytes=int(peak_mem), **st.checkpoint_bytes()),
+        "memory_model": layer_stack_bytes(cfg.layers, cfg.L, args.layer_interval, cfg.seg, cfg.H, cfg.P, cfg.N),
     }
     print(json.dumps(line))
     rep.close()

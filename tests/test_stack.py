@@ -129,3 +129,6 @@ def test_layer_interval_changes_no_bit(interval):
     kept = 1 + len([j for j in range(1, cfg.layers + 1) if j % interval == 0 or j == cfg.layers])
     one = inp["x"].numel() * inp["x"].element_size()
     assert mem["layer_inputs"] == kept * one < ref_mem["layer_inputs"] == (cfg.layers + 1) * one
+    from paper_2411_19460_b200.memory_model import layer_stack_bytes
+    model = layer_stack_bytes(cfg.layers, cfg.L, interval, cfg.seg, cfg.H, cfg.P, cfg.N)
+    assert model["layer_inputs"] == mem["layer_inputs"] and model["boundary_states"] == mem["boundary_states"]
