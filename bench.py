@@ -184,6 +184,8 @@ def run_ours(args):
     rep = Replicas(backend="nccl", device=dev)
     rank, world = rep.rank, rep.world
     cfg = CONFIGS[args.config]
+    if args.stream_len:
+        return run_stream(args, rep, dev)
     if cfg.layers != 1:
         return run_stack(args, rep, dev)
     seg = args.seg or cfg.seg
@@ -438,6 +440,104 @@ def run_stack(args, rep, dev):
     rep.close()
 
 
+def run_stream(args, rep, dev):
+    """Forward-only streaming over --stream-len tokens (default 2^21) of the configuration's layer: ssd_fwd
+    segment by segment with only the state carried, then single-token steps on the same state.  Scratch is
+    one segment's; nothing grows with the length but the input and output themselves."""
+    from paper_2411_19460_b200 import libssd
+
+    base = CONFIGS[args.config]
+    L = args.stream_len
+    seg = args.seg or 16384
+    cfg = base.scaled(L=L, seg=seg)
+    inp = make_inputs(cfg, dev, seed=cfg.seed + rep.rank)
+    x, dt, A, Bm, Cm, D = (inp[k] for k in ("x", "dt", "A", "Bm", "Cm", "D"))
+    B, _, H, P = x.shape
+    N = Bm.shape[3]
+    y = torch.empty_like(x)
+    h = torch.zeros(B, H, P, N, dtype=torch.float32, device=dev)
+    h2 = torch.zeros_like(h)
+    cell = libssd.make_shape(x[:, :seg], Bm[:, :seg], cfg.chunk, seg, 0)
+    ws = libssd.alloc_workspace(cell, libssd.SSD_OP_FWD, dev)
+    assert B == 1, "slices of the sequence are passed as offset pointers: batch 1"
+    nseg = L // seg
+    views = [(x[:, k * seg:(k + 1) * seg], dt[:, k * seg:(k + 1) * seg], Bm[:, k * seg:(k + 1) * seg],
+              Cm[:, k * seg:(k + 1) * seg], y[:, k * seg:(k + 1) * seg]) for k in range(nseg)]
+    stream = torch.cuda.current_stream()
+
+    def step():
+        hin, hout = None, h
+        for xs, dts, Bs, Cs, ys in views:
+            libssd.ssd_fwd(xs, dts, A, Bs, Cs, D, hin, chunk=cfg.chunk, seg=seg, y=ys, h_final=hout, ws=ws, stream=stream)
+            hin, hout = hout, (h2 if hout is h else h)
+
+    for _ in range(max(args.warmup, 1)):
+        step()
+    rep.barrier()
+    torch.cuda.reset_peak_memory_stats(dev)
+    sampler = ClockSampler(dev) if rep.rank == 0 else None
+    n0 = libssd.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rep.barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    rep.barrier()
+    ms = rep.max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    launches = libssd.launch_count() - n0
+    clocks = sampler.stop() if sampler else None
+    peak_mem = torch.cuda.max_memory_allocated(dev)
+    assert libssd.poll_status(ws) == 0
+    # single-token steps, captured in a graph of 64 so that launch latency is the GPU's, not Python's
+    tok = [(x[:, t:t + 1].contiguous(), dt[:, t:t + 1].contiguous(), Bm[:, t:t + 1].contiguous(),
+            Cm[:, t:t + 1].contiguous(), torch.empty(B, 1, H, P, dtype=x.dtype, device=dev)) for t in range(64)]
+    side = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(side):
+        sg = torch.cuda.current_stream()
+        for xt, dtt, Bt, Ct, yt in tok[:2]:
+            libssd.ssd_decode_step(xt, dtt, A, Bt, Ct, D, h, y=yt, stream=sg)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for xt, dtt, Bt, Ct, yt in tok:
+                libssd.ssd_decode_step(xt, dtt, A, Bt, Ct, D, h, y=yt, stream=sg)
+    torch.cuda.synchronize()
+    for _ in range(3):
+        g.replay()
+    e0.record(stream)
+    for _ in range(20):
+        g.replay()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    us_per_token = e0.elapsed_time(e1) * 1e3 / (20 * 64)
+    if rep.rank != 0:
+        rep.close()
+        return
+    peaks = load_peaks()
+    state_bytes = 2 * B * H * P * N * 4
+    e = x.element_size()
+    fwd_bytes = (2 * H * P + 2 * cfg.G * N) * e + 4 * H            # per token: x, y, B, C, dt
+    line = {
+        "metric": "ssd_fwd_stream_tokens_per_s", "value": rep.world * L / (ms * 1e-3), "unit": UNIT, "n_gpus": rep.world,
+        "steps": args.steps, "warmup": max(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if e == 2 else "f32", "data": "synthetic", "impl": "ours",
+        "config": {"workload": cfg.name + "_forward_stream", "B": B, "L": L, "H": H, "P": P, "N": N, "G": cfg.G,
+                   "chunk": cfg.chunk, "seg": seg, "l2": "inputs larger than L2",
+                   "parallelism": "replicas" if rep.world > 1 else "single"},
+        "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "achieved": fwd_bytes * L / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": fwd_bytes * L / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                     "peak_source": peaks["source"]},
+        "decode_step": {"us_per_token": us_per_token, "state_bytes_per_token": state_bytes,
+                        "achieved_gbs": state_bytes / (us_per_token * 1e-6) / 1e9, "launch": "cuda graph of 64 steps"},
+        "memory": {"peak_allocated_bytes": int(peak_mem), "workspace_bytes": ws.numel(), "state_bytes": h.numel() * 4,
+                   "io_bytes": int(sum(t.numel() * t.element_size() for t in (x, dt, Bm, Cm, y)))},
+    }
+    print(json.dumps(line))
+    rep.close()
+
+
 # ----------------------------------------------------------------------------- the CPU oracle legs
 def _oracle_sample(cfg, inp, sample_tokens):
     """fp64 host copies of the first `sample_tokens` tokens (all heads) of the workload."""
@@ -506,6 +606,8 @@ def main():
     ap.add_argument("--simt", action="store_true", help="force the CUDA-core kernels")
     ap.add_argument("--layer-interval", type=int, default=1, help="config 3: keep the input of every l-th layer")
     ap.add_argument("--stack-len", type=int, default=0, help="config 3: sequence length (default 131072 at layer interval 1, else the configuration's own)")
+    ap.add_argument("--stream-len", type=int, default=0, help="forward-only streaming over this many tokens "
+                    "(e.g. 2097152) instead of the training step")
     ap.add_argument("--layers", type=int, default=0, help="config 3: number of layers (default 64)")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="time plain stream launches instead of the replay of the step captured in a CUDA graph")

@@ -171,6 +171,20 @@ int ssd_glue_bwd(const ssd_shape_t *shape, const void *g_next, const float *W, v
 int ssd_glue_residual(const ssd_shape_t *shape, void *dx, const void *dz, void *stream);
 
 /*
+ * One token of Eq. 1 for forward-only streaming (autoregressive decoding, or the tail of a sequence
+ * that is not a multiple of `chunk`): memory does not grow with the sequence, the state is all that
+ * is carried.  `shape->L` must be 1; B, H, P, N, G, dtype and the batch strides are read, `chunk`,
+ * `seg` and `flags` are ignored.
+ *   x, y  [B, 1, H, P] I/O dtype;  dt [B, 1, H] fp32;  Bm, Cm [B, 1, G, N] I/O dtype;  A, D [H] fp32;
+ *   h     [B, H, P, N] fp32, dense: the state BEFORE the token on entry, AFTER it on return (in place).
+ * ssd_fwd over a prefix followed by ssd_decode_step per token continues the same recurrence: feed
+ * ssd_fwd's h_final as `h`.  Any P; N in {64,128}.  Device pointers, enqueued on `stream`, no scratch.
+ * Returns SSD_OK or SSD_EINVAL / SSD_EUNSUPPORTED / SSD_EALIGN / SSD_ECUDA.
+ */
+int ssd_decode_step(const ssd_shape_t *shape, const void *x, const float *dt, const float *A,
+                    const void *Bm, const void *Cm, const float *D, float *h, void *y, void *stream);
+
+/*
  * Reads the status word at the start of `ws` (device memory) with a blocking copy: call it after
  * synchronising the stream.  Returns SSD_OK, SSD_ETIMEOUT if some kernel abandoned a bounded wait
  * (its outputs are then undefined), or SSD_ECUDA if the copy failed.

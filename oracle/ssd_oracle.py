@@ -95,3 +95,17 @@ def glue_bwd(g_next, W):
     """dz = W^T g_next: gradient of (y + x) given the gradient of x_next (fp64)."""
     g_next, W = map(_f64, (g_next, W))
     return np.einsum("ij,bthi->bthj", W, g_next)
+
+
+def decode_step(x, dt, A, Bm, Cm, D, h):
+    """One token of Eq. 1 written out (fp64): returns (y [B,H,P], h_new [B,H,P,N]) for x [B,H,P], dt [B,H],
+    Bm/Cm [B,G,N], state h [B,H,P,N]; head hh uses group hh // (H // G)."""
+    x, dt, A, Bm, Cm, D, h = map(_f64, (x, dt, A, Bm, Cm, D, h))
+    Bsz, H, P = x.shape
+    G = Bm.shape[1]
+    grp = np.arange(H) // (H // G)
+    Bh, Ch = Bm[:, grp], Cm[:, grp]                                   # [B,H,N]
+    alpha = np.exp(dt * A[None, :])                                   # [B,H]
+    h_new = alpha[:, :, None, None] * h + (dt[:, :, None] * x)[:, :, :, None] * Bh[:, :, None, :]
+    y = np.einsum("bhn,bhpn->bhp", Ch, h_new) + D[None, :, None] * x
+    return y, h_new

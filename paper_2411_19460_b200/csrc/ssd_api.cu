@@ -24,7 +24,7 @@ static size_t g_prof_used = 0;
 
 static const char *const kKindNames[KIND_COUNT] = {
     "chunk_cumsum", "chunk_state", "state_pass_fwd", "chunk_scan_fwd", "dstate_contrib",
-    "state_pass_bwd", "bwd_dx", "bwd_dC", "bwd_dB", "bwd_finish", "reduce_dBdC", "final_dAdD", "glue"};
+    "state_pass_bwd", "bwd_dx", "bwd_dC", "bwd_dB", "bwd_finish", "reduce_dBdC", "final_dAdD", "glue", "decode_step"};
 
 static ProfEvent *prof_begin(int kind, cudaStream_t st) {
     if (!g_prof_on) return nullptr;
@@ -479,6 +479,25 @@ int ssd_glue_residual(const ssd_shape_t *shape, void *dx, const void *dz, void *
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     SSD_LAUNCH(KIND_GLUE, launch_residual(shape->dtype, dx, dz, (long long)shape->L * shape->H * shape->P, bs, shape->B, st));
+    return SSD_OK;
+}
+
+int ssd_decode_step(const ssd_shape_t *s, const void *x, const float *dt, const float *A, const void *Bm,
+                    const void *Cm, const float *D, float *h, void *y, void *stream) {
+    if (!s || !x || !dt || !A || !Bm || !Cm || !D || !h || !y) return SSD_EINVAL;
+    if (s->B <= 0 || s->L != 1 || s->H <= 0 || s->P <= 0 || s->G <= 0 || s->H % s->G) return SSD_EINVAL;
+    if (s->N != 64 && s->N != 128) return SSD_EUNSUPPORTED;
+    if (s->dtype != SSD_DTYPE_F32 && s->dtype != SSD_DTYPE_BF16) return SSD_EUNSUPPORTED;
+    const long long x_bs = s->x_bstride ? s->x_bstride : (long long)s->H * s->P;
+    const long long dt_bs = s->dt_bstride ? s->dt_bstride : (long long)s->H;
+    const long long bc_bs = s->bc_bstride ? s->bc_bstride : (long long)s->G * s->N;
+    if (x_bs < (long long)s->H * s->P || dt_bs < s->H || bc_bs < (long long)s->G * s->N) return SSD_EINVAL;
+    if (misaligned(x) || misaligned(dt) || misaligned(A) || misaligned(Bm) || misaligned(Cm) || misaligned(D) ||
+        misaligned(h) || misaligned(y))
+        return SSD_EALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    SSD_LAUNCH(KIND_DECODE, launch_decode_step(s->dtype, s->N, x, dt, A, Bm, Cm, D, h, y, s->B, s->H, s->P, s->G,
+                                               x_bs, dt_bs, bc_bs, st));
     return SSD_OK;
 }
 

@@ -74,6 +74,11 @@ cudaError_t launch_glue(int dtype, bool transpose, const void *a, const void *b,
 cudaError_t launch_residual(int dtype, void *dst, const void *src, long long n_per_batch, long long bstride, int B,
                             cudaStream_t st);
 
+// ssd_decode.cu : one token of the recurrence, state updated in place
+cudaError_t launch_decode_step(int dtype, int N, const void *x, const float *dt, const float *A, const void *Bm,
+                               const void *Cm, const float *D, float *h, void *y, int B, int H, int P, int G,
+                               long long x_bs, long long dt_bs, long long bc_bs, cudaStream_t st);
+
 // ssd_tc.cu : tensor-core (tcgen05 / TMEM / TMA) kernels, bf16 I/O
 struct TcMaps {
     CUtensorMap x, dy, Bm, Cm;  // [B][L][H*64] / [B][L][G*128], box 64 x 128 rows
@@ -95,7 +100,7 @@ enum { STATE_MODE_FWD = 0, STATE_MODE_DSTATE = 1 };
 enum {
     KIND_CUMSUM = 0, KIND_CHUNK_STATE, KIND_STATE_PASS_FWD, KIND_SCAN_FWD, KIND_DSTATE,
     KIND_STATE_PASS_BWD, KIND_BWD_DX, KIND_BWD_DC, KIND_BWD_DB, KIND_BWD_FINISH, KIND_REDUCE_DBDC,
-    KIND_FINAL, KIND_GLUE, KIND_COUNT
+    KIND_FINAL, KIND_GLUE, KIND_DECODE, KIND_COUNT
 };
 enum { MP_FWD = 0, MP_BWD_DX = 1, MP_DC = 2, MP_DB = 3 };
 

@@ -23,7 +23,7 @@ EXPORTS = ["ssd_workspace_bytes", "ssd_boundary_bytes", "ssd_fwd", "ssd_fwd_segm
            "ssd_bwd_segmented", "ssd_poll_status", "ssd_strerror", "ssd_version",
            "ssd_last_cuda_error", "ssd_launch_count", "ssd_kernel_kinds", "ssd_kernel_name",
            "ssd_profile", "ssd_profile_read", "ssd_fwd_static_ws", "ssd_glue_fwd", "ssd_glue_bwd",
-           "ssd_glue_residual"]
+           "ssd_glue_residual", "ssd_decode_step"]
 
 
 class SSDShape(ctypes.Structure):
@@ -70,6 +70,8 @@ def lib():
         L.ssd_glue_fwd.argtypes = [sp, vp, vp, fp, vp, vp]
         L.ssd_glue_bwd.restype = ctypes.c_int
         L.ssd_glue_bwd.argtypes = [sp, vp, fp, vp, vp]
+        L.ssd_decode_step.restype = ctypes.c_int
+        L.ssd_decode_step.argtypes = [sp, vp, fp, fp, vp, vp, fp, fp, vp, vp]
         L.ssd_glue_residual.restype = ctypes.c_int
         L.ssd_glue_residual.argtypes = [sp, vp, vp, vp]
         L.ssd_poll_status.restype = ctypes.c_int
@@ -241,6 +243,33 @@ def ssd_bwd_segmented(x, dt, A, Bm, Cm, D, boundary, dy, dh_final=None, *, chunk
     if rc != SSD_OK:
         raise SSDError(rc, "ssd_bwd_segmented")
     return out
+
+
+def ssd_decode_step(x, dt, A, Bm, Cm, D, h, y=None, stream=None):
+    """One token of Eq. 1: h (fp32 [B,H,P,N]) is advanced in place, y [B,1,H,P] is returned.
+    x [B,1,H,P], dt [B,1,H], Bm/Cm [B,1,G,N] may be one-token slices of longer tensors."""
+    if not (x.is_cuda and h.is_cuda):
+        raise ValueError("device tensors required")
+    B, L, H, P = x.shape
+    G, N = Bm.shape[2], Bm.shape[3]
+    if L != 1 or dt.shape != (B, 1, H) or Cm.shape != Bm.shape or Bm.shape[:2] != (B, 1):
+        raise ValueError("ssd_decode_step takes one token: x [B,1,H,P], dt [B,1,H], Bm/Cm [B,1,G,N]")
+    if h.shape != (B, H, P, N) or h.dtype != torch.float32 or not h.is_contiguous():
+        raise ValueError("h must be a contiguous float32 [B,H,P,N] tensor")
+    if x.dtype not in (torch.bfloat16, torch.float32) or Bm.dtype != x.dtype or Cm.dtype != x.dtype:
+        raise TypeError("x, Bm, Cm must share dtype float32 or bfloat16")
+    # one-token slices of longer tensors are made dense here (a few KB); the C call also takes batch strides
+    x, dt, Bm, Cm = x.contiguous(), dt.contiguous(), Bm.contiguous(), Cm.contiguous()
+    y = torch.empty(B, 1, H, P, dtype=x.dtype, device=x.device) if y is None else y
+    if not y.is_contiguous() or y.shape != x.shape or y.dtype != x.dtype:
+        raise ValueError("y must be a dense tensor like x")
+    code = SSD_DTYPE_BF16 if x.dtype == torch.bfloat16 else SSD_DTYPE_F32
+    shape = SSDShape(B, 1, H, P, N, G, 0, 0, code, 0, 0, 0, 0)
+    rc = lib().ssd_decode_step(ctypes.byref(shape), _ptr(x), _ptr(dt), _ptr(A), _ptr(Bm), _ptr(Cm), _ptr(D),
+                               _ptr(h), _ptr(y), _stream(stream))
+    if rc != SSD_OK:
+        raise SSDError(rc, "ssd_decode_step")
+    return y
 
 
 def _glue_shape(t):
