@@ -189,7 +189,7 @@ def run_ours(args):
     if cfg.layers != 1:
         return run_stack(args, rep, dev)
     seg = args.seg or cfg.seg
-    flags = libssd.SSD_FLAG_FORCE_SIMT if args.simt else 0
+    flags = (libssd.SSD_FLAG_FORCE_SIMT if args.simt else 0) | (libssd.SSD_FLAG_SERIAL if args.serial else 0)
     inp = make_inputs(cfg, dev, seed=cfg.seed + rank)
     x, dt, A, Bm, Cm, D, h0, dy = (inp[k] for k in ("x", "dt", "A", "Bm", "Cm", "D", "h0", "dy"))
     B, L, H, P = x.shape
@@ -611,6 +611,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="config 3: number of layers (default 64)")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="time plain stream launches instead of the replay of the step captured in a CUDA graph")
+    ap.add_argument("--serial", action="store_true", help="backward: no helper streams, every kernel in order on one stream")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-tokens", type=int, default=32768, help="tokens in the cpu_baseline sample")

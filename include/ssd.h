@@ -11,9 +11,10 @@
  * per batch b and head h; head h uses the B/C vectors of group g = h / (H/G).
  *
  * Conventions common to every call
- *  - All tensor pointers are DEVICE pointers owned by the caller.  The library allocates nothing,
- *    frees nothing and never synchronises; work is enqueued on `stream` (a cudaStream_t passed as
- *    void*, NULL = the legacy default stream).  `shape` is a HOST pointer, read before return.
+ *  - All tensor pointers are DEVICE pointers owned by the caller.  The library allocates no device
+ *    memory, frees nothing and never synchronises; work is enqueued on `stream` (a cudaStream_t passed
+ *    as void*, NULL = the legacy default stream) or ordered after and before it (see SSD_FLAG_SERIAL):
+ *    everything a call enqueued is complete once `stream` has reached the point of the call's return.  `shape` is a HOST pointer, read before return.
  *  - Row-major, innermost dimension contiguous:
  *      x, y, dy, dx        [B, L, H, P]   I/O dtype (fp32 or bf16), batch stride x_bstride
  *      dt, ddt             [B, L, H]      fp32, batch stride dt_bstride
@@ -53,8 +54,12 @@ enum { SSD_DTYPE_F32 = 0, SSD_DTYPE_BF16 = 1 };
 /* shape.flags */
 enum {
     SSD_FLAG_FORCE_SIMT = 1,       /* bf16 I/O: use the CUDA-core kernels instead of the tensor-core ones */
-    SSD_FLAG_ACCUM_PARAM_GRADS = 2 /* ssd_bwd_segmented: dA and dD are added to, not overwritten (a driver that
+    SSD_FLAG_ACCUM_PARAM_GRADS = 2,/* ssd_bwd_segmented: dA and dD are added to, not overwritten (a driver that
                                       back-propagates one grid cell at a time sums them over the cells) */
+    SSD_FLAG_SERIAL = 4            /* ssd_bwd_segmented: launch every kernel on `stream` itself, in order.  By default
+                                      the tensor-core path runs its three mutually independent gradient kernels of a
+                                      segment on two library-owned helper streams forked off `stream` and joined back
+                                      into it before the call returns to the next segment; results are the same bits */
 };
 
 /* `op` of ssd_workspace_bytes */

@@ -190,6 +190,31 @@ static int check_device() {
     return cached_ok ? SSD_OK : SSD_EDEVICE;
 }
 
+// Two helper streams per (host thread, device) for the backward's independent kernels, with the events
+// that fork them off the caller's stream and join them back.  Created on first use, never destroyed
+// (they hold no device memory); the caller's stream stays the only one the caller has to order against.
+struct SideStreams {
+    int dev = -1;
+    cudaStream_t s[2] = {nullptr, nullptr};
+    cudaEvent_t fork[2] = {nullptr, nullptr}, join[2] = {nullptr, nullptr};
+};
+static SideStreams *side_streams() {
+    static thread_local std::vector<SideStreams> all;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    for (auto &a : all)
+        if (a.dev == dev) return &a;
+    SideStreams a;
+    a.dev = dev;
+    for (int i = 0; i < 2; ++i) {
+        if (cudaStreamCreateWithFlags(&a.s[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&a.fork[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&a.join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    }
+    all.push_back(a);
+    return &all.back();
+}
+
 #define SSD_TRY(expr)                                   \
     do {                                                \
         cudaError_t e__ = (expr);                       \
@@ -406,6 +431,15 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
     TcMaps maps;
     if (pl.use_tc && !tc_make_maps(sp, maps)) return SSD_ECUDA;
     const long long PN = (long long)pl.P * pl.N;
+    // The dC kernel needs only the recomputed states, the dB and dx kernels also the state gradients; the
+    // three do not depend on one another.  Unless told otherwise they run on side streams forked off the
+    // caller's stream and joined back before the segment's finishing kernels, so that one kernel's tail
+    // (its last, partly idle wave) is filled by the next one's CTAs.
+    SideStreams *side = nullptr;
+    if (pl.use_tc && !(shape->flags & SSD_FLAG_SERIAL) && !g_prof_on) {
+        side = side_streams();
+        if (!side) { g_last_cuda = (int)cudaGetLastError(); return SSD_ECUDA; }
+    }
     for (int k = pl.nseg - 1; k >= 0; --k) {
         set_segment(pl, k, sp);
         // Recompute_Forward: chunk-entry states of segment k from the stored boundary state
@@ -417,15 +451,36 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
         }
         SSD_LAUNCH(KIND_STATE_PASS_FWD, launch_state_pass_fwd(sp, boundary + (size_t)k * pl.H * PN, (long long)pl.nseg * pl.H * PN,
                                       nullptr, 0, nullptr, pl.use_tc, st));
+        if (side) {
+            SSD_TRY(cudaEventRecord(side->fork[0], st));
+            SSD_TRY(cudaStreamWaitEvent(side->s[0], side->fork[0], 0));
+            {
+                cudaStream_t st = side->s[0];
+                SSD_LAUNCH(KIND_BWD_DC, launch_grad_bc_tc(sp, maps, GB_DC, st));
+                SSD_TRY(cudaEventRecord(side->join[0], st));
+            }
+        }
         // Backward through the segment; dh enters from the right, leaves to the left
         if (pl.use_tc) SSD_LAUNCH(KIND_DSTATE, launch_chunk_state_tc(sp, maps, STATE_MODE_DSTATE, st));
         else SSD_LAUNCH(KIND_DSTATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_DSTATE, st));
         const float *ginit = (k == pl.nseg - 1) ? dh_final : sp.gcarry;
         float *gleft = (k == 0 && dh0) ? dh0 : sp.gcarry;
         SSD_LAUNCH(KIND_STATE_PASS_BWD, launch_state_pass_bwd(sp, ginit, gleft, pl.use_tc, st));
+        if (side) {
+            SSD_TRY(cudaEventRecord(side->fork[1], st));
+            SSD_TRY(cudaStreamWaitEvent(side->s[1], side->fork[1], 0));
+            {
+                cudaStream_t st = side->s[1];
+                SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_tc(sp, maps, GB_DB, st));
+                SSD_TRY(cudaEventRecord(side->join[1], st));
+            }
+        }
         if (pl.use_tc) SSD_LAUNCH(KIND_BWD_DX, launch_scan_tc(sp, maps, SC_DX, st));
         else SSD_LAUNCH(KIND_BWD_DX, launch_masked_product_simt(sp, pl.dtype, MP_BWD_DX, st));
-        if (pl.use_tc) {
+        if (side) {
+            SSD_TRY(cudaStreamWaitEvent(st, side->join[0], 0));
+            SSD_TRY(cudaStreamWaitEvent(st, side->join[1], 0));
+        } else if (pl.use_tc) {
             SSD_LAUNCH(KIND_BWD_DC, launch_grad_bc_tc(sp, maps, GB_DC, st));
             SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_tc(sp, maps, GB_DB, st));
         } else {

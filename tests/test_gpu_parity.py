@@ -97,3 +97,21 @@ def test_status_word_clean():
                              chunk=cfg.chunk, seg=cfg.seg, ws=ws)
     torch.cuda.synchronize()
     assert libssd.poll_status(ws) == libssd.SSD_OK
+
+
+@pytest.mark.gpu
+def test_helper_streams_change_no_bit_and_respect_caller_stream():
+    """The backward's forked helper streams (default) against SSD_FLAG_SERIAL: the same bits, also when the
+    caller's stream is not the default one and is the only thing the caller synchronises."""
+    cfg = small(B=2, L=2048, H=8, G=2, seg=512)
+    inp = make_inputs(cfg, "cuda")
+    ref = pu.run_gpu(cfg, inp, flags=libssd.SSD_FLAG_SERIAL)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        g = libssd.ssd_bwd_segmented(inp["x"], inp["dt"], inp["A"], inp["Bm"], inp["Cm"], inp["D"], ref["boundary"],
+                                     inp["dy"], inp["dh_final"], chunk=cfg.chunk, seg=cfg.seg, stream=s)
+    s.synchronize()                                   # only the caller's stream
+    for k, v in g.items():
+        if v is not None:
+            assert torch.equal(v, ref[k]), k
