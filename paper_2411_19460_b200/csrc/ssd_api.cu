@@ -45,6 +45,7 @@ static void prof_end(ProfEvent *ev, cudaStream_t st) {
 
 struct Layout {
     size_t status, cs, dtT, Hst, Hbf, hcarry, Gst, Gbf, gcarry, ghdot, ddt_dir, rho, rho2, psi, psi2, pB, pC, dAp, dDp;
+    size_t dtT_b, rho2_b, ghdot_b;   // second copies: a segment's finishing kernels overlap the next segment's first ones
     size_t total;
 };
 
@@ -168,6 +169,9 @@ static void make_layout(const Plan &pl, int op, Layout &lo) {
         lo.pC = take(part);
         lo.dAp = take(BH * pl.nct * sizeof(float));
         lo.dDp = take(BH * pl.nct * 16 * sizeof(float));
+        lo.dtT_b = take(pl.use_tc ? vec : 0);
+        lo.rho2_b = take(pl.use_tc ? vec : 0);
+        lo.ghdot_b = take(pl.use_tc ? BH * pl.ncs * 8 * sizeof(float) : 0);
     }
     lo.total = o;
 }
@@ -195,8 +199,9 @@ static int check_device() {
 // (they hold no device memory); the caller's stream stays the only one the caller has to order against.
 struct SideStreams {
     int dev = -1;
-    cudaStream_t s[2] = {nullptr, nullptr};
+    cudaStream_t s[3] = {nullptr, nullptr, nullptr};
     cudaEvent_t fork[2] = {nullptr, nullptr}, join[2] = {nullptr, nullptr};
+    cudaEvent_t tail_go = nullptr, tail_done = nullptr;
 };
 static SideStreams *side_streams() {
     static thread_local std::vector<SideStreams> all;
@@ -206,11 +211,14 @@ static SideStreams *side_streams() {
         if (a.dev == dev) return &a;
     SideStreams a;
     a.dev = dev;
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < 3; ++i)
         if (cudaStreamCreateWithFlags(&a.s[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    for (int i = 0; i < 2; ++i) {
         if (cudaEventCreateWithFlags(&a.fork[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
         if (cudaEventCreateWithFlags(&a.join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
     }
+    if (cudaEventCreateWithFlags(&a.tail_go, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&a.tail_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     all.push_back(a);
     return &all.back();
 }
@@ -440,8 +448,18 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
         side = side_streams();
         if (!side) { g_last_cuda = (int)cudaGetLastError(); return SSD_ECUDA; }
     }
+    // With the helper streams, a segment's two finishing kernels (which are short and latency-bound) run on
+    // a third one while the caller's stream already recomputes the next segment; what they read and the
+    // next segment's first kernels rewrite (dt per chunk, rho2, <G,H>) alternates between two copies.
+    bool tail_pending = false;
     for (int k = pl.nseg - 1; k >= 0; --k) {
         set_segment(pl, k, sp);
+        if (side) {
+            const bool odd = ((pl.nseg - 1 - k) & 1) != 0;
+            sp.dtT = (float *)((char *)ws + (odd ? lo.dtT_b : lo.dtT));
+            sp.rho2 = (float *)((char *)ws + (odd ? lo.rho2_b : lo.rho2));
+            sp.ghdot = (float *)((char *)ws + (odd ? lo.ghdot_b : lo.ghdot));
+        }
         // Recompute_Forward: chunk-entry states of segment k from the stored boundary state
         if (pl.use_tc) {   // the tensor-core chunk-state kernel computes the chunk cumsum itself
             SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_tc(sp, maps, STATE_MODE_FWD, st));
@@ -454,6 +472,7 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
         if (side) {
             SSD_TRY(cudaEventRecord(side->fork[0], st));
             SSD_TRY(cudaStreamWaitEvent(side->s[0], side->fork[0], 0));
+            if (tail_pending) SSD_TRY(cudaStreamWaitEvent(side->s[0], side->tail_done, 0));
             {
                 cudaStream_t st = side->s[0];
                 SSD_LAUNCH(KIND_BWD_DC, launch_grad_bc_tc(sp, maps, GB_DC, st));
@@ -469,6 +488,11 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
         if (side) {
             SSD_TRY(cudaEventRecord(side->fork[1], st));
             SSD_TRY(cudaStreamWaitEvent(side->s[1], side->fork[1], 0));
+            if (tail_pending) {
+                SSD_TRY(cudaStreamWaitEvent(side->s[1], side->tail_done, 0));
+                SSD_TRY(cudaStreamWaitEvent(st, side->tail_done, 0));
+                tail_pending = false;
+            }
             {
                 cudaStream_t st = side->s[1];
                 SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_tc(sp, maps, GB_DB, st));
@@ -487,9 +511,22 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
             SSD_LAUNCH(KIND_BWD_DC, launch_masked_product_simt(sp, pl.dtype, MP_DC, st));
             SSD_LAUNCH(KIND_BWD_DB, launch_masked_product_simt(sp, pl.dtype, MP_DB, st));
         }
-        SSD_LAUNCH(KIND_BWD_FINISH, launch_bwd_finish(sp, st));
-        SSD_LAUNCH(KIND_REDUCE_DBDC, launch_reduce_dbdc(sp, pl.dtype, st));
+        if (side) {
+            SSD_TRY(cudaEventRecord(side->tail_go, st));
+            SSD_TRY(cudaStreamWaitEvent(side->s[2], side->tail_go, 0));
+            {
+                cudaStream_t st = side->s[2];
+                SSD_LAUNCH(KIND_BWD_FINISH, launch_bwd_finish(sp, st));
+                SSD_LAUNCH(KIND_REDUCE_DBDC, launch_reduce_dbdc(sp, pl.dtype, st));
+                SSD_TRY(cudaEventRecord(side->tail_done, st));
+            }
+            tail_pending = true;
+        } else {
+            SSD_LAUNCH(KIND_BWD_FINISH, launch_bwd_finish(sp, st));
+            SSD_LAUNCH(KIND_REDUCE_DBDC, launch_reduce_dbdc(sp, pl.dtype, st));
+        }
     }
+    if (tail_pending) SSD_TRY(cudaStreamWaitEvent(st, side->tail_done, 0));
     SSD_LAUNCH(KIND_FINAL, launch_final_dAdD(sp, dA, dD, (shape->flags & SSD_FLAG_ACCUM_PARAM_GRADS) != 0, st));
     return SSD_OK;
 }
