@@ -261,6 +261,35 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
         : "memory");
 }
 
+// The same with the accumulate flag fixed at compile time, and a descriptor rebuilt from its two words.
+// The thread that issues the MMAs executes roughly one dependent instruction every five cycles, so the
+// per-MMA bookkeeping decides whether the tensor pipe stays fed: issue loops are fully unrolled and
+// advance only the low descriptor word (the 14-bit address field, in 16-byte units, never carries out).
+template <bool ACCUMULATE>
+__device__ __forceinline__ void umma_bf16_fixed(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+    if (ACCUMULATE)
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "setp.eq.b32 p, 0, 0;\n"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+            "}\n" ::"r"(d_tmem),
+            "l"(adesc), "l"(bdesc), "r"(idesc)
+            : "memory");
+    else
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "setp.ne.b32 p, 0, 0;\n"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+            "}\n" ::"r"(d_tmem),
+            "l"(adesc), "l"(bdesc), "r"(idesc)
+            : "memory");
+}
+__device__ __forceinline__ uint64_t umma_desc_words(uint32_t lo, uint32_t hi) {
+    return ((uint64_t)hi << 32) | (uint64_t)lo;
+}
+
 // Makes `bar` complete once all MMAs issued so far by this thread have finished.
 __device__ __forceinline__ void umma_commit(uint64_t *bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))

@@ -27,6 +27,8 @@
 // sub-tile, j1 = last column of the column sub-tile), three factors that are each <= 1 because cs
 // is non-increasing, so only O(Q) exponentials are needed per head instead of O(Q^2); diagonal
 // sub-tiles are exponentiated element by element.
+#include <type_traits>
+
 #include "ssd_internal.h"
 #include "ssd_sm100.cuh"
 
@@ -112,15 +114,15 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
         for (int i = 0; i < 2; ++i) {
             mbar_init(&hfull[i], 1);
             mbar_init(&hempty[i], 1);
-            mbar_init(&mfull[i], 256);
+            mbar_init(&mfull[i], 4);           // one arrival per warp (lane 0, after __syncwarp()) of the slot's four
             mbar_init(&mempty[i], 1);
             mbar_init(&accfull[i], 1);
-            mbar_init(&accempty[i], 128);
-            mbar_init(&vfull[i], 32);
-            mbar_init(&vempty[i], 256 + 128);
+            mbar_init(&accempty[i], 4);
+            mbar_init(&vfull[i], 1);
+            mbar_init(&vempty[i], 8 + 4);
         }
         mbar_init(&xrfull, 1);
-        mbar_init(&xrempty, 128);
+        mbar_init(&xrempty, 4);
         abort_flag = 0;
         fence_barrier_init();
     }
@@ -178,38 +180,53 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                 umma_bf16(tm, ad, bd, idS, kk ? 1u : 0u);
             }
             umma_commit(&bar_s);
-            uint32_t mcnt = 0;   // pieces of M consumed so far
-            // descriptors of the loop-invariant operands, advanced by plain adds inside the loops
+            // Descriptors of the loop-invariant operands as (low word, high word); every offset below is a
+            // compile-time constant in 16-byte units once the loops are unrolled.
             const uint64_t dRows = umma_desc_sw128(sRows, 16, 1024), dSt = umma_desc_sw128(sSt, 16, 1024);
             const uint64_t dM = umma_desc_sw128(sM, 16, 1024), dX = umma_desc_sw128(sX, 8192, 1024);
-            for (int hi = 0; hi < nheads; ++hi) {
-                const int buf = hi & 1, xs = hi % 3, xuse = hi / 3;
-                const uint32_t acc1 = tm + 256 + buf * 128, acc2 = acc1 + 64;
-                if (hi >= 2) mbar_wait(&accempty[buf], ((hi >> 1) - 1) & 1, abortp, p.status);
-                mbar_wait(&hfull[buf], (hi >> 1) & 1, abortp, p.status);
-                tc_fence_after_sync();
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    umma_bf16(acc2, umma_desc_advance(dRows, (kk >> 2) * 16384 + (kk & 3) * 32),
-                              umma_desc_advance(dSt, buf * 16384 + (kk >> 2) * 8192 + (kk & 3) * 32), id3, kk ? 1u : 0u);
-                }
-                umma_commit(&hempty[buf]);
-                mbar_wait(&xfull[xs], xuse & 1, abortp, p.status);
-                for (int jj = 0; jj < npieces; ++jj) {
-                    const uint32_t ms = mcnt & 1;
-                    mbar_wait(&mfull[ms], (mcnt >> 1) & 1, abortp, p.status);
-                    ++mcnt;
+            const uint32_t loR = (uint32_t)dRows, hiR = (uint32_t)(dRows >> 32), loS = (uint32_t)dSt, hiS = (uint32_t)(dSt >> 32);
+            const uint32_t loM = (uint32_t)dM, hiM = (uint32_t)(dM >> 32), loX = (uint32_t)dX, hiX = (uint32_t)(dX >> 32);
+            auto run = [&](auto np_c) {
+                constexpr int NP = decltype(np_c)::value;     // pieces per head: 2 or 4, so piece jj uses ring slot jj & 1
+                int xs = 0, xuse = 0;
+                for (int hi = 0; hi < nheads; ++hi) {
+                    const int buf = hi & 1;
+                    const uint32_t acc1 = tm + 256 + buf * 128, acc2 = acc1 + 64;
+                    const uint32_t loSb = loS + buf * 1024, loXh = loX + xs * 2048;
+                    const uint32_t par = (uint32_t)(hi >> 1) & 1u;
+                    if (hi >= 2) mbar_wait(&accempty[buf], par ^ 1u, abortp, p.status);
+                    mbar_wait(&hfull[buf], par, abortp, p.status);
                     tc_fence_after_sync();
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        umma_bf16(acc1, umma_desc_advance(dM, ms * 16384 + k * 32),
-                                  umma_desc_advance(dX, xs * 32768 + (jj * 64 + k * 16) * 128), id2, (jj | k) ? 1u : 0u);
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const uint32_t oa = (kk >> 2) * 1024 + (kk & 3) * 2, ob = (kk >> 2) * 512 + (kk & 3) * 2;
+                        if (kk == 0) umma_bf16_fixed<false>(acc2, umma_desc_words(loR + oa, hiR), umma_desc_words(loSb + ob, hiS), id3);
+                        else umma_bf16_fixed<true>(acc2, umma_desc_words(loR + oa, hiR), umma_desc_words(loSb + ob, hiS), id3);
                     }
-                    umma_commit(&mempty[ms]);
+                    umma_commit(&hempty[buf]);
+                    mbar_wait(&xfull[xs], (uint32_t)xuse & 1u, abortp, p.status);
+                    const uint32_t pbase = (uint32_t)(hi * (NP / 2)) & 1u;      // parity of ring use (hi NP + jj) >> 1
+#pragma unroll
+                    for (int jj = 0; jj < NP; ++jj) {
+                        const int ms = jj & 1;
+                        mbar_wait(&mfull[ms], pbase ^ (uint32_t)((jj >> 1) & 1), abortp, p.status);
+                        tc_fence_after_sync();
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const uint64_t ad = umma_desc_words(loM + ms * 1024 + k * 2, hiM);
+                            const uint64_t bd = umma_desc_words(loXh + jj * 512 + k * 128, hiX);
+                            if (jj == 0 && k == 0) umma_bf16_fixed<false>(acc1, ad, bd, id2);
+                            else umma_bf16_fixed<true>(acc1, ad, bd, id2);
+                        }
+                        umma_commit(&mempty[ms]);
+                    }
+                    umma_commit(&accfull[buf]);
+                    umma_commit(&xempty[xs]);
+                    if (++xs == 3) { xs = 0; ++xuse; }
                 }
-                umma_commit(&accfull[buf]);
-                umma_commit(&xempty[xs]);
-            }
+            };
+            if (npieces == 4) run(std::integral_constant<int, 4>{});
+            else run(std::integral_constant<int, 2>{});
         }
     } else if (warp == 10) {
         // ------------------------------------------------------------ vector warp
@@ -245,12 +262,12 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                 const int idx = lane + 32 * w, i = idx >> 3, j = idx & 7;   // blk[i][j] = e^{cs[32 i] - cs[32 j + 31]}, j < i
                 blk[idx] = (j < i) ? ex2f(cs2[32 * i] - cs2[32 * j + 31]) : 0.f;
             }
-            mbar_arrive(&vfull[buf]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&vfull[buf]);
         }
     } else if (warp >= 2 && warp < 10) {
         // ------------------------------------------------------------ mask warps
-        // Two warps per TMEM lane quarter: warp (q, half) owns rows 32 q .. 32 q + 31 of the block and
-        // the 32-column sub-tile `half` of every 64-column piece.
+        // Two warps per TMEM lane quarter: warp (q, half) owns rows 32 q .. 32 q + 31 of the block.
         const int q = warp & 3;
         const int half = (warp - 2) >> 2;
         const int rl = q * 32 + lane;              // row inside the 128-row block
@@ -258,8 +275,11 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
         const int isub = r >> 5;
         const uint32_t tlane = (uint32_t)(q * 32) << 16;
         float *vec = reinterpret_cast<float *>(smem + OFF_VEC);
-        uint32_t mcnt = 0;   // pieces of M produced so far
 
+        // The two warps of a lane quarter alternate pieces: warp (q, half) masks pieces half, half + 2, ... in
+        // full (both 32-column sub-tiles) and always fills ring slot `half`, so the per-piece hand-over costs
+        // (slot wait, stores, proxy fence, arrival) of one group overlap the other group's arithmetic.
+        uint32_t muse = 0;   // how often this warp has filled its ring slot
         for (int hi = 0; hi < nheads; ++hi) {
             float *cs2 = vec + (hi & 1) * VEC_FLOATS, *cf = cs2 + 256, *dtv = cs2 + 512, *blk = cs2 + 768;
             mbar_wait(&vfull[hi & 1], (hi >> 1) & 1, abortp, p.status);
@@ -269,65 +289,70 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                 mbar_wait(&bar_s, 0, abortp, p.status);
                 tc_fence_after_sync();
             }
-            for (int jj = 0; jj < npieces; ++jj) {
-                const int cb = colbase + jj * 64 + half * 32;   // first column of this thread's sub-tile (in chunk)
-                const int jsub = cb >> 5;
-                const bool zero = FWD ? (jsub > isub) : (jsub < isub);
-                uint32_t pk[16];
-                if (zero) {
+            for (int jj = half; jj < npieces; jj += 2) {
+                uint32_t pk[32];
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) pk[k] = 0u;
-                } else {
-                    float v[32];
-                    tmem_ld32(tm + tlane + jj * 64 + half * 32, v);
-                    if (jsub != isub) {
-                        const float f = rowf * (FWD ? blk[isub * 8 + jsub] : blk[jsub * 8 + isub]);
+                for (int sub = 0; sub < 2; ++sub) {
+                    const int cb = colbase + jj * 64 + sub * 32;    // first column of the sub-tile (in chunk)
+                    const int jsub = cb >> 5;
+                    const bool zero = FWD ? (jsub > isub) : (jsub < isub);
+                    uint32_t *pks = pk + sub * 16;
+                    if (zero) {
 #pragma unroll
-                        for (int k = 0; k < 32; k += 4) {
-                            const float4 cv = *reinterpret_cast<const float4 *>(cf + cb + k);
-                            v[k] *= cv.x * f;
-                            v[k + 1] *= cv.y * f;
-                            v[k + 2] *= cv.z * f;
-                            v[k + 3] *= cv.w * f;
-                        }
+                        for (int k = 0; k < 16; ++k) pks[k] = 0u;
                     } else {
+                        float v[32];
+                        tmem_ld32(tm + tlane + jj * 64 + sub * 32, v);
+                        if (jsub != isub) {
+                            const float f = rowf * (FWD ? blk[isub * 8 + jsub] : blk[jsub * 8 + isub]);
+                            const float2 f2 = make_float2(f, f);
 #pragma unroll
-                        for (int k = 0; k < 32; k += 4) {
-                            const float4 cc = *reinterpret_cast<const float4 *>(cs2 + cb + k);
-                            const float ccv[4] = {cc.x, cc.y, cc.z, cc.w};
-                            float dv[4] = {1.f, 1.f, 1.f, 1.f};
-                            if (FWD) {
-                                const float4 d4 = *reinterpret_cast<const float4 *>(dtv + cb + k);
-                                dv[0] = d4.x; dv[1] = d4.y; dv[2] = d4.z; dv[3] = d4.w;
+                            for (int k = 0; k < 32; k += 4) {
+                                const float4 cv = *reinterpret_cast<const float4 *>(cf + cb + k);
+                                const float2 w0 = __fmul2_rn(make_float2(v[k], v[k + 1]), __fmul2_rn(make_float2(cv.x, cv.y), f2));
+                                const float2 w1 = __fmul2_rn(make_float2(v[k + 2], v[k + 3]), __fmul2_rn(make_float2(cv.z, cv.w), f2));
+                                pks[k >> 1] = pack2(w0.x, w0.y);
+                                pks[(k >> 1) + 1] = pack2(w1.x, w1.y);
                             }
+                        } else {
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const int col = cb + k + e;
-                                const bool on = FWD ? (col <= r) : (col >= r);
-                                const float ex = FWD ? ex2f(csr - ccv[e]) * dv[e] : ex2f(ccv[e] - csr);
-                                v[k + e] = on ? v[k + e] * ex : 0.f;
+                            for (int k = 0; k < 32; k += 4) {
+                                const float4 cc = *reinterpret_cast<const float4 *>(cs2 + cb + k);
+                                const float ccv[4] = {cc.x, cc.y, cc.z, cc.w};
+                                float dv[4] = {1.f, 1.f, 1.f, 1.f};
+                                if (FWD) {
+                                    const float4 d4 = *reinterpret_cast<const float4 *>(dtv + cb + k);
+                                    dv[0] = d4.x; dv[1] = d4.y; dv[2] = d4.z; dv[3] = d4.w;
+                                }
+                                float w[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const int col = cb + k + e;
+                                    const bool on = FWD ? (col <= r) : (col >= r);
+                                    const float ex = FWD ? ex2f(csr - ccv[e]) * dv[e] : ex2f(ccv[e] - csr);
+                                    w[e] = on ? v[k + e] * ex : 0.f;
+                                }
+                                pks[k >> 1] = pack2(w[0], w[1]);
+                                pks[(k >> 1) + 1] = pack2(w[2], w[3]);
                             }
                         }
                     }
-#pragma unroll
-                    for (int k = 0; k < 16; ++k) pk[k] = pack2(v[2 * k], v[2 * k + 1]);
                 }
                 // the ring slot is free once the MMAs of the piece that last used it are done
-                const uint32_t ms = mcnt & 1;
-                if (mcnt >= 2) mbar_wait(&mempty[ms], ((mcnt >> 1) - 1) & 1, abortp, p.status);
-                ++mcnt;
-                unsigned char *mrow = smem + OFF_M + ms * 16384 + rl * 128;
+                if (muse >= 1) mbar_wait(&mempty[half], (muse - 1) & 1, abortp, p.status);
+                ++muse;
+                unsigned char *mrow = smem + OFF_M + half * 16384 + rl * 128;
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    const int chunk16 = half * 4 + ch;
-                    *reinterpret_cast<uint4 *>(mrow + ((chunk16 ^ (rl & 7)) << 4)) =
+                for (int ch = 0; ch < 8; ++ch)
+                    *reinterpret_cast<uint4 *>(mrow + ((ch ^ (rl & 7)) << 4)) =
                         make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
-                }
                 tc_fence_before_sync();
                 fence_proxy_async_smem();
-                mbar_arrive(&mfull[ms]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&mfull[half]);
             }
-            mbar_arrive(&vempty[hi & 1]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&vempty[hi & 1]);
         }
     } else if (warp >= 11) {
         // ------------------------------------------------------------ epilogue warps (one per TMEM lane quarter)
@@ -346,7 +371,8 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             const float csr = cs2[r];
             const float offs = FWD ? ex2f(csr) : ex2f(cs2[255] - csr);
             const float dtr = dtv[r];
-            mbar_arrive(&vempty[buf]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&vempty[buf]);
             const float Dh = __ldg(p.D + h);
             mbar_wait(&xfull[xs], xuse & 1, abortp, p.status);
             if (!FWD) mbar_wait(&xrfull, hi & 1, abortp, p.status);
@@ -390,11 +416,11 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                 }
             }
             tc_fence_before_sync();
-            mbar_arrive(&accempty[buf]);
-            if (!FWD) mbar_arrive(&xrempty);
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
+                mbar_arrive(&accempty[buf]);
+                if (!FWD) mbar_arrive(&xrempty);
                 tma_store_3d(&tmOut, blockbase, h * 64, tok0 + rb * 128 + q * 32, b);
                 tma_store_commit();
                 tma_store_wait_read();              // the store has read the block: the stage may be refilled
