@@ -24,6 +24,8 @@
 // The accumulator stays in TMEM across all heads of the CTA: the head sum costs nothing, and there
 // is no per-head epilogue.  It is written once, as an fp32 partial slice; a later kernel adds the
 // slices of a group in a fixed order.
+#include <type_traits>
+
 #include "ssd_internal.h"
 #include "ssd_sm100.cuh"
 
@@ -161,8 +163,6 @@ k_grad_bc_tc(SegParams p, const __grid_constant__ CUtensorMap tmRow,   // DC: dy
             const uint32_t idCB = umma_idesc_bf16(128, (uint32_t)ncols, false, false);
             const uint32_t idS = umma_idesc_bf16(128, 128, false, false);   // rows (K-major) x 128 cols (K-major)
             const uint32_t idW = umma_idesc_bf16(128, 128, false, true);    // W / scaled rows (K-major) x V / state (MN-major)
-            uint32_t job = 0, acc_on = 0;
-
             // CB tile, once
             mbar_wait(&bar_ld, 0, abortp, p.status);
             tc_fence_after_sync();
@@ -172,65 +172,94 @@ k_grad_bc_tc(SegParams p, const __grid_constant__ CUtensorMap tmRow,   // DC: dy
                           umma_desc_sw128(sV + (kk >> 2) * (ncols * 128) + (kk & 3) * 32, 16, 1024), idCB, kk ? 1u : 0u);
             umma_commit(&bar_cb);
 
-            // scores of unit u of head hi into the S buffer (128 columns = one N = 128 product, K = P)
-            auto issue_scores = [&](int hi, int u) {
-                const int rbuf = hi & 1, cbuf = hi % ncb, cuse = hi / ncb;
-                if (u == 0) {
-                    mbar_wait(&rfull[rbuf], (hi >> 1) & 1, abortp, p.status);
-                    mbar_wait(&cfull[cbuf], cuse & 1, abortp, p.status);
-                    tc_fence_after_sync();
-                }
-                const uint32_t a = sR + rbuf * 16384, bc = sC + cbuf * 16384 + u * 16384;
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    umma_bf16(tm + TM_S, umma_desc_sw128(a + k * 32, 16, 1024), umma_desc_sw128(bc + k * 32, 16, 1024),
-                              idS, k ? 1u : 0u);
-                umma_commit(&sfull);
-                if (u == nunits - 1) umma_commit(&cempty[cbuf]);
-            };
+            // Descriptors as (low word, high word): inside the unrolled loops every operand address is the low
+            // word plus a compile-time constant (16-byte units), so an MMA costs the issuing thread an add or two.
+            const uint64_t dR = umma_desc_sw128(sR, 16, 1024), dC = umma_desc_sw128(sC, 16, 1024);
+            const uint64_t dMm = umma_desc_sw128(sM, 16, 1024), dSt = umma_desc_sw128(sSt, 8192, 1024);
+            const uint64_t dV = umma_desc_sw128(sV, (uint32_t)ncols * 128u, 1024);
+            const uint32_t loR = (uint32_t)dR, hiR = (uint32_t)(dR >> 32), loC = (uint32_t)dC, hiC = (uint32_t)(dC >> 32);
+            const uint32_t loM = (uint32_t)dMm, hiM = (uint32_t)(dMm >> 32), loSt = (uint32_t)dSt, hiSt = (uint32_t)(dSt >> 32);
+            const uint32_t loV = (uint32_t)dV, hiV = (uint32_t)(dV >> 32);
 
-            issue_scores(0, 0);
-            uint32_t sidx = 0;   // index of the score unit the mask warps are working on
-            for (int hi = 0; hi < nheads; ++hi) {
-                for (int u = 0; u < nunits; ++u) {
-                    // next score unit as soon as the mask warps have copied the current one out of TMEM
-                    const bool last_u = (u == nunits - 1);
-                    if (!last_u || hi + 1 < nheads) {
-                        mbar_wait(&sempty, sidx & 1, abortp, p.status);
+            auto run = [&](auto nu_c) {
+                constexpr int NU = decltype(nu_c)::value;      // score units per head: 1 or 2
+                constexpr int NCB = (NU == 1) ? 2 : 1;         // column-operand buffers
+                // scores of unit u of head hi into the S buffer (128 columns = one N = 128 product, K = P)
+                auto issue_scores = [&](int hi, int u, uint32_t lo_r, uint32_t lo_c) {
+                    if (u == 0) {
+                        const int rbuf = hi & 1, cbuf = (NCB == 2) ? (hi & 1) : 0, cuse = (NCB == 2) ? (hi >> 1) : hi;
+                        mbar_wait(&rfull[rbuf], (hi >> 1) & 1, abortp, p.status);
+                        mbar_wait(&cfull[cbuf], cuse & 1, abortp, p.status);
                         tc_fence_after_sync();
-                        if (!last_u) issue_scores(hi, u + 1);
-                        else issue_scores(hi + 1, 0);
                     }
-                    ++sidx;
-                    const uint32_t mb = job & 1;
-                    mbar_wait(&mfull[mb], (job >> 1) & 1, abortp, p.status);
-                    tc_fence_after_sync();
+                    umma_bf16_fixed<false>(tm + TM_S, umma_desc_words(lo_r, hiR), umma_desc_words(lo_c, hiC), idS);
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        umma_bf16(tm + TM_ACC, umma_desc_sw128(sM + mb * 32768 + (k >> 2) * 16384 + (k & 3) * 32, 16, 1024),
-                                  umma_desc_sw128(sV + (u * 128 + k * 16) * 128, (uint32_t)ncols * 128u, 1024), idW,
-                                  acc_on);
-                        acc_on = 1u;
+                    for (int k = 1; k < 4; ++k)
+                        umma_bf16_fixed<true>(tm + TM_S, umma_desc_words(lo_r + k * 2, hiR), umma_desc_words(lo_c + k * 2, hiC), idS);
+                    umma_commit(&sfull);
+                };
+                uint32_t sidx = 0;   // index of the score unit the mask warps are working on
+                uint32_t job = 0;    // M buffers consumed so far
+                issue_scores(0, 0, loR, loC);
+                if (NU == 1) umma_commit(&cempty[0]);
+                for (int hi = 0; hi < nheads; ++hi) {
+                    const int rbuf = hi & 1, cbuf = (NCB == 2) ? (hi & 1) : 0;
+                    const uint32_t lo_r = loR + rbuf * 1024, lo_c = loC + cbuf * 1024;
+                    const int nrbuf = (hi + 1) & 1, ncbuf = (NCB == 2) ? ((hi + 1) & 1) : 0;
+#pragma unroll
+                    for (int u = 0; u < NU; ++u) {
+                        // next score unit as soon as the mask warps have copied the current one out of TMEM
+                        const bool last_u = (u == NU - 1);
+                        if (!last_u || hi + 1 < nheads) {
+                            mbar_wait(&sempty, sidx & 1, abortp, p.status);
+                            tc_fence_after_sync();
+                            if (!last_u) {
+                                issue_scores(hi, u + 1, lo_r, lo_c + (u + 1) * 1024);
+                                if (u + 1 == NU - 1) umma_commit(&cempty[cbuf]);
+                            } else {
+                                issue_scores(hi + 1, 0, loR + nrbuf * 1024, loC + ncbuf * 1024);
+                                if (NU == 1) umma_commit(&cempty[ncbuf]);
+                            }
+                        }
+                        ++sidx;
+                        const uint32_t mb = job & 1;
+                        mbar_wait(&mfull[mb], (job >> 1) & 1, abortp, p.status);
+                        tc_fence_after_sync();
+                        const uint32_t lo_m = loM + mb * 2048, lo_v = loV + u * 1024;   // 32 KB buffers; 128 rows of V
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            const uint64_t ad = umma_desc_words(lo_m + (k >> 2) * 1024 + (k & 3) * 2, hiM);
+                            const uint64_t bd = umma_desc_words(lo_v + k * 128, hiV);
+                            if (u == 0 && k == 0) {
+                                if (hi == 0) umma_bf16_fixed<false>(tm + TM_ACC, ad, bd, idW);
+                                else umma_bf16_fixed<true>(tm + TM_ACC, ad, bd, idW);
+                            } else {
+                                umma_bf16_fixed<true>(tm + TM_ACC, ad, bd, idW);
+                            }
+                        }
+                        umma_commit(&mempty[mb]);
+                        ++job;
                     }
-                    umma_commit(&mempty[mb]);
-                    ++job;
-                }
-                {   // inter-chunk piece: (scaled rows) [128 x 64] x state [64 x 128]
-                    const uint32_t mb = job & 1;
-                    mbar_wait(&stfull, hi & 1, abortp, p.status);
-                    mbar_wait(&mfull[mb], (job >> 1) & 1, abortp, p.status);
-                    tc_fence_after_sync();
+                    {   // inter-chunk piece: (scaled rows) [128 x 64] x state [64 x 128]
+                        const uint32_t mb = job & 1;
+                        mbar_wait(&stfull, hi & 1, abortp, p.status);
+                        mbar_wait(&mfull[mb], (job >> 1) & 1, abortp, p.status);
+                        tc_fence_after_sync();
+                        const uint32_t lo_m = loM + mb * 2048;
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        umma_bf16(tm + TM_ACC, umma_desc_sw128(sM + mb * 32768 + k * 32, 16, 1024),
-                                  umma_desc_sw128(sSt + k * 2048, 8192, 1024), idW, 1u);
-                    umma_commit(&mempty[mb]);
-                    umma_commit(&stempty);
-                    umma_commit(&rempty[hi & 1]);
-                    ++job;
+                        for (int k = 0; k < 4; ++k)
+                            umma_bf16_fixed<true>(tm + TM_ACC, umma_desc_words(lo_m + k * 2, hiM),
+                                                  umma_desc_words(loSt + k * 128, hiSt), idW);
+                        umma_commit(&mempty[mb]);
+                        umma_commit(&stempty);
+                        umma_commit(&rempty[hi & 1]);
+                        ++job;
+                    }
                 }
-            }
-            umma_commit(&accfull);
+                umma_commit(&accfull);
+            };
+            if (nunits == 2) run(std::integral_constant<int, 2>{});
+            else run(std::integral_constant<int, 1>{});
         }
     } else if (warp == 18) {
         // ------------------------------------------------------------ vector warp
