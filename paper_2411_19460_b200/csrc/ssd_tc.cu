@@ -183,6 +183,12 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
     tc_fence_after_sync();
     const uint32_t tm = tmem_base;
     const uint32_t idesc = umma_idesc_bf16(128, 128, true, true);
+    // operand descriptors as (low word, high word); the issue loops below add compile-time constants
+    // (16-byte units) to the low word only
+    const uint64_t dXa = umma_desc_sw128(smem_u32(smem), 16384, 1024), dVb = umma_desc_sw128(smem_u32(smem + 32768), 16384, 1024);
+    const uint64_t dCk = umma_desc_sw128(smem_u32(smem + 32768), 16, 1024), dHk = umma_desc_sw128(smem_u32(smem + CS_STAGE), 16, 1024);
+    const uint32_t loXa = (uint32_t)dXa, hiXa = (uint32_t)(dXa >> 32), loVb = (uint32_t)dVb, hiVb = (uint32_t)(dVb >> 32);
+    const uint32_t loCk = (uint32_t)dCk, hiCk = (uint32_t)(dCk >> 32), loHk = (uint32_t)dHk, hiHk = (uint32_t)(dHk >> 32);
 
     for (int half = 0; half < 2; ++half) {
         mbar_wait(&bar_ld, half, &abort_flag, p.status);
@@ -204,11 +210,11 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
         __syncthreads();
         if (tid == 0) {
             tc_fence_after_sync();
-            const uint32_t sa = smem_u32(smem), sb = smem_u32(smem + 32768);
+            if (half == 0) umma_bf16_fixed<false>(tm, dXa, dVb, idesc);
+            else umma_bf16_fixed<true>(tm, dXa, dVb, idesc);
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
-                umma_bf16(tm, umma_desc_sw128(sa + ks * 2048, 16384, 1024), umma_desc_sw128(sb + ks * 2048, 16384, 1024),
-                          idesc, (half | ks) ? 1u : 0u);
+            for (int ks = 1; ks < 8; ++ks)
+                umma_bf16_fixed<true>(tm, umma_desc_words(loXa + ks * 128, hiXa), umma_desc_words(loVb + ks * 128, hiVb), idesc);
             if (dstate) {
                 // Yoff[t, p] = sum_n C[t, n] H_in[p, n] for the 128 time rows of this half, per head
                 if (half == 0) {
@@ -216,12 +222,15 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
                     tc_fence_after_sync();
                 }
                 const uint32_t idy = umma_idesc_bf16(128, 64, false, false);
-                for (int hh = 0; hh < 2; ++hh) {
-                    const uint32_t sh = smem_u32(smem + CS_STAGE + hh * 16384);
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        umma_bf16(tm + 128 + hh * 64, umma_desc_sw128(sb + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024),
-                                  umma_desc_sw128(sh + (kk >> 2) * 8192 + (kk & 3) * 32, 16, 1024), idy, kk ? 1u : 0u);
+                for (int hh = 0; hh < 2; ++hh) {
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const uint64_t ad = umma_desc_words(loCk + (kk >> 2) * 1024 + (kk & 3) * 2, hiCk);
+                        const uint64_t bd = umma_desc_words(loHk + hh * 1024 + (kk >> 2) * 512 + (kk & 3) * 2, hiHk);
+                        if (kk == 0) umma_bf16_fixed<false>(tm + 128 + hh * 64, ad, bd, idy);
+                        else umma_bf16_fixed<true>(tm + 128 + hh * 64, ad, bd, idy);
+                    }
                 }
             }
             umma_commit(&bar_mma);
