@@ -19,6 +19,7 @@ import statistics
 import subprocess
 import sys
 import tempfile
+import threading
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -92,11 +93,12 @@ def load_peaks():
 # to the timed workload by tokens x heads per launch (the traffic of these kernels grows in proportion).
 NCU_TRAFFIC_CFG1 = {
     # kernel kind: (bytes per launch, source file, sha256 of that file at capture time)
-    "bwd_dB": (17.22e6, "ssd_tc_bc.cu", "800395a98e29fa540b7f78cc9bd182ba6d9e044247f9fdbe3071ce2aa2e6c65e"),
-    "bwd_dC": (17.22e6, "ssd_tc_bc.cu", "800395a98e29fa540b7f78cc9bd182ba6d9e044247f9fdbe3071ce2aa2e6c65e"),
-    "bwd_dx": (17.22e6, "ssd_tc_scan.cu", "8c6e27020dadacba65067e5da6ee0d4454197329a58427ad979106ad1b61fb80"),
-    "chunk_state": (7.24e6, "ssd_tc.cu", "08ba9e297121e0bc3fe4bd835ce929e0578a9936620712ece7868ec0a7d6f316"),
-    "dstate_contrib": (7.24e6, "ssd_tc.cu", "08ba9e297121e0bc3fe4bd835ce929e0578a9936620712ece7868ec0a7d6f316"),
+    "bwd_dB": (17.23e6, "ssd_tc_bc.cu", "fa854348829bce649cc73d8e7c4852617f169d2b33dfc0b084ac08bddfa77ea2"),
+    "bwd_dC": (17.23e6, "ssd_tc_bc.cu", "fa854348829bce649cc73d8e7c4852617f169d2b33dfc0b084ac08bddfa77ea2"),
+    "bwd_dx": (17.24e6, "ssd_tc_scan.cu", "f9a69e821a37dbde6084db649db63a7c352b2be6226441be1a457ad7026a6f3b"),
+    "chunk_scan_fwd": (10.94e6, "ssd_tc_scan.cu", "f9a69e821a37dbde6084db649db63a7c352b2be6226441be1a457ad7026a6f3b"),
+    "chunk_state": (7.04e6, "ssd_tc.cu", "d08b62291f529092a782772fee2f8222d1a35a5f326c2cc1ac015e6d3ffe95a6"),
+    "dstate_contrib": (7.04e6, "ssd_tc.cu", "d08b62291f529092a782772fee2f8222d1a35a5f326c2cc1ac015e6d3ffe95a6"),
 }
 NCU_CFG1_UNITS = 2048 * 24
 
@@ -119,17 +121,55 @@ def ncu_traffic(kind, tokens_per_launch, heads):
 
 # ----------------------------------------------------------------------------- clocks sampling
 class ClockSampler:
+    """SM clock and clock-event reasons sampled DURING the timed region: an NVML polling thread (a sample
+    every few milliseconds, the first one at once), falling back to `nvidia-smi -lms` when NVML's Python
+    binding is missing.  Read-only: nothing about the GPU is changed."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    REASON_BITS = (("sw_power_cap", 0x4), ("hw_slowdown", 0x8), ("sw_thermal_slowdown", 0x20),
+                   ("hw_thermal_slowdown", 0x40))
 
-    def __init__(self, device):
+    def __init__(self, device, period_s=0.002):
         self.proc = None
         self.path = None
+        self.thread = None
+        self.sm, self.mx, self.reasons = [], [], set()
+        self._stop = threading.Event()
         try:
             uuid = str(torch.cuda.get_device_properties(device).uuid)
             if not uuid.startswith("GPU-"):
                 uuid = "GPU-" + uuid
+        except Exception:
+            return
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            handle = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if hasattr(uuid, "encode") else uuid)
+            mx = float(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM))
+            get_reasons = getattr(pynvml, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                getattr(pynvml, "nvmlDeviceGetCurrentClocksThrottleReasons")
+
+            def poll():
+                while True:
+                    try:
+                        self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(handle, pynvml.NVML_CLOCK_SM)))
+                        self.mx.append(mx)
+                        bits = int(get_reasons(handle))
+                        for name, bit in self.REASON_BITS:
+                            if bits & bit:
+                                self.reasons.add(name)
+                    except Exception:
+                        pass
+                    if self._stop.wait(period_s):
+                        return
+
+            self.thread = threading.Thread(target=poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.thread = None
+        try:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(
@@ -141,6 +181,14 @@ class ClockSampler:
 
     def stop(self):
         out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        if self.thread is not None:
+            self._stop.set()
+            self.thread.join(timeout=2)
+            if self.sm:
+                out.update(sm_mhz=statistics.median(self.sm), sm_max_mhz=max(self.mx), samples=len(self.sm),
+                           source="nvml")
+            out["reasons"] = sorted(self.reasons)
+            return out
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -167,7 +215,7 @@ class ClockSampler:
         except Exception:
             pass
         if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm), source="nvidia-smi")
         out["reasons"] = sorted(reasons)
         return out
 
