@@ -38,7 +38,7 @@ using namespace sm100;
 
 namespace {
 
-constexpr int SC_THREADS = 480;           // warp 0 producer, 1 MMA, 2..9 mask, 10 vectors, 11..14 epilogue
+constexpr int SC_THREADS = 736;           // warp 0 producer, 1 MMA, 2..17 mask, 18 vectors, 19..22 epilogue
 constexpr uint32_t OFF_ROWS = 0;          // 32 KB  [n-half][128 rows][128 B]
 constexpr uint32_t OFF_X = 32768;         // 3 x 32 KB value stages; first the score-columns operand (<= 64 KB)
 constexpr uint32_t OFF_M = 131072;        // 2 x 16 KB ring of masked pieces
@@ -114,12 +114,12 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
         for (int i = 0; i < 2; ++i) {
             mbar_init(&hfull[i], 1);
             mbar_init(&hempty[i], 1);
-            mbar_init(&mfull[i], 4);           // one arrival per warp (lane 0, after __syncwarp()) of the slot's four
+            mbar_init(&mfull[i], 8);           // one arrival per warp (lane 0, after __syncwarp()) of the slot's eight
             mbar_init(&mempty[i], 1);
             mbar_init(&accfull[i], 1);
             mbar_init(&accempty[i], 4);
             mbar_init(&vfull[i], 1);
-            mbar_init(&vempty[i], 8 + 4);
+            mbar_init(&vempty[i], 16 + 4);
         }
         mbar_init(&xrfull, 1);
         mbar_init(&xrempty, 4);
@@ -228,7 +228,7 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             if (npieces == 4) run(std::integral_constant<int, 4>{});
             else run(std::integral_constant<int, 2>{});
         }
-    } else if (warp == 10) {
+    } else if (warp == 18) {
         // ------------------------------------------------------------ vector warp
         // Per head: the 256 cumulative sums (log2 units) and step sizes of the chunk, the column factor
         // of the mask factorisation and the 8 x 8 table of sub-tile-to-sub-tile decays, written to a
@@ -265,20 +265,21 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             __syncwarp();
             if (lane == 0) mbar_arrive(&vfull[buf]);
         }
-    } else if (warp >= 2 && warp < 10) {
+    } else if (warp >= 2 && warp < 18) {
         // ------------------------------------------------------------ mask warps
         // Two warps per TMEM lane quarter: warp (q, half) owns rows 32 q .. 32 q + 31 of the block.
         const int q = warp & 3;
-        const int half = (warp - 2) >> 2;
+        const int half = (warp - 2) >> 3;          // which pieces (and ring slot) this warp's group takes
+        const int sub = ((warp - 2) >> 2) & 1;     // which 32-column sub-tile of those pieces
         const int rl = q * 32 + lane;              // row inside the 128-row block
         const int r = rb * 128 + rl;               // row inside the chunk
         const int isub = r >> 5;
         const uint32_t tlane = (uint32_t)(q * 32) << 16;
         float *vec = reinterpret_cast<float *>(smem + OFF_VEC);
 
-        // The two warps of a lane quarter alternate pieces: warp (q, half) masks pieces half, half + 2, ... in
-        // full (both 32-column sub-tiles) and always fills ring slot `half`, so the per-piece hand-over costs
-        // (slot wait, stores, proxy fence, arrival) of one group overlap the other group's arithmetic.
+        // Four warps per lane quarter in two groups that alternate pieces: group `half` masks pieces half,
+        // half + 2, ... (one 32-column sub-tile per warp) and always fills ring slot `half`, so the per-piece
+        // hand-over costs (slot wait, stores, proxy fence, arrival) of one group overlap the other's arithmetic.
         uint32_t muse = 0;   // how often this warp has filled its ring slot
         for (int hi = 0; hi < nheads; ++hi) {
             float *cs2 = vec + (hi & 1) * VEC_FLOATS, *cf = cs2 + 256, *dtv = cs2 + 512, *blk = cs2 + 768;
@@ -290,13 +291,11 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                 tc_fence_after_sync();
             }
             for (int jj = half; jj < npieces; jj += 2) {
-                uint32_t pk[32];
-#pragma unroll
-                for (int sub = 0; sub < 2; ++sub) {
+                uint32_t pks[16];
+                {
                     const int cb = colbase + jj * 64 + sub * 32;    // first column of the sub-tile (in chunk)
                     const int jsub = cb >> 5;
                     const bool zero = FWD ? (jsub > isub) : (jsub < isub);
-                    uint32_t *pks = pk + sub * 16;
                     if (zero) {
 #pragma unroll
                         for (int k = 0; k < 16; ++k) pks[k] = 0u;
@@ -343,9 +342,9 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                 ++muse;
                 unsigned char *mrow = smem + OFF_M + half * 16384 + rl * 128;
 #pragma unroll
-                for (int ch = 0; ch < 8; ++ch)
-                    *reinterpret_cast<uint4 *>(mrow + ((ch ^ (rl & 7)) << 4)) =
-                        make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+                for (int ch = 0; ch < 4; ++ch)
+                    *reinterpret_cast<uint4 *>(mrow + (((sub * 4 + ch) ^ (rl & 7)) << 4)) =
+                        make_uint4(pks[4 * ch], pks[4 * ch + 1], pks[4 * ch + 2], pks[4 * ch + 3]);
                 tc_fence_before_sync();
                 fence_proxy_async_smem();
                 __syncwarp();
@@ -354,7 +353,7 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             __syncwarp();
             if (lane == 0) mbar_arrive(&vempty[hi & 1]);
         }
-    } else if (warp >= 11) {
+    } else if (warp >= 19) {
         // ------------------------------------------------------------ epilogue warps (one per TMEM lane quarter)
         // x (and dy) come from the tiles TMA already brought to shared memory; the output overwrites the
         // rows just read, in place (the MMAs of the head are done with the stage), and leaves by one TMA
