@@ -8,6 +8,12 @@
 // All of it is Eq. 1 of the paper regrouped by chunks; the segment hand-off is Algorithms 1 and 2.
 #include "ssd_internal.h"
 
+#ifndef SP_BWD_CTAS
+#define SP_BWD_CTAS 5
+#define SP_BWD_PF 4
+#define SP_FWD_CTAS 5
+#define SP_FWD_PF 4
+#endif
 namespace ssd {
 
 // ------------------------------------------------------------------ small helpers
@@ -154,7 +160,7 @@ cudaError_t launch_chunk_state_simt(const SegParams &p, int dtype, int mode, cud
 // bits do not depend on how the sequence is cut into segments.  Each thread owns one float4.
 // Also stores the segment-entry state into `boundary` (the sequence-axis checkpoint) and hands the
 // segment-exit state to the next segment through hcarry.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, SP_FWD_CTAS)
 k_state_pass_fwd(SegParams p, const float *init, long long init_bs, float *boundary_out,
                  long long bnd_bs, float *final_out, int want_bf16) {
     const int h = blockIdx.y, b = blockIdx.z;
@@ -182,7 +188,7 @@ k_state_pass_fwd(SegParams p, const float *init, long long init_bs, float *bound
     put(slot_off(p, b, 0, h) + e, carry);
     // The chunk sums and decays do not depend on the carry: fetch eight chunks ahead of the serial
     // recurrence, so that a segment costs a few memory latencies instead of one per chunk.
-    constexpr int PF = 8;
+    constexpr int PF = SP_FWD_PF;
     for (int c0 = 1; c0 <= p.nc; c0 += PF) {
         float4 sv[PF];
         float dec[PF];
@@ -220,9 +226,9 @@ cudaError_t launch_state_pass_fwd(const SegParams &p, const float *init, long lo
 // Gslot[c] = exp(cs_last,c) Gslot[c+1] + E_c.  Gslot[c+1] is Gout of chunk c.  Also emits, per chunk,
 // the partial sums of exp(cs_last,c) <Gout_c, H_in,c> (one per CTA, summed later in a fixed order):
 // the part of da_t that couples the gradient from the right with the state from the left.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, SP_BWD_CTAS)
 k_state_pass_bwd(SegParams p, const float *init, float *left_out, int want_bf16) {
-    __shared__ float red[8][8];
+    __shared__ float red[SP_BWD_PF][8];
     const int h = blockIdx.y, b = blockIdx.z;
     const int PN = p.P * p.N;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -245,7 +251,7 @@ k_state_pass_bwd(SegParams p, const float *init, float *left_out, int want_bf16)
     put(slot_off(p, b, p.nc, h) + e, carry);
     // Eight chunks at a time: their E_c, entry states and decays are fetched ahead of the serial
     // recurrence; the eight <Gout, H_in> partials of a batch share one block-wide reduction step.
-    constexpr int PF = 8;
+    constexpr int PF = SP_BWD_PF;
     for (int c0 = p.nc - 1; c0 >= 0; c0 -= PF) {
         float4 ev[PF], hv[PF];
         float dec[PF];
