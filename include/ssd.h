@@ -56,6 +56,9 @@ enum {
     SSD_FLAG_FORCE_SIMT = 1,       /* bf16 I/O: use the CUDA-core kernels instead of the tensor-core ones */
     SSD_FLAG_ACCUM_PARAM_GRADS = 2,/* ssd_bwd_segmented: dA and dD are added to, not overwritten (a driver that
                                       back-propagates one grid cell at a time sums them over the cells) */
+    SSD_FLAG_SPLIT_BC = 8,         /* ssd_bwd_segmented, tensor-core path: dB and dC by two kernels that each mask the
+                                      score tiles themselves, instead of the one that masks them once for both (a
+                                      cross-check; the same values up to the order of the fp32 head sums) */
     SSD_FLAG_SERIAL = 4            /* ssd_bwd_segmented: launch every kernel on `stream` itself, in order.  By default
                                       the tensor-core path runs its three mutually independent gradient kernels of a
                                       segment on two library-owned helper streams forked off `stream` and joined back

@@ -45,12 +45,12 @@ static void prof_end(ProfEvent *ev, cudaStream_t st) {
 
 struct Layout {
     size_t status, cs, dtT, Hst, Hbf, hcarry, Gst, Gbf, gcarry, ghdot, ddt_dir, rho, rho2, psi, psi2, pB, pC, dAp, dDp;
-    size_t dtT_b, rho2_b, ghdot_b;   // second copies: a segment's finishing kernels overlap the next segment's first ones
+    size_t dtT_b, rho2_b, ghdot_b, rhob, psib;   // second copies: a segment's finishing kernels overlap the next segment's first ones
     size_t total;
 };
 
 struct Plan {
-    int B, L, H, P, N, G, Q, seg, nseg, ncs, nct, hpg, nsl, dtype;
+    int B, L, H, P, N, G, Q, seg, nseg, ncs, nct, hpg, nsl, nslf, dtype;
     bool use_tc;
     int64_t x_bs, dt_bs, bc_bs;
     size_t esz;
@@ -96,6 +96,24 @@ static int best_head_split(int nchunks, int groups, int batch, int hpg, int max_
     return best;
 }
 
+// Head ranges per group for the fused dB/dC kernel, whose CTAs are (chunk, one of the three causal 128 x 128
+// tiles, head range), all of about the same cost: whole waves of 148 CTAs times (one head-time of set-up plus
+// the heads of a range), for a reference launch of 16 chunks.  A function of H and G only, so the summation
+// order of dB/dC does not depend on the segment length.
+static int fused_head_split(int groups, int hpg) {
+    int best = 1;
+    long best_t = -1;
+    const int max_split = hpg >= 4 ? hpg / 4 : 1;
+    for (int ns = 1; ns <= max_split; ++ns) {
+        const int hps = (hpg + ns - 1) / ns;
+        if ((hpg + hps - 1) / hps != ns) continue;
+        const long ctas = 16L * 3 * groups * ns;
+        const long t = ((ctas + 147) / 148) * (1 + hps);
+        if (best_t < 0 || t < best_t) { best_t = t; best = ns; }
+    }
+    return best;
+}
+
 static int make_plan(const ssd_shape_t *s, Plan &pl) {
     if (!s) return SSD_EINVAL;
     if (s->B <= 0 || s->L <= 0 || s->H <= 0 || s->P <= 0 || s->N <= 0 || s->G <= 0 || s->chunk <= 0 ||
@@ -134,8 +152,10 @@ static int make_plan(const ssd_shape_t *s, Plan &pl) {
     // of dB/dC, is the same for every segment length.
     if (pl.use_tc) {
         pl.nsl = best_head_split(16, pl.G, 1, pl.hpg, pl.hpg >= 4 ? pl.hpg / 4 : 1);
+        pl.nslf = fused_head_split(pl.G, pl.hpg);
     } else {
         pl.nsl = pl.hpg;
+        pl.nslf = 0;
     }
     return SSD_OK;
 }
@@ -164,7 +184,8 @@ static void make_layout(const Plan &pl, int op, Layout &lo) {
         lo.rho2 = take(pl.use_tc ? vec : 0);
         lo.psi = take(vec);
         lo.psi2 = take(vec);
-        const size_t part = (size_t)pl.B * pl.seg * pl.G * pl.nsl * pl.N * sizeof(float);
+        const int slots = (2 * pl.nslf > pl.nsl) ? 2 * pl.nslf : pl.nsl;   // fused kernel: two slots per head range
+        const size_t part = (size_t)pl.B * pl.seg * pl.G * slots * pl.N * sizeof(float);
         lo.pB = take(part);
         lo.pC = take(part);
         lo.dAp = take(BH * pl.nct * sizeof(float));
@@ -172,6 +193,8 @@ static void make_layout(const Plan &pl, int op, Layout &lo) {
         lo.dtT_b = take(pl.use_tc ? vec : 0);
         lo.rho2_b = take(pl.use_tc ? vec : 0);
         lo.ghdot_b = take(pl.use_tc ? BH * pl.ncs * 8 * sizeof(float) : 0);
+        lo.rhob = take(pl.use_tc ? vec : 0);
+        lo.psib = take(pl.use_tc ? vec : 0);
     }
     lo.total = o;
 }
@@ -443,6 +466,13 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
     // three do not depend on one another.  Unless told otherwise they run on side streams forked off the
     // caller's stream and joined back before the segment's finishing kernels, so that one kernel's tail
     // (its last, partly idle wave) is filled by the next one's CTAs.
+    const bool fused_bc = pl.use_tc && !(shape->flags & SSD_FLAG_SPLIT_BC);
+    if (fused_bc) {
+        sp.nsl = pl.nslf;
+        sp.bc_fused = 1;
+        sp.rhob = (float *)((char *)ws + lo.rhob);
+        sp.psib = (float *)((char *)ws + lo.psib);
+    }
     SideStreams *side = nullptr;
     if (pl.use_tc && !(shape->flags & SSD_FLAG_SERIAL) && !g_prof_on) {
         side = side_streams();
@@ -469,7 +499,7 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
         }
         SSD_LAUNCH(KIND_STATE_PASS_FWD, launch_state_pass_fwd(sp, boundary + (size_t)k * pl.H * PN, (long long)pl.nseg * pl.H * PN,
                                       nullptr, 0, nullptr, pl.use_tc, st));
-        if (side) {
+        if (side && !fused_bc) {
             SSD_TRY(cudaEventRecord(side->fork[0], st));
             SSD_TRY(cudaStreamWaitEvent(side->s[0], side->fork[0], 0));
             if (tail_pending) SSD_TRY(cudaStreamWaitEvent(side->s[0], side->tail_done, 0));
@@ -495,15 +525,18 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
             }
             {
                 cudaStream_t st = side->s[1];
-                SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_tc(sp, maps, GB_DB, st));
+                if (fused_bc) SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_fused(sp, maps, st));
+                else SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_tc(sp, maps, GB_DB, st));
                 SSD_TRY(cudaEventRecord(side->join[1], st));
             }
         }
         if (pl.use_tc) SSD_LAUNCH(KIND_BWD_DX, launch_scan_tc(sp, maps, SC_DX, st));
         else SSD_LAUNCH(KIND_BWD_DX, launch_masked_product_simt(sp, pl.dtype, MP_BWD_DX, st));
         if (side) {
-            SSD_TRY(cudaStreamWaitEvent(st, side->join[0], 0));
+            if (!fused_bc) SSD_TRY(cudaStreamWaitEvent(st, side->join[0], 0));
             SSD_TRY(cudaStreamWaitEvent(st, side->join[1], 0));
+        } else if (fused_bc) {
+            SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_fused(sp, maps, st));
         } else if (pl.use_tc) {
             SSD_LAUNCH(KIND_BWD_DC, launch_grad_bc_tc(sp, maps, GB_DC, st));
             SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_tc(sp, maps, GB_DB, st));

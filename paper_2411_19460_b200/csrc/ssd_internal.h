@@ -19,6 +19,7 @@ struct SegParams {
     int ncs;       // chunk capacity of the workspace (chunks of a full segment)
     int nct;       // chunks in the whole sequence (L / Q)
     int nsl;       // head slices per group in the dB/dC partial buffers
+    int bc_fused;  // 1: the fused dB/dC kernel wrote them: two slots per slice (see ssd_tc_bcf.cu), second parts of rho/psi
     int ndd;          // partial sums of dD per (head, chunk) that the kernels of this path write (<= 16)
     int nsplit_scan;  // head ranges per group in the tensor-core scan kernels (no effect on results)
     int64_t x_bs, dt_bs, bc_bs;  // batch strides, elements
@@ -43,6 +44,7 @@ struct SegParams {
     float *ddt_dir;        // [B,H,ncs,Q]   direct part of ddt
     float *rho;            // [B,H,ncs,Q]   C_t . dC_t of this head (CUDA-core path: all of it; tensor-core
                            //               path: its intra-chunk part)
+    float *rhob, *psib;    // [B,H,ncs,Q]   fused dB/dC kernel: second parts of rho / psi (else NULL)
     float *rho2;           // [B,H,ncs,Q]   tensor-core path: C_t . (inter-chunk part of this head's dC_t); else NULL
     float *psi;            // [B,H,ncs,Q]   B_t . (intra-chunk part of this head's dB_t)
     float *psi2;           // [B,H,ncs,Q]   B_t . (inter-chunk part of this head's dB_t)
@@ -94,6 +96,8 @@ enum { SC_FWD = 0, SC_DX = 1 };
 // ssd_tc_bc.cu : per-slice partial dC, rho (GB_DC) or partial dB, psi, psi2 (GB_DB)
 cudaError_t launch_grad_bc_tc(const SegParams &p, const TcMaps &m, int mode, cudaStream_t st);
 enum { GB_DC = 0, GB_DB = 1 };
+// ssd_tc_bcf.cu : dB and dC from one masked tile (partial slices, rho, psi and their second parts)
+cudaError_t launch_grad_bc_fused(const SegParams &p, const TcMaps &m, cudaStream_t st);
 
 enum { STATE_MODE_FWD = 0, STATE_MODE_DSTATE = 1 };
 // kernel kinds, for the launch counter and the optional per-kind timing

@@ -622,7 +622,9 @@ __global__ void __launch_bounds__(128) k_bwd_finish(SegParams p) {
         if (j < per) {
             dtv[j] = p.dtT[vo + j];
             dd[j] = p.ddt_dir[vo + j];
-            run += (p.rho[vo + j] - p.psi[vo + j]) + (p.rho2 ? p.rho2[vo + j] : 0.f);
+            const float rh = p.rhob ? p.rho[vo + j] + p.rhob[vo + j] : p.rho[vo + j];
+            const float ps = p.psib ? p.psi[vo + j] + p.psib[vo + j] : p.psi[vo + j];
+            run += (rh - ps) + (p.rho2 ? p.rho2[vo + j] : 0.f);
             sfx[j] = run;
         }
     float incl = run;
@@ -685,6 +687,18 @@ __global__ void __launch_bounds__(256) k_reduce_dbdc(SegParams p) {
     const size_t segcap = (size_t)p.ncs * p.Q;
     const size_t src = ((((size_t)b * segcap + tl) * p.G + g) * p.nsl) * p.N + n;
     float sB = 0.f, sC = 0.f;
+    if (p.bc_fused) {
+        // two slots per slice; the second exists only for dC rows of the upper half of a chunk and dB rows
+        // of the lower half (the rows that two tiles of the causal triangle contribute to)
+        const bool upper = ((tl % (size_t)p.Q) >= (size_t)(p.Q / 2));
+        const size_t src2 = ((((size_t)b * segcap + tl) * p.G + g) * (2 * p.nsl)) * p.N + n;
+        for (int s = 0; s < p.nsl; ++s) {
+            sB += p.pB[src2 + (size_t)(2 * s) * p.N];
+            if (!upper) sB += p.pB[src2 + (size_t)(2 * s + 1) * p.N];
+            sC += p.pC[src2 + (size_t)(2 * s) * p.N];
+            if (upper) sC += p.pC[src2 + (size_t)(2 * s + 1) * p.N];
+        }
+    } else
     for (int s = 0; s < p.nsl; ++s) {
         sB += p.pB[src + (size_t)s * p.N];
         sC += p.pC[src + (size_t)s * p.N];
