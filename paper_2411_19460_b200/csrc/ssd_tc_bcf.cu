@@ -195,54 +195,56 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
                     tc_fence_after_sync();
                     issue_scores(hi + 1);
                 }
+                // inter-chunk terms: scaled rows (K = p) times a chunk state.  A tile's first one goes ahead of
+                // the W products (its operand is ready earlier), the second one of tile (1,1) after them.
+                auto inter_dC = [&]() {   // dC += (e^{cs_t} dy_t) H_in
+                    mbar_wait(&hfull, hi & 1, abortp, p.status);
+                    mbar_wait(&scfull, scuse & 1, abortp, p.status);
+                    ++scuse;
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint64_t ad = umma_desc_words(loSk + k * 2, hiK), bd = umma_desc_words(loSt + k * 128, hiSt);
+                        if (k == 0 && hi == 0) umma_bf16_fixed<false>(tm + TF_ACCC, ad, bd, idKM);
+                        else umma_bf16_fixed<true>(tm + TF_ACCC, ad, bd, idKM);
+                    }
+                    umma_commit(&scempty);
+                    umma_commit(&hempty);
+                };
+                auto inter_dB = [&](bool first_into_acc) {   // dB += (dt_s e^{cs_last-cs_s} x_s) Gout
+                    mbar_wait(&gfull, hi & 1, abortp, p.status);
+                    mbar_wait(&scfull, scuse & 1, abortp, p.status);
+                    ++scuse;
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint64_t ad = umma_desc_words(loSk + k * 2, hiK), bd = umma_desc_words(loSt + 1024 + k * 128, hiSt);
+                        if (k == 0 && first_into_acc) umma_bf16_fixed<false>(tm + TF_ACCB, ad, bd, idKM);
+                        else umma_bf16_fixed<true>(tm + TF_ACCB, ad, bd, idKM);
+                    }
+                    umma_commit(&scempty);
+                    umma_commit(&gempty);
+                };
+                if (doC) inter_dC();
+                else inter_dB(hi == 0);
                 mbar_wait(&wfull, hi & 1, abortp, p.status);
                 tc_fence_after_sync();
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {   // dC += W B : K = s
                     const uint64_t ad = umma_desc_words(loWk + (k >> 2) * 1024 + (k & 3) * 2, hiK);
                     const uint64_t bd = umma_desc_words(loBm + k * 128, hiM);
-                    if (k == 0) {
-                        if (hi == 0) umma_bf16_fixed<false>(tm + TF_ACCC, ad, bd, idKM);
-                        else umma_bf16_fixed<true>(tm + TF_ACCC, ad, bd, idKM);
-                    } else {
-                        umma_bf16_fixed<true>(tm + TF_ACCC, ad, bd, idKM);
-                    }
+                    if (k == 0 && hi == 0 && !doC) umma_bf16_fixed<false>(tm + TF_ACCC, ad, bd, idKM);
+                    else umma_bf16_fixed<true>(tm + TF_ACCC, ad, bd, idKM);
                 }
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {   // dB += W^T C : K = t
                     const uint64_t ad = umma_desc_words(loWm + k * 128, hiM);
                     const uint64_t bd = umma_desc_words(loCm + k * 128, hiM);
-                    if (k == 0) {
-                        if (hi == 0) umma_bf16_fixed<false>(tm + TF_ACCB, ad, bd, idMM);
-                        else umma_bf16_fixed<true>(tm + TF_ACCB, ad, bd, idMM);
-                    } else {
-                        umma_bf16_fixed<true>(tm + TF_ACCB, ad, bd, idMM);
-                    }
+                    if (k == 0 && hi == 0 && doC) umma_bf16_fixed<false>(tm + TF_ACCB, ad, bd, idMM);
+                    else umma_bf16_fixed<true>(tm + TF_ACCB, ad, bd, idMM);
                 }
                 umma_commit(&wempty);
-                if (doC) {   // dC += (e^{cs_t} dy_t) H_in : K = p
-                    mbar_wait(&hfull, hi & 1, abortp, p.status);
-                    mbar_wait(&scfull, scuse & 1, abortp, p.status);
-                    ++scuse;
-                    tc_fence_after_sync();
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        umma_bf16_fixed<true>(tm + TF_ACCC, umma_desc_words(loSk + k * 2, hiK), umma_desc_words(loSt + k * 128, hiSt), idKM);
-                    umma_commit(&scempty);
-                    umma_commit(&hempty);
-                }
-                if (doB) {   // dB += (dt_s e^{cs_last-cs_s} x_s) Gout : K = p
-                    mbar_wait(&gfull, hi & 1, abortp, p.status);
-                    mbar_wait(&scfull, scuse & 1, abortp, p.status);
-                    ++scuse;
-                    tc_fence_after_sync();
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        umma_bf16_fixed<true>(tm + TF_ACCB, umma_desc_words(loSk + k * 2, hiK),
-                                              umma_desc_words(loSt + 1024 + k * 128, hiSt), idKM);
-                    umma_commit(&scempty);
-                    umma_commit(&gempty);
-                }
+                if (doC && doB) inter_dB(false);
                 umma_commit(&rempty[hi & 1]);
             }
             umma_commit(&accfull);
@@ -332,6 +334,37 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
             __syncwarp();
             if (lane == 0) mbar_arrive(&sempty);
 
+            // ---- inter-chunk terms: the head's rows scaled per row, as one more K = P operand (dy rows of the
+            // t-block by e^{cs_t} for dC, x rows of the s-block by dt_s e^{cs_last-cs_s} for dB).  A tile's first one
+            // is published before the masking below, so that its MMAs run while W is being made.
+            auto scale_rows = [&](int which) {
+                const unsigned char *rrow = smem + GF_OFF_R + (hi & 1) * 32768 + which * 16384 + rl * 128;
+                unsigned char *srow = smem + GF_OFF_SC + rl * 128;
+                const float sc = which == 0 ? offsC : offsB;
+                uint4 o[2];
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    const uint4 qv = *reinterpret_cast<const uint4 *>(rrow + (((quar * 2 + k) ^ (rl & 7)) << 4));
+                    const uint32_t *qw = reinterpret_cast<const uint32_t *>(&qv);
+                    uint32_t *ow = reinterpret_cast<uint32_t *>(&o[k]);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 f = unpack2g(qw[e]);
+                        ow[e] = pack2g(f.x * sc, f.y * sc);
+                    }
+                }
+                if (scuse >= 1) mbar_wait(&scempty, (scuse - 1) & 1, abortp, p.status);
+                ++scuse;
+#pragma unroll
+                for (int k = 0; k < 2; ++k)
+                    *reinterpret_cast<uint4 *>(srow + (((quar * 2 + k) ^ (rl & 7)) << 4)) = o[k];
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&scfull);
+            };
+            mbar_wait(&rfull[hi & 1], (hi >> 1) & 1, abortp, p.status);
+            scale_rows(doC ? 0 : 1);
+
             // ---- W = score o mask (fp32), Z = W o CB for the row / column sums, W rounded to bf16 for the MMAs
             float2 dacc = make_float2(0.f, 0.f);
             uint32_t pk[2][8];
@@ -403,40 +436,9 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
                 mbar_arrive(&vempty[hi & 1]);
             }
 
-            // ---- inter-chunk terms: the head's rows scaled per row, as one more K = P operand
-            {
-                const int rbuf = hi & 1;
-                const unsigned char *rbase = smem + GF_OFF_R + rbuf * 32768;
-                unsigned char *srow = smem + GF_OFF_SC + rl * 128;
-#pragma unroll
-                for (int which = 0; which < 2; ++which) {
-                    if (which == 0 ? !doC : !doB) continue;
-                    const unsigned char *rrow = rbase + which * 16384 + rl * 128;     // dy row t / x row s
-                    const float sc = which == 0 ? offsC : offsB;
-                    uint4 o[2];
-#pragma unroll
-                    for (int k = 0; k < 2; ++k) {
-                        const uint4 qv = *reinterpret_cast<const uint4 *>(rrow + (((quar * 2 + k) ^ (rl & 7)) << 4));
-                        const uint32_t *qw = reinterpret_cast<const uint32_t *>(&qv);
-                        uint32_t *ow = reinterpret_cast<uint32_t *>(&o[k]);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float2 f = unpack2g(qw[e]);
-                            ow[e] = pack2g(f.x * sc, f.y * sc);
-                        }
-                    }
-                    if (scuse >= 1) mbar_wait(&scempty, (scuse - 1) & 1, abortp, p.status);
-                    ++scuse;
-#pragma unroll
-                    for (int k = 0; k < 2; ++k)
-                        *reinterpret_cast<uint4 *>(srow + (((quar * 2 + k) ^ (rl & 7)) << 4)) = o[k];
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&scfull);
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&rempty[rbuf]);     // this warp has read the head's rows
-            }
+            if (doC && doB) scale_rows(1);     // tile (1,1): its second inter-chunk term
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&rempty[hi & 1]);     // this warp has read the head's rows
 
             // ---- rho_t: the four column slices of a row meet through shared memory
             const size_t vbase = (((size_t)b * p.H + h_begin + hi) * p.ncs + c) << 8;
