@@ -59,6 +59,8 @@ def kind_model(cfg):
         "bwd_dx": ("tensor", 2.0 * HPN + 2 * k * Q * (G * N + H * P), e * (3 * H * P + 2 * G * N) + st),
         "bwd_dC": ("tensor", 2.0 * HPN + 2 * k * Q * (G * N + H * P), e * (2 * H * P + 2 * G * N) + st),
         "bwd_dB": ("tensor", 2.0 * HPN + 2 * k * Q * (G * N), e * (2 * H * P + 2 * G * N) + st),
+        # dB and dC from one masked tile: scores once, the two products of the head-summed tile, two state terms
+        "bwd_dBdC": ("tensor", 4.0 * HPN + 2 * k * Q * (H * P + 2 * G * N), e * (2 * H * P + 2 * G * N) + 2 * st),
         "bwd_finish": ("hbm", 0.0, 16.0 * H),
         "reduce_dBdC": ("hbm", 0.0, 2.0 * e * G * N),
         "final_dAdD": ("hbm", 0.0, 0.0),

@@ -24,7 +24,7 @@ static size_t g_prof_used = 0;
 
 static const char *const kKindNames[KIND_COUNT] = {
     "chunk_cumsum", "chunk_state", "state_pass_fwd", "chunk_scan_fwd", "dstate_contrib",
-    "state_pass_bwd", "bwd_dx", "bwd_dC", "bwd_dB", "bwd_finish", "reduce_dBdC", "final_dAdD", "glue", "decode_step"};
+    "state_pass_bwd", "bwd_dx", "bwd_dC", "bwd_dB", "bwd_finish", "reduce_dBdC", "final_dAdD", "glue", "decode_step", "bwd_dBdC"};
 
 static ProfEvent *prof_begin(int kind, cudaStream_t st) {
     if (!g_prof_on) return nullptr;
@@ -525,7 +525,7 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
             }
             {
                 cudaStream_t st = side->s[1];
-                if (fused_bc) SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_fused(sp, maps, st));
+                if (fused_bc) SSD_LAUNCH(KIND_BWD_DBDC, launch_grad_bc_fused(sp, maps, st));
                 else SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_tc(sp, maps, GB_DB, st));
                 SSD_TRY(cudaEventRecord(side->join[1], st));
             }
@@ -536,7 +536,7 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
             if (!fused_bc) SSD_TRY(cudaStreamWaitEvent(st, side->join[0], 0));
             SSD_TRY(cudaStreamWaitEvent(st, side->join[1], 0));
         } else if (fused_bc) {
-            SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_fused(sp, maps, st));
+            SSD_LAUNCH(KIND_BWD_DBDC, launch_grad_bc_fused(sp, maps, st));
         } else if (pl.use_tc) {
             SSD_LAUNCH(KIND_BWD_DC, launch_grad_bc_tc(sp, maps, GB_DC, st));
             SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_tc(sp, maps, GB_DB, st));

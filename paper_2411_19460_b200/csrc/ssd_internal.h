@@ -104,7 +104,7 @@ enum { STATE_MODE_FWD = 0, STATE_MODE_DSTATE = 1 };
 enum {
     KIND_CUMSUM = 0, KIND_CHUNK_STATE, KIND_STATE_PASS_FWD, KIND_SCAN_FWD, KIND_DSTATE,
     KIND_STATE_PASS_BWD, KIND_BWD_DX, KIND_BWD_DC, KIND_BWD_DB, KIND_BWD_FINISH, KIND_REDUCE_DBDC,
-    KIND_FINAL, KIND_GLUE, KIND_DECODE, KIND_COUNT
+    KIND_FINAL, KIND_GLUE, KIND_DECODE, KIND_BWD_DBDC, KIND_COUNT
 };
 enum { MP_FWD = 0, MP_BWD_DX = 1, MP_DC = 2, MP_DB = 3 };
 

@@ -64,7 +64,7 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
                 const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmG) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ uint64_t bar_ld, bar_cb, rfull[2], rempty[2], sfull, sempty, wfull, wempty, scfull, scempty, hfull, hempty,
+    __shared__ uint64_t bar_ld, bar_cb, rfull[2], rempty[2], sfull, sempty, wfull, scfull, scempty, hfull, hempty,
         gfull, gempty, accfull, vfull[2], vempty[2];
     __shared__ uint32_t tmem_base, abort_flag;
 
@@ -97,7 +97,6 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
         mbar_init(&sfull, 1);
         mbar_init(&sempty, 16);
         mbar_init(&wfull, 16);
-        mbar_init(&wempty, 1);
         mbar_init(&scfull, 16);
         mbar_init(&scempty, 1);
         mbar_init(&hfull, 1);
@@ -227,25 +226,25 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
                 };
                 if (doC) inter_dC();
                 else inter_dB(hi == 0);
-                mbar_wait(&wfull, hi & 1, abortp, p.status);
-                tc_fence_after_sync();
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {   // dC += W B : K = s
-                    const uint64_t ad = umma_desc_words(loWk + (k >> 2) * 1024 + (k & 3) * 2, hiK);
-                    const uint64_t bd = umma_desc_words(loBm + k * 128, hiM);
-                    if (k == 0 && hi == 0 && !doC) umma_bf16_fixed<false>(tm + TF_ACCC, ad, bd, idKM);
-                    else umma_bf16_fixed<true>(tm + TF_ACCC, ad, bd, idKM);
-                }
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {   // dB += W^T C : K = t
-                    const uint64_t ad = umma_desc_words(loWm + k * 128, hiM);
-                    const uint64_t bd = umma_desc_words(loCm + k * 128, hiM);
-                    if (k == 0 && hi == 0 && doC) umma_bf16_fixed<false>(tm + TF_ACCB, ad, bd, idMM);
-                    else umma_bf16_fixed<true>(tm + TF_ACCB, ad, bd, idMM);
-                }
-                umma_commit(&wempty);
-                if (doC && doB) inter_dB(false);
+                if (doC && doB) inter_dB(hi == 0);
                 umma_commit(&rempty[hi & 1]);
+            }
+            // the head sum of the masked tiles (made in fp32 by the mask warps, rounded once): both products
+            mbar_wait(&wfull, 0, abortp, p.status);
+            tc_fence_after_sync();
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {   // dC += Wsum B : K = s
+                const uint64_t ad = umma_desc_words(loWk + (k >> 2) * 1024 + (k & 3) * 2, hiK);
+                const uint64_t bd = umma_desc_words(loBm + k * 128, hiM);
+                if (k == 0 && !doC) umma_bf16_fixed<false>(tm + TF_ACCC, ad, bd, idKM);
+                else umma_bf16_fixed<true>(tm + TF_ACCC, ad, bd, idKM);
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {   // dB += Wsum^T C : K = t
+                const uint64_t ad = umma_desc_words(loWm + k * 128, hiM);
+                const uint64_t bd = umma_desc_words(loCm + k * 128, hiM);
+                if (k == 0 && !doB) umma_bf16_fixed<false>(tm + TF_ACCB, ad, bd, idMM);
+                else umma_bf16_fixed<true>(tm + TF_ACCB, ad, bd, idMM);
             }
             umma_commit(&accfull);
         }
@@ -303,6 +302,9 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
         float *part_rho = reinterpret_cast<float *>(smem + GF_OFF_PART);          // [head parity][3][128]
         float *part_psi = part_rho + 2 * 384;                                     // [head parity][3][128]
         uint32_t scuse = 0;
+        float wsum[32];                             // this thread's row of sum_h W_h: columns w * 16 + j of its two slices
+#pragma unroll
+        for (int k = 0; k < 32; ++k) wsum[k] = 0.f;
 
         for (int hi = 0; hi < nheads; ++hi) {
             float *cs2 = vec + (hi & 1) * GF_VEC_FLOATS, *cf = cs2 + 256, *dtv = cs2 + 512, *blk = cs2 + 768;
@@ -315,24 +317,6 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
                 mbar_wait(&bar_cb, 0, abortp, p.status);
                 tc_fence_after_sync();
             }
-
-            // ---- this thread's two 16-column score slices out of TMEM
-            float v[2][16];
-            bool z[2];
-            mbar_wait(&sfull, hi & 1, abortp, p.status);
-            tc_fence_after_sync();
-#pragma unroll
-            for (int w = 0; w < 2; ++w) {
-                const int jsub = (sb * 128 + w * 64 + quar * 16) >> 5;
-                z[w] = diag && (jsub > isub);
-                if (!z[w]) tmem_ld16_nowait(tm + tlane + TF_S + w * 64 + quar * 16, v[w]);
-            }
-#pragma unroll
-            for (int w = 0; w < 2; ++w)
-                if (!z[w]) tmem_ld_wait16(v[w]);
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sempty);
 
             // ---- inter-chunk terms: the head's rows scaled per row, as one more K = P operand (dy rows of the
             // t-block by e^{cs_t} for dC, x rows of the s-block by dt_s e^{cs_last-cs_s} for dB).  A tile's first one
@@ -365,77 +349,79 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
             mbar_wait(&rfull[hi & 1], (hi >> 1) & 1, abortp, p.status);
             scale_rows(doC ? 0 : 1);
 
-            // ---- W = score o mask (fp32), Z = W o CB for the row / column sums, W rounded to bf16 for the MMAs
+            // ---- W = score o mask (fp32) for this thread's two 16-column slices, one after the other: added to
+            // the head sum; Z = W o CB gives the row sum (rho) and, through a transposing butterfly over the
+            // warp's 32 rows, the column sums (psi).  The score buffer is released after the second slice.
             float2 dacc = make_float2(0.f, 0.f);
-            uint32_t pk[2][8];
+            float csum = 0.f;                                // lanes 0..15: column j of slice 0, lanes 16..31: of slice 1
+            mbar_wait(&sfull, hi & 1, abortp, p.status);
+            tc_fence_after_sync();
 #pragma unroll
             for (int w = 0; w < 2; ++w) {
                 const int cb = sb * 128 + w * 64 + quar * 16;   // first column of the slice (s in chunk)
                 const int jsub = cb >> 5;
-                if (z[w]) {
+                if (diag && (jsub > isub)) continue;            // above the diagonal: W = 0 (uniform over the warp)
+                float vv[16], cbv[16];
+                tmem_ld16_nowait(tm + tlane + TF_S + w * 64 + quar * 16, vv);
+                tmem_ld16_nowait(tm + tlane + TF_CB + w * 64 + quar * 16, cbv);
+                tmem_ld_wait16(vv);
+                if (jsub != isub) {
+                    const float s1 = rowf * blk[isub * 8 + jsub];
+                    const float2 s1v = make_float2(s1, s1);
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) pk[w][k] = 0u;
-#pragma unroll
-                    for (int k = 0; k < 16; ++k) v[w][k] = 0.f;
-                } else {
-                    float *vv = v[w];
-                    float cbv[16];
-                    tmem_ld16_nowait(tm + tlane + TF_CB + w * 64 + quar * 16, cbv);
-                    if (jsub != isub) {
-                        const float s1 = rowf * blk[isub * 8 + jsub];
-                        const float2 s1v = make_float2(s1, s1);
-#pragma unroll
-                        for (int k = 0; k < 16; k += 4) {
-                            const float4 cv = *reinterpret_cast<const float4 *>(cf + cb + k);
-                            const float2 w0 = __fmul2_rn(make_float2(vv[k], vv[k + 1]), __fmul2_rn(make_float2(cv.x, cv.y), s1v));
-                            const float2 w1 = __fmul2_rn(make_float2(vv[k + 2], vv[k + 3]), __fmul2_rn(make_float2(cv.z, cv.w), s1v));
-                            vv[k] = w0.x; vv[k + 1] = w0.y; vv[k + 2] = w1.x; vv[k + 3] = w1.y;
-                        }
-                    } else {
-#pragma unroll
-                        for (int k = 0; k < 16; k += 4) {
-                            const float4 cc = *reinterpret_cast<const float4 *>(cs2 + cb + k);
-                            const float4 d4 = *reinterpret_cast<const float4 *>(dtv + cb + k);
-                            const float ccv[4] = {cc.x, cc.y, cc.z, cc.w};
-                            const float dv[4] = {d4.x, d4.y, d4.z, d4.w};
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const bool on = (cb + k + e) <= r;
-                                const float ex = ex2g(csr - ccv[e]) * dv[e];
-                                vv[k + e] = on ? vv[k + e] * ex : 0.f;
-                            }
-                        }
+                    for (int k = 0; k < 16; k += 4) {
+                        const float4 cv = *reinterpret_cast<const float4 *>(cf + cb + k);
+                        const float2 w0 = __fmul2_rn(make_float2(vv[k], vv[k + 1]), __fmul2_rn(make_float2(cv.x, cv.y), s1v));
+                        const float2 w1 = __fmul2_rn(make_float2(vv[k + 2], vv[k + 3]), __fmul2_rn(make_float2(cv.z, cv.w), s1v));
+                        vv[k] = w0.x; vv[k + 1] = w0.y; vv[k + 2] = w1.x; vv[k + 3] = w1.y;
                     }
+                } else {
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) pk[w][k] = pack2g(vv[2 * k], vv[2 * k + 1]);
-                    tmem_ld_wait16(cbv);
+                    for (int k = 0; k < 16; k += 4) {
+                        const float4 cc = *reinterpret_cast<const float4 *>(cs2 + cb + k);
+                        const float4 d4 = *reinterpret_cast<const float4 *>(dtv + cb + k);
+                        const float ccv[4] = {cc.x, cc.y, cc.z, cc.w};
+                        const float dv[4] = {d4.x, d4.y, d4.z, d4.w};
 #pragma unroll
-                    for (int k = 0; k < 16; k += 2) {
-                        const float2 zz = __fmul2_rn(make_float2(vv[k], vv[k + 1]), make_float2(cbv[k], cbv[k + 1]));
-                        vv[k] = zz.x;          // v now holds this thread's row of Z = W o CB
-                        vv[k + 1] = zz.y;
-                        dacc = __fadd2_rn(dacc, zz);
+                        for (int e = 0; e < 4; ++e) {
+                            const bool on = (cb + k + e) <= r;
+                            const float ex = ex2g(csr - ccv[e]) * dv[e];
+                            vv[k + e] = on ? vv[k + e] * ex : 0.f;
+                        }
                     }
                 }
-            }
-            // ---- publish W: [s-half w][row][128 B], this thread's 16 columns = chunks quar * 2, quar * 2 + 1
-            if (hi >= 1) mbar_wait(&wempty, (hi - 1) & 1, abortp, p.status);
+                tmem_ld_wait16(cbv);
 #pragma unroll
-            for (int w = 0; w < 2; ++w) {
-                unsigned char *mrow = smem + GF_OFF_W + w * 16384 + rl * 128;
+                for (int k = 0; k < 16; k += 2) {
+                    const float2 wv = make_float2(vv[k], vv[k + 1]);
+                    const float2 a = __fadd2_rn(make_float2(wsum[w * 16 + k], wsum[w * 16 + k + 1]), wv);
+                    wsum[w * 16 + k] = a.x;
+                    wsum[w * 16 + k + 1] = a.y;
+                    const float2 zz = __fmul2_rn(wv, make_float2(cbv[k], cbv[k + 1]));
+                    vv[k] = zz.x;
+                    vv[k + 1] = zz.y;
+                    dacc = __fadd2_rn(dacc, zz);
+                }
+                // column sums of Z over the warp's rows: 16 values -> lane l ends with column l & 15
 #pragma unroll
-                for (int ch = 0; ch < 2; ++ch)
-                    *reinterpret_cast<uint4 *>(mrow + (((quar * 2 + ch) ^ (rl & 7)) << 4)) =
-                        make_uint4(pk[w][4 * ch], pk[w][4 * ch + 1], pk[w][4 * ch + 2], pk[w][4 * ch + 3]);
+                for (int o = 8, cnt = 16; o >= 1; o >>= 1, cnt >>= 1) {
+                    const bool up = (lane & o) != 0;
+#pragma unroll
+                    for (int i = 0; i < cnt / 2; ++i) {
+                        const float send = up ? vv[i] : vv[i + cnt / 2];
+                        const float keep = up ? vv[i + cnt / 2] : vv[i];
+                        vv[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+                    }
+                }
+                const float tot = vv[0] + __shfl_xor_sync(0xffffffffu, vv[0], 16);
+                if ((lane >> 4) == w) csum = tot;
             }
             tc_fence_before_sync();
-            fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(&wfull);
+                mbar_arrive(&sempty);
                 mbar_arrive(&vempty[hi & 1]);
             }
-
             if (doC && doB) scale_rows(1);     // tile (1,1): its second inter-chunk term
             __syncwarp();
             if (lane == 0) mbar_arrive(&rempty[hi & 1]);     // this warp has read the head's rows
@@ -455,22 +441,8 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
                     if (kind == 1) p.rhob[vbase + r] = 0.f;
                 }
             }
-            // ---- psi_s: column sums over the 128 rows.  Inside a warp a transposing butterfly leaves lane l
-            // with the sum over the warp's 32 rows of local column l (w * 16 + j); the four row quarters of a
-            // column slice then meet through shared memory.
+            // ---- psi_s: the four row quarters of a column slice meet through shared memory
             {
-                float *zz = &v[0][0];
-#pragma unroll
-                for (int o = 16, cnt = 32; o >= 1; o >>= 1, cnt >>= 1) {
-                    const bool up = (lane & o) != 0;
-#pragma unroll
-                    for (int i = 0; i < cnt / 2; ++i) {
-                        const float send = up ? zz[i] : zz[i + cnt / 2];
-                        const float keep = up ? zz[i + cnt / 2] : zz[i];
-                        zz[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
-                    }
-                }
-                const float csum = zz[0];
                 float *pp = part_psi + (hi & 1) * 384;
                 const int lc = (lane >> 4) * 64 + quar * 16 + (lane & 15);     // column of the tile this lane holds
                 if (q > 0) pp[(q - 1) * 128 + lc] = csum;
@@ -485,6 +457,22 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
                 }
             }
         }
+
+        // ---- the head sum of W, rounded once to bf16: [s-half w][row][128 B], this thread's 16 columns of a
+        // half = chunks quar * 2, quar * 2 + 1
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {
+            unsigned char *mrow = smem + GF_OFF_W + w * 16384 + rl * 128;
+#pragma unroll
+            for (int ch = 0; ch < 2; ++ch) {
+                const float *a = wsum + w * 16 + ch * 8;
+                *reinterpret_cast<uint4 *>(mrow + (((quar * 2 + ch) ^ (rl & 7)) << 4)) =
+                    make_uint4(pack2g(a[0], a[1]), pack2g(a[2], a[3]), pack2g(a[4], a[5]), pack2g(a[6], a[7]));
+            }
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&wfull);
 
         // ---- the CTA's partial slices of the group sums: [B, seg, G, 2 nsl, N] fp32
         mbar_wait(&accfull, 0, abortp, p.status);

@@ -45,7 +45,14 @@ def test_parity_default_path(name):
     print(name, errs)
 
 
-@pytest.mark.parametrize("flags", [SIMT, 0])
+@pytest.mark.parametrize("name", ["bf16_base", "bf16_ragged_g2_b2", "bf16_stiff"])
+def test_parity_two_kernel_dB_dC_path(name):
+    """SSD_FLAG_SPLIT_BC: dB and dC by the two separate tensor-core kernels (the cross-check of the fused one)."""
+    cfg = CASES[name]
+    pu.full_parity(cfg, flags=libssd.SSD_FLAG_SPLIT_BC)
+
+
+@pytest.mark.parametrize("flags", [SIMT, 0, libssd.SSD_FLAG_SPLIT_BC])
 @pytest.mark.parametrize("name", ["cfg0_fp32", "bf16_ragged_g2_b2", "bf16_stiff"])
 def test_segmented_backward_bit_exact_vs_unsegmented(name, flags):
     """The gradients must not depend on the segment length (seg == L is the unsegmented run)."""
