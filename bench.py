@@ -95,10 +95,9 @@ def load_peaks():
 # to the timed workload by tokens x heads per launch (the traffic of these kernels grows in proportion).
 NCU_TRAFFIC_CFG1 = {
     # kernel kind: (bytes per launch, source file, sha256 of that file at capture time)
-    "bwd_dB": (17.23e6, "ssd_tc_bc.cu", "fa854348829bce649cc73d8e7c4852617f169d2b33dfc0b084ac08bddfa77ea2"),
-    "bwd_dC": (17.23e6, "ssd_tc_bc.cu", "fa854348829bce649cc73d8e7c4852617f169d2b33dfc0b084ac08bddfa77ea2"),
-    "bwd_dx": (17.24e6, "ssd_tc_scan.cu", "f9a69e821a37dbde6084db649db63a7c352b2be6226441be1a457ad7026a6f3b"),
-    "chunk_scan_fwd": (10.94e6, "ssd_tc_scan.cu", "f9a69e821a37dbde6084db649db63a7c352b2be6226441be1a457ad7026a6f3b"),
+    "bwd_dBdC": (20.55e6, "ssd_tc_bcf.cu", "83954d5dd60c3cb17a3a7cab87e111b86a0d66df56ff2025b10429034fd70e24"),
+    "bwd_dx": (17.23e6, "ssd_tc_scan.cu", "0b66fe3c6f3bb9b1cb10be98fafc0e1506fdc30e49957ec586b8f877cadf4b68"),
+    "chunk_scan_fwd": (10.94e6, "ssd_tc_scan.cu", "0b66fe3c6f3bb9b1cb10be98fafc0e1506fdc30e49957ec586b8f877cadf4b68"),
     "chunk_state": (7.04e6, "ssd_tc.cu", "d08b62291f529092a782772fee2f8222d1a35a5f326c2cc1ac015e6d3ffe95a6"),
     "dstate_contrib": (7.04e6, "ssd_tc.cu", "d08b62291f529092a782772fee2f8222d1a35a5f326c2cc1ac015e6d3ffe95a6"),
 }
