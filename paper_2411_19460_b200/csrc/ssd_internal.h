@@ -10,6 +10,30 @@
 namespace ssd {
 
 // Everything one segment's kernels need.  Passed by value to every kernel.
+// Programmatic dependent launch: a kernel launched through launch_pdl() may be scheduled while its predecessor
+// in the stream is still running (its CTAs take the SMs the predecessor's last wave leaves idle, and set up
+// their barriers / tensor memory there); pdl_wait() returns once the predecessor has completed and its writes
+// are visible, and must precede the kernel's first global-memory access.  pdl_launch_dependents() lets the
+// successor be scheduled from this point on.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
 struct SegParams {
     int B, L, H, P, N, G, Q;
     int hpg;       // heads per group

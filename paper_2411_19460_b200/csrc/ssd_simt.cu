@@ -163,6 +163,8 @@ cudaError_t launch_chunk_state_simt(const SegParams &p, int dtype, int mode, cud
 __global__ void __launch_bounds__(256, SP_FWD_CTAS)
 k_state_pass_fwd(SegParams p, const float *init, long long init_bs, float *boundary_out,
                  long long bnd_bs, float *final_out, int want_bf16) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int h = blockIdx.y, b = blockIdx.z;
     const int PN = p.P * p.N;
     const int e = blockIdx.x * 1024 + threadIdx.x * 4;
@@ -217,8 +219,7 @@ cudaError_t launch_state_pass_fwd(const SegParams &p, const float *init, long lo
                                   float *boundary_out, long long bnd_bs, float *final_out,
                                   bool want_bf16, cudaStream_t st) {
     dim3 grid(p.P * p.N / 1024, p.H, p.B);
-    k_state_pass_fwd<<<grid, 256, 0, st>>>(p, init, init_bs, boundary_out, bnd_bs, final_out, want_bf16 ? 1 : 0);
-    return cudaGetLastError();
+    return launch_pdl(k_state_pass_fwd, grid, dim3(256), 0, st, p, init, init_bs, boundary_out, bnd_bs, final_out, want_bf16 ? 1 : 0);
 }
 
 // ------------------------------------------------------------------ a9: backward state passing
@@ -228,6 +229,8 @@ cudaError_t launch_state_pass_fwd(const SegParams &p, const float *init, long lo
 // the part of da_t that couples the gradient from the right with the state from the left.
 __global__ void __launch_bounds__(256, SP_BWD_CTAS)
 k_state_pass_bwd(SegParams p, const float *init, float *left_out, int want_bf16) {
+    pdl_launch_dependents();
+    pdl_wait();
     __shared__ float red[SP_BWD_PF][8];
     const int h = blockIdx.y, b = blockIdx.z;
     const int PN = p.P * p.N;
@@ -303,8 +306,7 @@ k_state_pass_bwd(SegParams p, const float *init, float *left_out, int want_bf16)
 cudaError_t launch_state_pass_bwd(const SegParams &p, const float *init, float *left_out,
                                   bool want_bf16, cudaStream_t st) {
     dim3 grid(p.P * p.N / 1024, p.H, p.B);
-    k_state_pass_bwd<<<grid, 256, 0, st>>>(p, init, left_out, want_bf16 ? 1 : 0);
-    return cudaGetLastError();
+    return launch_pdl(k_state_pass_bwd, grid, dim3(256), 0, st, p, init, left_out, want_bf16 ? 1 : 0);
 }
 
 // ------------------------------------------------------------------ a5+a6, a10, a11: masked products (FFMA)
@@ -607,6 +609,8 @@ cudaError_t launch_masked_product_simt(const SegParams &p, int dtype, int mode, 
 // (the CUDA-core kernels store rho = rho_intra + rho_inter as one vector and no rho2).  Suffix/prefix scans: serial inside a lane,
 // warp shuffles across lanes.  Then ddt = ddt_direct + A da, dA partial = sum_t dt_t da_t.
 __global__ void __launch_bounds__(128) k_bwd_finish(SegParams p) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int c = blockIdx.x * 4 + warp, h = blockIdx.y, b = blockIdx.z;
     if (c >= p.nc) return;
@@ -667,13 +671,14 @@ __global__ void __launch_bounds__(128) k_bwd_finish(SegParams p) {
 }
 
 cudaError_t launch_bwd_finish(const SegParams &p, cudaStream_t st) {
-    k_bwd_finish<<<dim3((p.nc + 3) / 4, p.H, p.B), 128, 0, st>>>(p);
-    return cudaGetLastError();
+    return launch_pdl(k_bwd_finish, dim3((p.nc + 3) / 4, p.H, p.B), dim3(128), 0, st, p);
 }
 
 // ------------------------------------------------------------------ a11 tail: sum the head slices of a group
 template <typename T>
 __global__ void __launch_bounds__(256) k_reduce_dbdc(SegParams p) {
+    pdl_launch_dependents();
+    pdl_wait();
     const size_t total = (size_t)p.B * p.nc * p.Q * p.G * p.N;
     const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
     if (i >= total) return;
@@ -711,14 +716,15 @@ __global__ void __launch_bounds__(256) k_reduce_dbdc(SegParams p) {
 cudaError_t launch_reduce_dbdc(const SegParams &p, int dtype, cudaStream_t st) {
     const size_t total = (size_t)p.B * p.nc * p.Q * p.G * p.N;
     const unsigned blocks = (unsigned)((total + 255) / 256);
-    if (dtype == SSD_DTYPE_F32) k_reduce_dbdc<float><<<blocks, 256, 0, st>>>(p);
-    else k_reduce_dbdc<__nv_bfloat16><<<blocks, 256, 0, st>>>(p);
-    return cudaGetLastError();
+    if (dtype == SSD_DTYPE_F32) return launch_pdl(k_reduce_dbdc<float>, dim3(blocks), dim3(256), 0, st, p);
+    return launch_pdl(k_reduce_dbdc<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, p);
 }
 
 // ------------------------------------------------------------------ a13 tail: dA, dD over (batch, chunks)
 // One warp per head; lanes stride over the per-chunk partials in fp64, then a fixed shuffle tree.
 __global__ void __launch_bounds__(32) k_final_dAdD(SegParams p, float *dA, float *dD, int accumulate) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int h = blockIdx.x, lane = threadIdx.x;
     const int nrt = p.ndd;
     double sA = 0.0, sD = 0.0;
@@ -741,8 +747,7 @@ __global__ void __launch_bounds__(32) k_final_dAdD(SegParams p, float *dA, float
 }
 
 cudaError_t launch_final_dAdD(const SegParams &p, float *dA, float *dD, bool accumulate, cudaStream_t st) {
-    k_final_dAdD<<<p.H, 32, 0, st>>>(p, dA, dD, accumulate ? 1 : 0);
-    return cudaGetLastError();
+    return launch_pdl(k_final_dAdD, dim3(p.H), dim3(32), 0, st, p, dA, dD, accumulate ? 1 : 0);
 }
 
 }  // namespace ssd

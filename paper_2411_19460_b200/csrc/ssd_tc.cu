@@ -98,6 +98,8 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
     __shared__ uint32_t tmem_base, abort_flag;
     __shared__ float wsm[2][256];
 
+    pdl_launch_dependents();
+    pdl_wait();       // the first loads are issued right below, by the thread that also sets up the barriers
     const int c = blockIdx.x, hp = blockIdx.y, b = blockIdx.z;
     const int h0 = hp * 2, g = h0 / p.hpg;
     const int tid = threadIdx.x, warp = tid >> 5;
@@ -307,9 +309,8 @@ cudaError_t launch_chunk_state_tc(const SegParams &p, const TcMaps &m, int mode,
                                          CS_STAGE + 32768 + 1024);
     if (e != cudaSuccess) return e;
     dim3 grid(p.nc, p.H / 2, p.B);
-    if (mode == STATE_MODE_FWD) k_chunk_state_tc<<<grid, CS_THREADS, smem, st>>>(p, mode, m.x, m.Bm, m.Hbf);
-    else k_chunk_state_tc<<<grid, CS_THREADS, smem, st>>>(p, mode, m.dy, m.Cm, m.Hbf);
-    return cudaGetLastError();
+    if (mode == STATE_MODE_FWD) return launch_pdl(k_chunk_state_tc, grid, dim3(CS_THREADS), (size_t)smem, st, p, mode, m.x, m.Bm, m.Hbf);
+    return launch_pdl(k_chunk_state_tc, grid, dim3(CS_THREADS), (size_t)smem, st, p, mode, m.dy, m.Cm, m.Hbf);
 }
 
 }  // namespace ssd

@@ -124,6 +124,8 @@ k_grad_bc_tc(SegParams p, const __grid_constant__ CUtensorMap tmRow,   // DC: dy
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    pdl_launch_dependents();
+    pdl_wait();       // barriers and tensor memory are set up; everything below reads what earlier kernels wrote
     const uint32_t tm = tmem_base;
     volatile uint32_t *abortp = &abort_flag;
 
@@ -494,11 +496,11 @@ cudaError_t launch_grad_bc_tc(const SegParams &p, const TcMaps &m, int mode, cud
     if (mode == GB_DC) {
         e = cudaFuncSetAttribute(k_grad_bc_tc<GB_DC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GB_SMEM);
         if (e != cudaSuccess) return e;
-        k_grad_bc_tc<GB_DC><<<grid, GB_THREADS, GB_SMEM, st>>>(p, m.dy, m.x, m.Bm, m.Cm, m.Hbf);
+        return launch_pdl(k_grad_bc_tc<GB_DC>, grid, dim3(GB_THREADS), (size_t)GB_SMEM, st, p, m.dy, m.x, m.Bm, m.Cm, m.Hbf);
     } else {
         e = cudaFuncSetAttribute(k_grad_bc_tc<GB_DB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GB_SMEM);
         if (e != cudaSuccess) return e;
-        k_grad_bc_tc<GB_DB><<<grid, GB_THREADS, GB_SMEM, st>>>(p, m.x, m.dy, m.Cm, m.Bm, m.Gbf);
+        return launch_pdl(k_grad_bc_tc<GB_DB>, grid, dim3(GB_THREADS), (size_t)GB_SMEM, st, p, m.x, m.dy, m.Cm, m.Bm, m.Gbf);
     }
     return cudaGetLastError();
 }

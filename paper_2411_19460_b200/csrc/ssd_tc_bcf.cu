@@ -111,6 +111,8 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    pdl_launch_dependents();
+    pdl_wait();       // barriers and tensor memory are set up; everything below reads what earlier kernels wrote
     const uint32_t tm = tmem_base;
     volatile uint32_t *abortp = &abort_flag;
 
@@ -516,8 +518,7 @@ cudaError_t launch_grad_bc_fused(const SegParams &p, const TcMaps &m, cudaStream
     dim3 grid(3 * p.nc * p.nsl * p.G * p.B);
     cudaError_t e = cudaFuncSetAttribute(k_grad_bc_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GF_SMEM);
     if (e != cudaSuccess) return e;
-    k_grad_bc_fused<<<grid, GF_THREADS, GF_SMEM, st>>>(p, m.x, m.dy, m.Bm, m.Cm, m.Hbf, m.Gbf);
-    return cudaGetLastError();
+    return launch_pdl(k_grad_bc_fused, grid, dim3(GF_THREADS), (size_t)GF_SMEM, st, p, m.x, m.dy, m.Bm, m.Cm, m.Hbf, m.Gbf);
 }
 
 }  // namespace ssd

@@ -130,6 +130,8 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    pdl_launch_dependents();
+    pdl_wait();       // barriers and tensor memory are set up; everything below reads what earlier kernels wrote
     const uint32_t tm = tmem_base;
     // TMEM columns: S [0,256) ; acc1[b] at 256 + 128 b ; acc2[b] at 320 + 128 b
     volatile uint32_t *abortp = &abort_flag;
@@ -454,11 +456,11 @@ cudaError_t launch_scan_tc(const SegParams &p, const TcMaps &m, int mode, cudaSt
     if (mode == SC_FWD) {
         e = cudaFuncSetAttribute(k_scan_tc<SC_FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SC_SMEM);
         if (e != cudaSuccess) return e;
-        k_scan_tc<SC_FWD><<<grid, SC_THREADS, SC_SMEM, st>>>(p, nsplit, m.Cm, m.Bm, m.x, m.Hbf, m.y, m.x);
+        return launch_pdl(k_scan_tc<SC_FWD>, grid, dim3(SC_THREADS), (size_t)SC_SMEM, st, p, nsplit, m.Cm, m.Bm, m.x, m.Hbf, m.y, m.x);
     } else {
         e = cudaFuncSetAttribute(k_scan_tc<SC_DX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SC_SMEM);
         if (e != cudaSuccess) return e;
-        k_scan_tc<SC_DX><<<grid, SC_THREADS, SC_SMEM, st>>>(p, nsplit, m.Bm, m.Cm, m.dy, m.Gbf, m.dx, m.x);
+        return launch_pdl(k_scan_tc<SC_DX>, grid, dim3(SC_THREADS), (size_t)SC_SMEM, st, p, nsplit, m.Bm, m.Cm, m.dy, m.Gbf, m.dx, m.x);
     }
     return cudaGetLastError();
 }
