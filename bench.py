@@ -235,6 +235,8 @@ def run_ours(args):
     cfg = CONFIGS[args.config]
     if args.stream_len:
         return run_stream(args, rep, dev)
+    if args.conv:
+        return run_conv(args, rep, dev)
     if cfg.layers != 1:
         return run_stack(args, rep, dev)
     seg = args.seg or cfg.seg
@@ -587,6 +589,96 @@ def run_stream(args, rep, dev):
     rep.close()
 
 
+def run_conv(args, rep, dev):
+    """The depthwise causal conv + SiLU stage in front of the SSD layer, forward and backward segment by segment with
+    its three-input state carried across the cuts (channels = d_inner + 2 G N of the configuration)."""
+    from paper_2411_19460_b200 import libssd
+
+    cfg = CONFIGS[args.config]
+    seg = args.seg or cfg.seg
+    B, L, C = cfg.B, cfg.L, cfg.H * cfg.P + 2 * cfg.G * cfg.N
+    td = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    gen = torch.Generator(device=dev).manual_seed(cfg.seed + rep.rank)
+    u = torch.randn(B, L, C, generator=gen, device=dev, dtype=torch.float32).to(td)
+    g = torch.randn(B, L, C, generator=gen, device=dev, dtype=torch.float32).to(td)
+    w = torch.randn(C, 4, generator=gen, device=dev) * 0.5
+    bias = torch.randn(C, generator=gen, device=dev) * 0.1
+    out, du = torch.empty_like(u), torch.empty_like(u)
+    nseg = L // seg
+    assert B == 1 and L % seg == 0, "segments are passed as offset pointers: batch 1, L a multiple of seg"
+    states = torch.zeros(nseg + 1, B, 3, C, dtype=td, device=dev)
+    dst = torch.zeros(2, B, 3, C, dtype=torch.float32, device=dev)
+    dw, db = torch.zeros(C, 4, device=dev), torch.zeros(C, device=dev)
+    ws = torch.empty(int(libssd.lib().ssd_conv_workspace_bytes(B, seg, C)), dtype=torch.uint8, device=dev)
+    sl = [(u[:, k * seg:(k + 1) * seg], g[:, k * seg:(k + 1) * seg], out[:, k * seg:(k + 1) * seg],
+           du[:, k * seg:(k + 1) * seg]) for k in range(nseg)]
+    stream = torch.cuda.current_stream()
+
+    def step():
+        for k in range(nseg):
+            libssd.ssd_conv_fwd(sl[k][0], w, bias, states[k], out=sl[k][2], state_out=states[k + 1], stream=stream)
+        dw.zero_()
+        db.zero_()
+        for k in range(nseg - 1, -1, -1):
+            cur = (nseg - 1 - k) & 1
+            libssd.ssd_conv_bwd(sl[k][0], w, bias, states[k], sl[k][1], None if k == nseg - 1 else dst[cur],
+                                du=sl[k][3], dstate=dst[1 - cur], dw=dw, dbias=db, accumulate=True, ws=ws, stream=stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    rep.barrier()
+    run_step, per_replay = step, None
+    if args.graph:
+        # the per-segment calls are short: replay them from a CUDA graph so that the host does not pace them
+        side = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(side):
+            stream = torch.cuda.current_stream()
+            step()
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            nc0 = libssd.launch_count()
+            with torch.cuda.graph(graph, stream=side):
+                step()
+            per_replay = libssd.launch_count() - nc0
+        stream = torch.cuda.current_stream()
+        torch.cuda.synchronize()
+        run_step = graph.replay
+        for _ in range(3):
+            run_step()
+    sampler = ClockSampler(dev) if rep.rank == 0 else None
+    n0 = libssd.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rep.barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        run_step()
+    e1.record(stream)
+    rep.barrier()
+    ms = rep.max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    launches = per_replay * args.steps if per_replay is not None else libssd.launch_count() - n0
+    clocks = sampler.stop() if sampler else None
+    if rep.rank != 0:
+        rep.close()
+        return
+    peaks = load_peaks()
+    e = u.element_size()
+    byts = 5 * e * C                       # fwd: u in, out out; bwd: u, dout in, du out
+    ach = byts * B * L / (ms * 1e-3) / 1e9
+    line = {
+        "metric": "conv1d_fwd_bwd_segmented_tokens_per_s", "value": rep.world * B * L / (ms * 1e-3), "unit": UNIT,
+        "n_gpus": rep.world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+        "impl": "ours",
+        "config": {"workload": cfg.name + "_conv1d", "B": B, "L": L, "channels": C, "width": 4, "seg": seg, "nseg": nseg,
+                   "launch": "cuda graph replay" if args.graph else "stream launches", "l2": "inputs larger than L2", "parallelism": "replicas" if rep.world > 1 else "single"},
+        "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+        "roofline": {"kernel": "conv1d fwd+bwd", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]},
+    }
+    print(json.dumps(line))
+    rep.close()
+
+
 # ----------------------------------------------------------------------------- the CPU oracle legs
 def _oracle_sample(cfg, inp, sample_tokens):
     """fp64 host copies of the first `sample_tokens` tokens (all heads) of the workload."""
@@ -657,6 +749,8 @@ def main():
     ap.add_argument("--stack-len", type=int, default=0, help="config 3: sequence length (default 131072 at layer interval 1, else the configuration's own)")
     ap.add_argument("--stream-len", type=int, default=0, help="forward-only streaming over this many tokens "
                     "(e.g. 2097152) instead of the training step")
+    ap.add_argument("--conv", action="store_true", help="time the depthwise conv + SiLU stage (forward + backward, "
+                    "segment by segment) instead of the SSD step")
     ap.add_argument("--layers", type=int, default=0, help="config 3: number of layers (default 64)")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="time plain stream launches instead of the replay of the step captured in a CUDA graph")

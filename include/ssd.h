@@ -193,6 +193,33 @@ int ssd_decode_step(const ssd_shape_t *shape, const void *x, const float *dt, co
                     const void *Bm, const void *Cm, const float *D, float *h, void *y, void *stream);
 
 /*
+ * Depthwise causal convolution of width 4 followed by SiLU, the stage in front of the SSD layer in a Mamba-2
+ * block, over C channels (x, B and C together: d_inner + 2 G N), with the sequence-axis checkpoint of its own
+ * state: the last three inputs per channel (Appendix C counts them into the sequence checkpoint constant).
+ *     pre[t,c] = bias[c] + sum_{k<4} w[c,k] u[t-3+k, c] ,   out = pre * sigmoid(pre)
+ *   u, out, dout, du   [B, L, C]  I/O dtype, batch stride u_bstride elements (0 = dense); C % 8 == 0, L >= 3
+ *   w [C,4], bias [C]  fp32
+ *   state_in, state_out [B,3,C]   I/O dtype, dense: the three inputs in front of the segment (NULL = zeros) and
+ *                                 the last three of it (NULL = not wanted); forward a segment at a time by
+ *                                 feeding each call's state_out to the next call's state_in
+ * ssd_conv_bwd: for Loss = <out, dout> + (what later segments contribute), walking the segments right to left:
+ *   dtail  [B,3,C] fp32 or NULL: gradient that the segment to the right sends to this segment's last three
+ *                                inputs (that call's `dstate`); NULL for the last segment
+ *   dstate [B,3,C] fp32 or NULL: out: gradient reaching the three inputs in front of this segment
+ *   du: written; dw [C,4], dbias [C]: written, or added to when `accumulate` != 0 (sum over segments)
+ *   ws: ssd_conv_workspace_bytes(B, L, C) bytes of scratch, 256-byte aligned (per-tile partials of dw, dbias,
+ *       added in a fixed order: deterministic)
+ * Device pointers, enqueued on `stream`.  Returns SSD_OK or SSD_EINVAL / SSD_EUNSUPPORTED / SSD_EALIGN /
+ * SSD_EWORKSPACE / SSD_EDEVICE / SSD_ECUDA.
+ */
+size_t ssd_conv_workspace_bytes(int B, int L, int C);
+int ssd_conv_fwd(int B, int L, int C, int dtype, const void *u, long long u_bstride, const float *w, const float *bias,
+                 const void *state_in, void *out, void *state_out, void *stream);
+int ssd_conv_bwd(int B, int L, int C, int dtype, const void *u, long long u_bstride, const float *w, const float *bias,
+                 const void *state_in, const void *dout, const float *dtail, void *du, float *dstate, float *dw,
+                 float *dbias, int accumulate, void *ws, size_t ws_bytes, void *stream);
+
+/*
  * Reads the status word at the start of `ws` (device memory) with a blocking copy: call it after
  * synchronising the stream.  Returns SSD_OK, SSD_ETIMEOUT if some kernel abandoned a bounded wait
  * (its outputs are then undefined), or SSD_ECUDA if the copy failed.

@@ -109,3 +109,38 @@ def decode_step(x, dt, A, Bm, Cm, D, h):
     h_new = alpha[:, :, None, None] * h + (dt[:, :, None] * x)[:, :, :, None] * Bh[:, :, None, :]
     y = np.einsum("bhn,bhpn->bhp", Ch, h_new) + D[None, :, None] * x
     return y, h_new
+
+
+def conv_fwd(u, w, bias, state_in=None):
+    """Depthwise causal convolution of width 4 + SiLU written out (fp64): pre[t,c] = bias[c] + sum_k w[c,k] u[t-3+k,c]
+    with u[-3..-1] = state_in (zeros without one); returns (out [B,L,C], pre, state_out = the last three inputs)."""
+    u, w, bias = map(_f64, (u, w, bias))
+    Bsz, L, C = u.shape
+    st = np.zeros((Bsz, 3, C)) if state_in is None else _f64(state_in)
+    ext = np.concatenate([st, u], axis=1)                       # ext[:, t+3] = u[:, t]
+    pre = np.broadcast_to(bias[None, None, :], (Bsz, L, C)).copy()
+    for k in range(4):
+        pre += w[None, None, :, k] * ext[:, k:k + L, :]
+    out = pre / (1.0 + np.exp(-pre))
+    return out, pre, ext[:, L:L + 3, :].copy()
+
+
+def conv_bwd(u, w, bias, state_in, dout, dtail=None):
+    """Gradients of Loss = <out, dout> (+ dtail on the last three inputs): du, dstate (to the three inputs in front),
+    dw [C,4], dbias [C] (fp64)."""
+    u, w, bias, dout = map(_f64, (u, w, bias, dout))
+    Bsz, L, C = u.shape
+    _, pre, _ = conv_fwd(u, w, bias, state_in)
+    st = np.zeros((Bsz, 3, C)) if state_in is None else _f64(state_in)
+    ext = np.concatenate([st, u], axis=1)
+    sg = 1.0 / (1.0 + np.exp(-pre))
+    dpre = dout * sg * (1.0 + pre * (1.0 - sg))
+    dext = np.zeros_like(ext)
+    dw = np.zeros((C, 4))
+    for k in range(4):
+        dext[:, k:k + L, :] += w[None, None, :, k] * dpre
+        dw[:, k] = np.einsum("blc,blc->c", dpre, ext[:, k:k + L, :])
+    du = dext[:, 3:, :].copy()
+    if dtail is not None:
+        du[:, L - 3:, :] += _f64(dtail)
+    return du, dext[:, :3, :].copy(), dw, dpre.sum(axis=(0, 1))

@@ -24,7 +24,7 @@ static size_t g_prof_used = 0;
 
 static const char *const kKindNames[KIND_COUNT] = {
     "chunk_cumsum", "chunk_state", "state_pass_fwd", "chunk_scan_fwd", "dstate_contrib",
-    "state_pass_bwd", "bwd_dx", "bwd_dC", "bwd_dB", "bwd_finish", "reduce_dBdC", "final_dAdD", "glue", "decode_step", "bwd_dBdC"};
+    "state_pass_bwd", "bwd_dx", "bwd_dC", "bwd_dB", "bwd_finish", "reduce_dBdC", "final_dAdD", "glue", "decode_step", "bwd_dBdC", "conv1d"};
 
 static ProfEvent *prof_begin(int kind, cudaStream_t st) {
     if (!g_prof_on) return nullptr;
@@ -623,6 +623,56 @@ int ssd_decode_step(const ssd_shape_t *s, const void *x, const float *dt, const 
     cudaStream_t st = (cudaStream_t)stream;
     SSD_LAUNCH(KIND_DECODE, launch_decode_step(s->dtype, s->N, x, dt, A, Bm, Cm, D, h, y, s->B, s->H, s->P, s->G,
                                                x_bs, dt_bs, bc_bs, st));
+    return SSD_OK;
+}
+
+static int conv_check(int B, int L, int C, int dtype, long long &bs, long long u_bstride) {
+    if (B <= 0 || L < 3 || C <= 0 || (C % 8)) return SSD_EINVAL;
+    if (dtype != SSD_DTYPE_F32 && dtype != SSD_DTYPE_BF16) return SSD_EUNSUPPORTED;
+    bs = u_bstride ? u_bstride : (long long)L * C;
+    if (bs < (long long)L * C) return SSD_EINVAL;
+    if (((size_t)bs * (dtype == SSD_DTYPE_BF16 ? 2 : 4)) % 16) return SSD_EALIGN;
+    return SSD_OK;
+}
+
+size_t ssd_conv_workspace_bytes(int B, int L, int C) {
+    if (B <= 0 || L <= 0 || C <= 0) return 0;
+    return (size_t)B * conv_tiles(L) * 5 * C * sizeof(float);
+}
+
+int ssd_conv_fwd(int B, int L, int C, int dtype, const void *u, long long u_bstride, const float *w, const float *bias,
+                 const void *state_in, void *out, void *state_out, void *stream) {
+    long long bs;
+    int rc = conv_check(B, L, C, dtype, bs, u_bstride);
+    if (rc) return rc;
+    if (!u || !w || !bias || !out) return SSD_EINVAL;
+    if (misaligned(u) || misaligned(w) || misaligned(bias) || misaligned(out) || (state_in && misaligned(state_in)) ||
+        (state_out && misaligned(state_out)))
+        return SSD_EALIGN;
+    rc = check_device();
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    SSD_LAUNCH(KIND_CONV, launch_conv_fwd(dtype, u, bs, w, bias, state_in, out, state_out, B, L, C, st));
+    return SSD_OK;
+}
+
+int ssd_conv_bwd(int B, int L, int C, int dtype, const void *u, long long u_bstride, const float *w, const float *bias,
+                 const void *state_in, const void *dout, const float *dtail, void *du, float *dstate, float *dw,
+                 float *dbias, int accumulate, void *ws, size_t ws_bytes, void *stream) {
+    long long bs;
+    int rc = conv_check(B, L, C, dtype, bs, u_bstride);
+    if (rc) return rc;
+    if (!u || !w || !bias || !dout || !du || !dw || !dbias || !ws) return SSD_EINVAL;
+    if (misaligned(u) || misaligned(w) || misaligned(bias) || misaligned(dout) || misaligned(du) || misaligned(dw) ||
+        misaligned(dbias) || (state_in && misaligned(state_in)) || (dtail && misaligned(dtail)) ||
+        (dstate && misaligned(dstate)))
+        return SSD_EALIGN;
+    if (((uintptr_t)ws & 255u) || ws_bytes < ssd_conv_workspace_bytes(B, L, C)) return SSD_EWORKSPACE;
+    rc = check_device();
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    SSD_LAUNCH(KIND_CONV, launch_conv_bwd(dtype, u, bs, w, bias, state_in, dout, dtail, du, dstate, dw, dbias,
+                                          accumulate ? 1 : 0, (float *)ws, B, L, C, st));
     return SSD_OK;
 }
 

@@ -1,0 +1,387 @@
+// Depthwise causal convolution (width 4) with SiLU: the stage in front of the SSD layer in a Mamba-2 block,
+// over the channels (x, B, C) = d_inner + 2 G N.  Its only state across a sequence cut is the last three
+// inputs per channel, which is why Appendix C of the paper counts (d_conv - 1)(d_inner + 2 G N) elements of
+// "convolution state" into the sequence-axis checkpoint: forward hands the last three tokens of a segment to
+// the next one; backward walks the segments right to left and hands the gradient that reaches the three
+// tokens in front of a segment to the segment on its left.
+//     pre[t,c] = bias[c] + sum_{k<4} w[c,k] u[t-3+k, c]        out = pre * sigmoid(pre)
+// Bandwidth-shaped kernels: a CTA owns (a block of up to 512 adjacent channels) x (a tile of tokens); one thread
+// brings the tile's rows (plus the three-token halo) into shared memory with bulk async copies, one per token row
+// (the channels of a row are contiguous: up to 1 KB), so that many kilobytes per SM are in flight without holding
+// registers; then a thread owns 4 adjacent channels and walks the tile with a sliding window in registers, writing
+// its results straight to global memory (8 or 16 bytes per thread, coalesced over the channels).  Weight and bias
+// gradients: one partial per token tile, then a fixed-order sum (no atomics).
+#include "ssd_internal.h"
+#include "ssd_sm100.cuh"
+
+namespace ssd {
+
+using namespace sm100;
+
+namespace {
+
+constexpr int CV_THREADS = 128;   // x 4 channels = 512 channels per CTA
+constexpr int CV_CH = 4;          // channels per thread: one 8-byte bf16 vector (16 bytes in fp32)
+constexpr int CV_TILE_F = 32;     // tokens per CTA, forward
+constexpr int CV_TILE_B = 32;     // tokens per CTA, backward (it stages u and dout, with three more tokens of each)
+
+// 1 / (1 + e^-x) from one ex2.approx and one rcp.approx (relative error of the order of 1e-7; the kernels are bound
+// by instruction issue, not by memory, and an IEEE division alone would cost as much as the rest of an element)
+__device__ __forceinline__ float sigmoid_fast(float x) {
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * -1.4426950408889634f));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.f + e));
+    return r;
+}
+
+template <typename T> __device__ __forceinline__ void ld4(const T *p, float *f);
+template <> __device__ __forceinline__ void ld4<float>(const float *p, float *f) {
+    const float4 a = *reinterpret_cast<const float4 *>(p);
+    f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w;
+}
+template <> __device__ __forceinline__ void ld4<__nv_bfloat16>(const __nv_bfloat16 *p, float *f) {
+    const uint2 v = *reinterpret_cast<const uint2 *>(p);
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&v.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&v.y));
+    f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y;
+}
+template <typename T> __device__ __forceinline__ void st4(T *p, const float *f);
+template <> __device__ __forceinline__ void st4<float>(float *p, const float *f) {
+    *reinterpret_cast<float4 *>(p) = make_float4(f[0], f[1], f[2], f[3]);
+}
+template <> __device__ __forceinline__ void st4<__nv_bfloat16>(__nv_bfloat16 *p, const float *f) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(f[0], f[1]), hi = __floats2bfloat162_rn(f[2], f[3]);
+    uint2 v;
+    v.x = *reinterpret_cast<unsigned int *>(&lo);
+    v.y = *reinterpret_cast<unsigned int *>(&hi);
+    *reinterpret_cast<uint2 *>(p) = v;
+}
+
+// Stage rows [t_first, t_last) of a [L, C] tensor (channels cbase .. cbase + nch) into shared memory, row r of the
+// stage = token t_first + r, 512 channels of room per row.  Tokens in front of the segment come from the carried
+// state (3 rows) or are zero-filled; called by one thread, completion on `bar`.
+template <typename T>
+__device__ __forceinline__ void stage_rows(T *stage, const T *src, const T *state, long long t_first, long long t_last, int C,
+                                           int cbase, int nch, uint64_t *bar) {
+    const uint32_t row_bytes = (uint32_t)nch * sizeof(T);
+    uint32_t total = 0;
+    for (long long t = t_first; t < t_last; ++t)
+        if (t >= 0 || state) total += row_bytes;
+    if (total) mbar_arrive_expect_tx(bar, total);
+    else mbar_arrive(bar);
+    for (long long t = t_first; t < t_last; ++t) {
+        T *dst = stage + (size_t)(t - t_first) * 512;
+        if (t >= 0) bulk_load(dst, src + (size_t)t * C + cbase, row_bytes, bar);
+        else if (state) bulk_load(dst, state + (size_t)(3 + t) * C + cbase, row_bytes, bar);
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(CV_THREADS) k_conv_fwd(const T *u, long long u_bs, const float *w, const float *bias,
+                                                         const T *state_in, T *out, T *state_out, int L, int C) {
+    extern __shared__ __align__(128) unsigned char cv_smem[];
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    __shared__ unsigned int status_dummy;
+    T *su = reinterpret_cast<T *>(cv_smem);                       // [CV_TILE_F + 3][512]
+    const int cbase = blockIdx.x * 512, nch = min(512, C - cbase);
+    const int c0 = cbase + threadIdx.x * CV_CH;
+    const int b = blockIdx.z;
+    const long long t_begin = (long long)blockIdx.y * CV_TILE_F, t_end = min(t_begin + (long long)CV_TILE_F, (long long)L);
+    const T *ub = u + (size_t)b * u_bs;
+    const T *sb = state_in ? state_in + (size_t)b * 3 * C : nullptr;
+    T *ob = out + (size_t)b * u_bs;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        status_dummy = 0;
+        fence_barrier_init();
+    }
+    // rows in front of the segment without a carried state: zeros (plain stores, before the barrier below)
+    if (!sb && t_begin < 3)
+        for (int i = threadIdx.x; i < (int)(3 - t_begin) * 512; i += CV_THREADS) su[i] = (T)0.f;
+    __syncthreads();
+    if (threadIdx.x == 0) stage_rows(su, ub, sb, t_begin - 3, t_end, C, cbase, nch, &bar);
+    const bool active = c0 < C;
+    float wk[CV_CH][4], bs[CV_CH];
+    if (active) {
+#pragma unroll
+        for (int i = 0; i < CV_CH; ++i) {
+            const float4 wv = *reinterpret_cast<const float4 *>(w + (size_t)(c0 + i) * 4);
+            wk[i][0] = wv.x; wk[i][1] = wv.y; wk[i][2] = wv.z; wk[i][3] = wv.w;
+            bs[i] = bias[c0 + i];
+        }
+    }
+    mbar_wait(&bar, 0, &abort_flag, &status_dummy);
+    if (!active) return;
+    const T *sp = su + threadIdx.x * CV_CH;
+    float x0[CV_CH], x1[CV_CH], x2[CV_CH], x3[CV_CH];   // u[t-3], u[t-2], u[t-1], u[t]
+    ld4(sp, x0);
+    ld4(sp + 512, x1);
+    ld4(sp + 1024, x2);
+    const int nt = (int)(t_end - t_begin);
+#pragma unroll 4
+    for (int j = 0; j < nt; ++j) {
+        ld4(sp + (size_t)(j + 3) * 512, x3);
+        float o[CV_CH];
+#pragma unroll
+        for (int i = 0; i < CV_CH; ++i) {
+            const float pre = fmaf(wk[i][3], x3[i], fmaf(wk[i][2], x2[i], fmaf(wk[i][1], x1[i], fmaf(wk[i][0], x0[i], bs[i]))));
+            o[i] = pre * sigmoid_fast(pre);
+            x0[i] = x1[i]; x1[i] = x2[i]; x2[i] = x3[i];
+        }
+        st4(ob + (size_t)(t_begin + j) * C + c0, o);
+    }
+    // the last three inputs of the segment are the state of the next one
+    if (state_out && t_end == L) {
+        T *so = state_out + (size_t)b * 3 * C;
+        st4(so + c0, x0);
+        st4(so + (size_t)C + c0, x1);
+        st4(so + (size_t)2 * C + c0, x2);
+    }
+}
+
+// Backward over one token tile.  dpre[t] = dout[t] * silu'(pre[t]);  du[t] = sum_k w[k] dpre[t+3-k], so a tile also
+// forms dpre of the three tokens to its right (for du only); past the end of the segment they are not formed: their
+// effect on the last three tokens arrives as `dtail`.  dw, dbias: the tile's own tokens.
+template <typename T>
+__global__ void __launch_bounds__(CV_THREADS) k_conv_bwd(const T *u, long long u_bs, const float *w, const float *bias,
+                                                         const T *state_in, const T *dout, const float *dtail, T *du,
+                                                         float *part, int L, int C) {
+    extern __shared__ __align__(128) unsigned char cv_smem[];
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    __shared__ unsigned int status_dummy;
+    T *su = reinterpret_cast<T *>(cv_smem);                       // [CV_TILE_B + 6][512]  u rows t_begin-3 .. s_end
+    T *sg = su + (size_t)(CV_TILE_B + 6) * 512;                   // [CV_TILE_B + 3][512]  dout rows t_begin .. s_end
+    const int cbase = blockIdx.x * 512, nch = min(512, C - cbase);
+    const int c0 = cbase + threadIdx.x * CV_CH;
+    const int b = blockIdx.z;
+    const long long t_begin = (long long)blockIdx.y * CV_TILE_B, t_end = min(t_begin + (long long)CV_TILE_B, (long long)L);
+    const long long s_end = min(t_end + 3, (long long)L);
+    const T *ub = u + (size_t)b * u_bs, *gb = dout + (size_t)b * u_bs;
+    const T *sb = state_in ? state_in + (size_t)b * 3 * C : nullptr;
+    T *dub = du + (size_t)b * u_bs;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 2);
+        abort_flag = 0;
+        status_dummy = 0;
+        fence_barrier_init();
+    }
+    if (!sb && t_begin < 3)
+        for (int i = threadIdx.x; i < (int)(3 - t_begin) * 512; i += CV_THREADS) su[i] = (T)0.f;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        stage_rows(su, ub, sb, t_begin - 3, s_end, C, cbase, nch, &bar);
+        stage_rows(sg, gb, (const T *)nullptr, t_begin, s_end, C, cbase, nch, &bar);
+    }
+    const bool active = c0 < C;
+    float wk[CV_CH][4], bs[CV_CH];
+    if (active) {
+#pragma unroll
+        for (int i = 0; i < CV_CH; ++i) {
+            const float4 wv = *reinterpret_cast<const float4 *>(w + (size_t)(c0 + i) * 4);
+            wk[i][0] = wv.x; wk[i][1] = wv.y; wk[i][2] = wv.z; wk[i][3] = wv.w;
+            bs[i] = bias[c0 + i];
+        }
+    }
+    mbar_wait(&bar, 0, &abort_flag, &status_dummy);
+    if (!active) return;
+    const T *spu = su + threadIdx.x * CV_CH, *spg = sg + threadIdx.x * CV_CH;
+    float x0[CV_CH], x1[CV_CH], x2[CV_CH], x3[CV_CH];
+    float d0[CV_CH], d1[CV_CH], d2[CV_CH], d3[CV_CH];     // dpre[t], dpre[t+1], dpre[t+2], dpre[t+3] while emitting du[t]
+    float aw[CV_CH][4], ab[CV_CH];
+#pragma unroll
+    for (int i = 0; i < CV_CH; ++i) {
+        aw[i][0] = aw[i][1] = aw[i][2] = aw[i][3] = 0.f;
+        ab[i] = 0.f;
+        d0[i] = d1[i] = d2[i] = d3[i] = 0.f;
+    }
+    ld4(spu, x0);
+    ld4(spu + 512, x1);
+    ld4(spu + 1024, x2);
+    const int ns = (int)(s_end - t_begin), nt = (int)(t_end - t_begin);
+    for (int j = 0; j < ns + 3; ++j) {                     // s = t_begin + j
+        float dp[CV_CH];
+        if (j < ns) {
+            float g[CV_CH];
+            ld4(spu + (size_t)(j + 3) * 512, x3);
+            ld4(spg + (size_t)j * 512, g);
+#pragma unroll
+            for (int i = 0; i < CV_CH; ++i) {
+                const float pre = fmaf(wk[i][3], x3[i], fmaf(wk[i][2], x2[i], fmaf(wk[i][1], x1[i], fmaf(wk[i][0], x0[i], bs[i]))));
+                const float sgm = sigmoid_fast(pre);
+                dp[i] = g[i] * sgm * fmaf(pre, 1.f - sgm, 1.f);
+                if (j < nt) {   // the tile's own tokens: weight and bias gradients
+                    aw[i][0] = fmaf(dp[i], x0[i], aw[i][0]);
+                    aw[i][1] = fmaf(dp[i], x1[i], aw[i][1]);
+                    aw[i][2] = fmaf(dp[i], x2[i], aw[i][2]);
+                    aw[i][3] = fmaf(dp[i], x3[i], aw[i][3]);
+                    ab[i] += dp[i];
+                }
+                x0[i] = x1[i]; x1[i] = x2[i]; x2[i] = x3[i];
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < CV_CH; ++i) dp[i] = 0.f;
+        }
+        // shift the dpre window; after it d3 = dpre[s], d0 = dpre[s-3]: du[s-3] is complete
+#pragma unroll
+        for (int i = 0; i < CV_CH; ++i) { d0[i] = d1[i]; d1[i] = d2[i]; d2[i] = d3[i]; d3[i] = dp[i]; }
+        const int jt = j - 3;
+        if (jt >= 0 && jt < nt) {
+            const long long t = t_begin + jt;
+            float o[CV_CH];
+#pragma unroll
+            for (int i = 0; i < CV_CH; ++i)
+                o[i] = fmaf(wk[i][3], d0[i], fmaf(wk[i][2], d1[i], fmaf(wk[i][1], d2[i], wk[i][0] * d3[i])));
+            if (dtail && t >= (long long)L - 3) {
+                float e[CV_CH];
+                ld4(dtail + ((size_t)b * 3 + (size_t)(t - ((long long)L - 3))) * C + c0, e);
+#pragma unroll
+                for (int i = 0; i < CV_CH; ++i) o[i] += e[i];
+            }
+            st4(dub + (size_t)t * C + c0, o);
+        }
+    }
+    // partial weight / bias gradients of this tile: part[b][tile][5][C]
+    {
+        float *pp = part + (((size_t)b * gridDim.y + blockIdx.y) * 5) * C + c0;
+        float col[CV_CH];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+#pragma unroll
+            for (int i = 0; i < CV_CH; ++i) col[i] = aw[i][k];
+            st4(pp + (size_t)k * C, col);
+        }
+        st4(pp + (size_t)4 * C, ab);
+    }
+}
+
+// What the first three dpre rows of the segment send to the three tokens in front of it (their dpre is recomputed
+// here: three tokens per channel, plain loads).
+template <typename T>
+__global__ void __launch_bounds__(CV_THREADS) k_conv_dstate(const T *u, long long u_bs, const float *w, const float *bias,
+                                                            const T *state_in, const T *dout, float *dstate, int L, int C) {
+    const int c0 = (blockIdx.x * CV_THREADS + threadIdx.x) * CV_CH;
+    if (c0 >= C) return;
+    const int b = blockIdx.z;
+    const T *ub = u + (size_t)b * u_bs, *gb = dout + (size_t)b * u_bs;
+    const T *sb = state_in ? state_in + (size_t)b * 3 * C : nullptr;
+    float wk[CV_CH][4], bs[CV_CH];
+#pragma unroll
+    for (int i = 0; i < CV_CH; ++i) {
+        const float4 wv = *reinterpret_cast<const float4 *>(w + (size_t)(c0 + i) * 4);
+        wk[i][0] = wv.x; wk[i][1] = wv.y; wk[i][2] = wv.z; wk[i][3] = wv.w;
+        bs[i] = bias[c0 + i];
+    }
+    float y0[CV_CH], y1[CV_CH], y2[CV_CH], y3[CV_CH], q[3][CV_CH];
+#pragma unroll
+    for (int i = 0; i < CV_CH; ++i) y0[i] = y1[i] = y2[i] = 0.f;
+    if (sb) {
+        ld4(sb + c0, y0);
+        ld4(sb + (size_t)C + c0, y1);
+        ld4(sb + (size_t)2 * C + c0, y2);
+    }
+#pragma unroll
+    for (int s = 0; s < 3; ++s) {
+        float g[CV_CH];
+        ld4(ub + (size_t)s * C + c0, y3);
+        ld4(gb + (size_t)s * C + c0, g);
+#pragma unroll
+        for (int i = 0; i < CV_CH; ++i) {
+            const float pre = fmaf(wk[i][3], y3[i], fmaf(wk[i][2], y2[i], fmaf(wk[i][1], y1[i], fmaf(wk[i][0], y0[i], bs[i]))));
+            const float sgm = sigmoid_fast(pre);
+            q[s][i] = g[i] * sgm * fmaf(pre, 1.f - sgm, 1.f);
+            y0[i] = y1[i]; y1[i] = y2[i]; y2[i] = y3[i];
+        }
+    }
+    // token -3 feeds pre[0] through w[0]; token -2: pre[0] w[1], pre[1] w[0]; token -1: pre[0] w[2], pre[1] w[1], pre[2] w[0]
+    float e[CV_CH];
+    float *ds = dstate + (size_t)b * 3 * C + c0;
+#pragma unroll
+    for (int i = 0; i < CV_CH; ++i) e[i] = wk[i][0] * q[0][i];
+    st4(ds, e);
+#pragma unroll
+    for (int i = 0; i < CV_CH; ++i) e[i] = fmaf(wk[i][0], q[1][i], wk[i][1] * q[0][i]);
+    st4(ds + (size_t)C, e);
+#pragma unroll
+    for (int i = 0; i < CV_CH; ++i) e[i] = fmaf(wk[i][0], q[2][i], fmaf(wk[i][1], q[1][i], wk[i][2] * q[0][i]));
+    st4(ds + (size_t)2 * C, e);
+}
+
+// dw[c][k], dbias[c]: the tile partials added in tile order (then batch order), in fp64
+__global__ void __launch_bounds__(128) k_conv_reduce(const float *part, float *dw, float *dbias, int C, int ntiles, int B,
+                                                     int accumulate) {
+    const int idx = blockIdx.x * 128 + threadIdx.x;      // (k, c), k = 0..4
+    if (idx >= 5 * C) return;
+    const int k = idx / C, c = idx % C;
+    double s = 0.0;
+    for (int b = 0; b < B; ++b)
+        for (int t = 0; t < ntiles; ++t) s += (double)part[(((size_t)b * ntiles + t) * 5 + k) * C + c];
+    if (k < 4) {
+        float *d = dw + (size_t)c * 4 + k;
+        *d = accumulate ? *d + (float)s : (float)s;
+    } else {
+        dbias[c] = accumulate ? dbias[c] + (float)s : (float)s;
+    }
+}
+
+template <typename T>
+cudaError_t conv_fwd_t(const T *u, long long u_bs, const float *w, const float *bias, const T *state_in, T *out, T *state_out,
+                       int B, int L, int C, cudaStream_t st) {
+    const int smem = (CV_TILE_F + 3) * 512 * (int)sizeof(T);
+    cudaError_t e = cudaFuncSetAttribute(k_conv_fwd<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    dim3 grid((C + 511) / 512, (L + CV_TILE_F - 1) / CV_TILE_F, B);
+    k_conv_fwd<T><<<grid, CV_THREADS, smem, st>>>(u, u_bs, w, bias, state_in, out, state_out, L, C);
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t conv_bwd_t(const T *u, long long u_bs, const float *w, const float *bias, const T *state_in, const T *dout,
+                       const float *dtail, T *du, float *dstate, float *part, int B, int L, int C, cudaStream_t st) {
+    const int smem = (2 * CV_TILE_B + 9) * 512 * (int)sizeof(T);
+    cudaError_t e = cudaFuncSetAttribute(k_conv_bwd<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    dim3 grid((C + 511) / 512, (L + CV_TILE_B - 1) / CV_TILE_B, B);
+    k_conv_bwd<T><<<grid, CV_THREADS, smem, st>>>(u, u_bs, w, bias, state_in, dout, dtail, du, part, L, C);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (dstate) {
+        dim3 g1((C / CV_CH + CV_THREADS - 1) / CV_THREADS, 1, B);
+        k_conv_dstate<T><<<g1, CV_THREADS, 0, st>>>(u, u_bs, w, bias, state_in, dout, dstate, L, C);
+        e = cudaGetLastError();
+    }
+    return e;
+}
+
+}  // namespace
+
+int conv_tiles(int L) { return (L + CV_TILE_B - 1) / CV_TILE_B; }
+
+cudaError_t launch_conv_fwd(int dtype, const void *u, long long u_bs, const float *w, const float *bias,
+                            const void *state_in, void *out, void *state_out, int B, int L, int C, cudaStream_t st) {
+    if (dtype == SSD_DTYPE_F32)
+        return conv_fwd_t<float>((const float *)u, u_bs, w, bias, (const float *)state_in, (float *)out, (float *)state_out, B,
+                                 L, C, st);
+    return conv_fwd_t<__nv_bfloat16>((const __nv_bfloat16 *)u, u_bs, w, bias, (const __nv_bfloat16 *)state_in,
+                                     (__nv_bfloat16 *)out, (__nv_bfloat16 *)state_out, B, L, C, st);
+}
+
+cudaError_t launch_conv_bwd(int dtype, const void *u, long long u_bs, const float *w, const float *bias,
+                            const void *state_in, const void *dout, const float *dtail, void *du, float *dstate,
+                            float *dw, float *dbias, int accumulate, float *part, int B, int L, int C, cudaStream_t st) {
+    cudaError_t e;
+    if (dtype == SSD_DTYPE_F32)
+        e = conv_bwd_t<float>((const float *)u, u_bs, w, bias, (const float *)state_in, (const float *)dout, dtail, (float *)du,
+                              dstate, part, B, L, C, st);
+    else
+        e = conv_bwd_t<__nv_bfloat16>((const __nv_bfloat16 *)u, u_bs, w, bias, (const __nv_bfloat16 *)state_in,
+                                      (const __nv_bfloat16 *)dout, dtail, (__nv_bfloat16 *)du, dstate, part, B, L, C, st);
+    if (e != cudaSuccess) return e;
+    k_conv_reduce<<<(5 * C + 127) / 128, 128, 0, st>>>(part, dw, dbias, C, conv_tiles(L), B, accumulate);
+    return cudaGetLastError();
+}
+
+}  // namespace ssd

@@ -100,6 +100,13 @@ cudaError_t launch_glue(int dtype, bool transpose, const void *a, const void *b,
 cudaError_t launch_residual(int dtype, void *dst, const void *src, long long n_per_batch, long long bstride, int B,
                             cudaStream_t st);
 
+// ssd_conv.cu : depthwise causal convolution (width 4) + SiLU in front of the SSD layer, with its 3-token state
+int conv_tiles(int L);
+cudaError_t launch_conv_fwd(int dtype, const void *u, long long u_bs, const float *w, const float *bias,
+                            const void *state_in, void *out, void *state_out, int B, int L, int C, cudaStream_t st);
+cudaError_t launch_conv_bwd(int dtype, const void *u, long long u_bs, const float *w, const float *bias,
+                            const void *state_in, const void *dout, const float *dtail, void *du, float *dstate,
+                            float *dw, float *dbias, int accumulate, float *part, int B, int L, int C, cudaStream_t st);
 // ssd_decode.cu : one token of the recurrence, state updated in place
 cudaError_t launch_decode_step(int dtype, int N, const void *x, const float *dt, const float *A, const void *Bm,
                                const void *Cm, const float *D, float *h, void *y, int B, int H, int P, int G,
@@ -128,7 +135,7 @@ enum { STATE_MODE_FWD = 0, STATE_MODE_DSTATE = 1 };
 enum {
     KIND_CUMSUM = 0, KIND_CHUNK_STATE, KIND_STATE_PASS_FWD, KIND_SCAN_FWD, KIND_DSTATE,
     KIND_STATE_PASS_BWD, KIND_BWD_DX, KIND_BWD_DC, KIND_BWD_DB, KIND_BWD_FINISH, KIND_REDUCE_DBDC,
-    KIND_FINAL, KIND_GLUE, KIND_DECODE, KIND_BWD_DBDC, KIND_COUNT
+    KIND_FINAL, KIND_GLUE, KIND_DECODE, KIND_BWD_DBDC, KIND_CONV, KIND_COUNT
 };
 enum { MP_FWD = 0, MP_BWD_DX = 1, MP_DC = 2, MP_DB = 3 };
 

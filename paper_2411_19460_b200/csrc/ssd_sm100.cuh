@@ -114,6 +114,14 @@ __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.b
 // all earlier stores of this thread are complete
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
+// Untiled bulk load global -> shared: `bytes` contiguous bytes (a multiple of 16, both addresses 16-byte aligned);
+// completes on `bar` (count the bytes in with mbar_arrive_expect_tx).  No multicast.
+__device__ __forceinline__ void bulk_load(void *sdst, const void *gsrc, uint32_t bytes, uint64_t *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(sdst)),
+                 "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+
 // Untiled bulk store shared -> global: `bytes` contiguous bytes (a multiple of 16, both addresses 16-byte
 // aligned), in the bulk async group of the issuing thread.
 __device__ __forceinline__ void bulk_store(void *gdst, const void *ssrc, uint32_t bytes) {

@@ -25,7 +25,8 @@ EXPORTS = ["ssd_workspace_bytes", "ssd_boundary_bytes", "ssd_fwd", "ssd_fwd_segm
            "ssd_bwd_segmented", "ssd_poll_status", "ssd_strerror", "ssd_version",
            "ssd_last_cuda_error", "ssd_launch_count", "ssd_kernel_kinds", "ssd_kernel_name",
            "ssd_profile", "ssd_profile_read", "ssd_fwd_static_ws", "ssd_glue_fwd", "ssd_glue_bwd",
-           "ssd_glue_residual", "ssd_decode_step"]
+           "ssd_glue_residual", "ssd_decode_step", "ssd_conv_fwd", "ssd_conv_bwd",
+           "ssd_conv_workspace_bytes"]
 
 
 class SSDShape(ctypes.Structure):
@@ -72,6 +73,13 @@ def lib():
         L.ssd_glue_fwd.argtypes = [sp, vp, vp, fp, vp, vp]
         L.ssd_glue_bwd.restype = ctypes.c_int
         L.ssd_glue_bwd.argtypes = [sp, vp, fp, vp, vp]
+        ci, ll = ctypes.c_int, ctypes.c_longlong
+        L.ssd_conv_workspace_bytes.restype = ctypes.c_size_t
+        L.ssd_conv_workspace_bytes.argtypes = [ci, ci, ci]
+        L.ssd_conv_fwd.restype = ctypes.c_int
+        L.ssd_conv_fwd.argtypes = [ci, ci, ci, ci, vp, ll, fp, fp, vp, vp, vp, vp]
+        L.ssd_conv_bwd.restype = ctypes.c_int
+        L.ssd_conv_bwd.argtypes = [ci, ci, ci, ci, vp, ll, fp, fp, vp, vp, fp, vp, fp, fp, fp, ci, vp, ctypes.c_size_t, vp]
         L.ssd_decode_step.restype = ctypes.c_int
         L.ssd_decode_step.argtypes = [sp, vp, fp, fp, vp, vp, fp, fp, vp, vp]
         L.ssd_glue_residual.restype = ctypes.c_int
@@ -272,6 +280,52 @@ def ssd_decode_step(x, dt, A, Bm, Cm, D, h, y=None, stream=None):
     if rc != SSD_OK:
         raise SSDError(rc, "ssd_decode_step")
     return y
+
+
+def _conv_args(u):
+    B, L, C = u.shape
+    if u.dtype == torch.bfloat16:
+        code = SSD_DTYPE_BF16
+    elif u.dtype == torch.float32:
+        code = SSD_DTYPE_F32
+    else:
+        raise TypeError("u must be float32 or bfloat16")
+    if not u.is_cuda or u.stride(2) != 1 or u.stride(1) != C:
+        raise ValueError("u must be a CUDA tensor [B, L, C] with contiguous rows")
+    return B, L, C, code, (u.stride(0) if B > 1 else 0)
+
+
+def ssd_conv_fwd(u, w, bias, state_in=None, *, out=None, state_out=None, stream=None):
+    """out, state_out = SiLU(depthwise causal conv4(u)); state_in / state_out [B,3,C] carry the three inputs across
+    a segment cut."""
+    B, L, C, code, bs = _conv_args(u)
+    out = torch.empty_like(u) if out is None else out
+    state_out = torch.empty(B, 3, C, dtype=u.dtype, device=u.device) if state_out is None else state_out
+    rc = lib().ssd_conv_fwd(B, L, C, code, _ptr(u), bs, _ptr(w), _ptr(bias), _ptr(state_in), _ptr(out), _ptr(state_out),
+                            _stream(stream))
+    if rc != SSD_OK:
+        raise SSDError(rc, "ssd_conv_fwd")
+    return out, state_out
+
+
+def ssd_conv_bwd(u, w, bias, state_in, dout, dtail=None, *, du=None, dstate=None, dw=None, dbias=None, accumulate=False,
+                 ws=None, stream=None):
+    """du, dstate, dw, dbias of one segment (Algorithm 2's order: the segment to the right first; its dstate is this
+    call's dtail)."""
+    B, L, C, code, bs = _conv_args(u)
+    dev = u.device
+    du = torch.empty_like(u) if du is None else du
+    dstate = torch.empty(B, 3, C, dtype=torch.float32, device=dev) if dstate is None else dstate
+    dw = torch.zeros(C, 4, dtype=torch.float32, device=dev) if dw is None else dw
+    dbias = torch.zeros(C, dtype=torch.float32, device=dev) if dbias is None else dbias
+    nws = int(lib().ssd_conv_workspace_bytes(B, L, C))
+    ws = torch.empty(nws, dtype=torch.uint8, device=dev) if ws is None else ws
+    rc = lib().ssd_conv_bwd(B, L, C, code, _ptr(u), bs, _ptr(w), _ptr(bias), _ptr(state_in), _ptr(dout), _ptr(dtail),
+                            _ptr(du), _ptr(dstate), _ptr(dw), _ptr(dbias), 1 if accumulate else 0, _ptr(ws), ws.numel(),
+                            _stream(stream))
+    if rc != SSD_OK:
+        raise SSDError(rc, "ssd_conv_bwd")
+    return du, dstate, dw, dbias
 
 
 def _glue_shape(t):
