@@ -95,11 +95,11 @@ def load_peaks():
 # to the timed workload by tokens x heads per launch (the traffic of these kernels grows in proportion).
 NCU_TRAFFIC_CFG1 = {
     # kernel kind: (bytes per launch, source file, sha256 of that file at capture time)
-    "bwd_dBdC": (20.55e6, "ssd_tc_bcf.cu", "83954d5dd60c3cb17a3a7cab87e111b86a0d66df56ff2025b10429034fd70e24"),
-    "bwd_dx": (17.23e6, "ssd_tc_scan.cu", "0b66fe3c6f3bb9b1cb10be98fafc0e1506fdc30e49957ec586b8f877cadf4b68"),
-    "chunk_scan_fwd": (10.94e6, "ssd_tc_scan.cu", "0b66fe3c6f3bb9b1cb10be98fafc0e1506fdc30e49957ec586b8f877cadf4b68"),
-    "chunk_state": (7.04e6, "ssd_tc.cu", "d08b62291f529092a782772fee2f8222d1a35a5f326c2cc1ac015e6d3ffe95a6"),
-    "dstate_contrib": (7.04e6, "ssd_tc.cu", "d08b62291f529092a782772fee2f8222d1a35a5f326c2cc1ac015e6d3ffe95a6"),
+    "bwd_dBdC": (20.55e6, "ssd_tc_bcf.cu", "859295b23fee1e4bd90f5ad8d9328f5793795a8a7698b9087b2286f5d42b35af"),
+    "bwd_dx": (17.23e6, "ssd_tc_scan.cu", "3ea5757da6501f0ea6a699499461cb3b9279fc57cceda76140ade8c4444a5dcd"),
+    "chunk_scan_fwd": (10.94e6, "ssd_tc_scan.cu", "3ea5757da6501f0ea6a699499461cb3b9279fc57cceda76140ade8c4444a5dcd"),
+    "chunk_state": (7.04e6, "ssd_tc.cu", "476c275026f7e136b96cec13cc7c617ea7c59d6fc34edbe9bc79467efbc16aee"),
+    "dstate_contrib": (7.04e6, "ssd_tc.cu", "476c275026f7e136b96cec13cc7c617ea7c59d6fc34edbe9bc79467efbc16aee"),
 }
 NCU_CFG1_UNITS = 2048 * 24
 
