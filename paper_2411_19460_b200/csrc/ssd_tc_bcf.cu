@@ -190,14 +190,9 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
             issue_scores(0);
             uint32_t scuse = 0;   // uses of the scaled-rows buffer so far
             for (int hi = 0; hi < nheads; ++hi) {
-                // next head's scores as soon as the mask warps have copied this head's out of TMEM
-                if (hi + 1 < nheads) {
-                    mbar_wait(&sempty, hi & 1, abortp, p.status);
-                    tc_fence_after_sync();
-                    issue_scores(hi + 1);
-                }
-                // inter-chunk terms: scaled rows (K = p) times a chunk state.  A tile's first one goes ahead of
-                // the W products (its operand is ready earlier), the second one of tile (1,1) after them.
+                // inter-chunk terms: scaled rows (K = p) times a chunk state.  A tile's first one is published by the
+                // mask warps before they mask the head, so it is issued first: the scaled-rows buffer is free again
+                // by the time tile (1,1) wants it for its second one.
                 auto inter_dC = [&]() {   // dC += (e^{cs_t} dy_t) H_in
                     mbar_wait(&hfull, hi & 1, abortp, p.status);
                     mbar_wait(&scfull, scuse & 1, abortp, p.status);
@@ -228,6 +223,12 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
                 };
                 if (doC) inter_dC();
                 else inter_dB(hi == 0);
+                // next head's scores as soon as the mask warps are done with this head's (they read them last)
+                if (hi + 1 < nheads) {
+                    mbar_wait(&sempty, hi & 1, abortp, p.status);
+                    tc_fence_after_sync();
+                    issue_scores(hi + 1);
+                }
                 if (doC && doB) inter_dB(hi == 0);
                 umma_commit(&rempty[hi & 1]);
             }
