@@ -36,8 +36,8 @@ constexpr uint32_t GF_OFF_SC = 163840;     // 16 KB  scaled rows of an inter-chu
 constexpr uint32_t GF_OFF_ST = 180224;     // 2 x 16 KB  bf16 chunk states (entering: H, gradient leaving: G)
 constexpr uint32_t GF_OFF_VEC = 212992;    // per-head vectors, double buffered
 constexpr uint32_t GF_VEC_FLOATS = 256 * 3 + 64;
-constexpr uint32_t GF_OFF_PART = GF_OFF_VEC + 2 * GF_VEC_FLOATS * 4;   // rho: [2][3][128] ; psi: [2][3][128] floats
-constexpr uint32_t GF_SMEM = GF_OFF_PART + 2 * 2 * 384 * 4 + 1024;
+constexpr uint32_t GF_OFF_PART = GF_OFF_VEC + 2 * GF_VEC_FLOATS * 4;   // [head parity][rho: 4 slices x 128 rows | psi: 4 quarters x 128 cols]
+constexpr uint32_t GF_SMEM = GF_OFF_PART + 2 * 1024 * 4 + 1024;
 
 constexpr uint32_t TF_CB = 0, TF_S = 128, TF_ACCC = 256, TF_ACCB = 384;
 
@@ -65,7 +65,7 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     __shared__ uint64_t bar_ld, bar_cb, rfull[2], rempty[2], sfull, sempty, wfull, scfull, scempty, hfull, hempty,
-        gfull, gempty, accfull, vfull[2], vempty[2];
+        gfull, gempty, accfull, vfull[2], vempty[2], pfull[2], pempty[2];
     __shared__ uint32_t tmem_base, abort_flag;
 
     // 1-D grid: all full tiles first (they have the most mask work), then the two diagonal kinds
@@ -93,6 +93,8 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
             mbar_init(&rempty[i], 1 + 16);    // the head's MMAs (one commit) + the mask warps that scaled its rows
             mbar_init(&vfull[i], 1);
             mbar_init(&vempty[i], 16);
+            mbar_init(&pfull[i], 16);         // the mask warps' partial sums of rho / psi of a head
+            mbar_init(&pempty[i], 1);
         }
         mbar_init(&sfull, 1);
         mbar_init(&sempty, 16);
@@ -258,6 +260,30 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
         // decays, written to a double-buffered area one head ahead of the mask warps.
         if (nheads > 0) {
             float *vec = reinterpret_cast<float *>(smem + GF_OFF_VEC);
+            // rho / psi of a finished head: the mask warps' partial sums added in a fixed order.  Rows of t-block 1
+            // (columns of s-block 0) are covered by two tiles: the second part goes to rhob (psib), and the tile
+            // that has no partner writes a zero there.
+            auto finish_head = [&](int hj) {
+                const int par = hj & 1;
+                const float *pr = reinterpret_cast<const float *>(smem + GF_OFF_PART) + par * 1024;
+                mbar_wait(&pfull[par], (hj >> 1) & 1, abortp, p.status);
+                const size_t vb = (((size_t)b * p.H + h_begin + hj) * p.ncs + c) << 8;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int i = k * 32 + lane;
+                    const float er = ((pr[i] + pr[128 + i]) + pr[256 + i]) + pr[384 + i];
+                    const float ep = ((pr[512 + i] + pr[640 + i]) + pr[768 + i]) + pr[896 + i];
+                    const size_t ro = vb + tb * 128 + i, so = vb + sb * 128 + i;
+                    if (kind == 2) p.rhob[ro] = er;
+                    else p.rho[ro] = er;
+                    if (kind == 1) p.rhob[ro] = 0.f;
+                    if (kind == 0) p.psib[so] = ep;
+                    else p.psi[so] = ep;
+                    if (kind == 2) p.psib[so] = 0.f;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&pempty[par]);
+            };
             for (int hi = 0; hi < nheads; ++hi) {
                 const int buf = hi & 1, h = h_begin + hi;
                 const size_t vo = ((((size_t)b * p.H + h) * p.ncs + c) << 8) + lane * 8;
@@ -288,7 +314,9 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&vfull[buf]);
+                if (hi >= 1) finish_head(hi - 1);
             }
+            finish_head(nheads - 1);
         }
     } else if (nheads > 0) {
         // ------------------------------------------------------------ mask warps
@@ -302,8 +330,6 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
         const int isub = r >> 5;
         const uint32_t tlane = (uint32_t)(q * 32) << 16;
         float *vec = reinterpret_cast<float *>(smem + GF_OFF_VEC);
-        float *part_rho = reinterpret_cast<float *>(smem + GF_OFF_PART);          // [head parity][3][128]
-        float *part_psi = part_rho + 2 * 384;                                     // [head parity][3][128]
         uint32_t scuse = 0;
         float wsum[32];                             // this thread's row of sum_h W_h: columns w * 16 + j of its two slices
 #pragma unroll
@@ -429,35 +455,18 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
             __syncwarp();
             if (lane == 0) mbar_arrive(&rempty[hi & 1]);     // this warp has read the head's rows
 
-            // ---- rho_t: the four column slices of a row meet through shared memory
-            const size_t vbase = (((size_t)b * p.H + h_begin + hi) * p.ncs + c) << 8;
+            // ---- rho_t / psi_s: every warp leaves its partial sums (over its 16-column slice / its 32 rows) in
+            // shared memory; the vector warp adds them in a fixed order and writes them out, so no mask warp waits
+            // for another one here
             {
-                const float dsum = dacc.x + dacc.y;
-                float *pp = part_rho + (hi & 1) * 384;
-                if (quar > 0) pp[(quar - 1) * 128 + rl] = dsum;
-                asm volatile("bar.sync %0, 128;" ::"r"(2 + q) : "memory");
-                if (quar == 0) {
-                    const float e = ((dsum + pp[rl]) + pp[128 + rl]) + pp[256 + rl];
-                    // tile (1,1) holds the second part of the rows of t-block 1; (0,0) has no second part
-                    if (kind == 2) p.rhob[vbase + r] = e;
-                    else p.rho[vbase + r] = e;
-                    if (kind == 1) p.rhob[vbase + r] = 0.f;
-                }
-            }
-            // ---- psi_s: the four row quarters of a column slice meet through shared memory
-            {
-                float *pp = part_psi + (hi & 1) * 384;
+                const int par = hi & 1;
+                float *pr = reinterpret_cast<float *>(smem + GF_OFF_PART) + par * 1024;
+                if (hi >= 2) mbar_wait(&pempty[par], ((hi >> 1) - 1) & 1, abortp, p.status);
+                pr[quar * 128 + rl] = dacc.x + dacc.y;
                 const int lc = (lane >> 4) * 64 + quar * 16 + (lane & 15);     // column of the tile this lane holds
-                if (q > 0) pp[(q - 1) * 128 + lc] = csum;
-                asm volatile("bar.sync %0, 128;" ::"r"(6 + quar) : "memory");
-                if (q == 0) {
-                    const float e = ((csum + pp[lc]) + pp[128 + lc]) + pp[256 + lc];
-                    const size_t so = vbase + sb * 128 + lc;
-                    // tile (1,0) holds the second part of the columns of s-block 0; (1,1) has no second part
-                    if (kind == 0) p.psib[so] = e;
-                    else p.psi[so] = e;
-                    if (kind == 2) p.psib[so] = 0.f;
-                }
+                pr[512 + q * 128 + lc] = csum;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&pfull[par]);
             }
         }
 
