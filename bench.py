@@ -237,6 +237,8 @@ def run_ours(args):
         return run_stream(args, rep, dev)
     if args.conv:
         return run_conv(args, rep, dev)
+    if args.gated_norm:
+        return run_gated_norm(args, rep, dev)
     if cfg.layers != 1:
         return run_stack(args, rep, dev)
     seg = args.seg or cfg.seg
@@ -679,6 +681,91 @@ def run_conv(args, rep, dev):
     rep.close()
 
 
+def run_gated_norm(args, rep, dev):
+    """The gated RMS normalisation behind the SSD layer, forward and backward segment by segment (token-local: nothing
+    is carried across the cuts; dgamma is summed over the segments)."""
+    from paper_2411_19460_b200 import libssd
+
+    cfg = CONFIGS[args.config]
+    seg = args.seg or cfg.seg
+    B, L, D = cfg.B, cfg.L, cfg.H * cfg.P
+    group = D // cfg.G
+    td = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    gen = torch.Generator(device=dev).manual_seed(cfg.seed + rep.rank)
+    y = torch.randn(B * L, D, generator=gen, device=dev, dtype=torch.float32).to(td)
+    z = torch.randn(B * L, D, generator=gen, device=dev, dtype=torch.float32).to(td)
+    g = torch.randn(B * L, D, generator=gen, device=dev, dtype=torch.float32).to(td)
+    gamma = 1.0 + 0.1 * torch.randn(D, generator=gen, device=dev)
+    out, dy, dz = torch.empty_like(y), torch.empty_like(y), torch.empty_like(y)
+    dg = torch.zeros(D, device=dev)
+    rows = B * seg
+    nseg = (B * L) // rows
+    ws = torch.empty(int(libssd.lib().ssd_gated_norm_workspace_bytes(rows, D)), dtype=torch.uint8, device=dev)
+    sl = [slice(k * rows, (k + 1) * rows) for k in range(nseg)]
+    stream = torch.cuda.current_stream()
+
+    def step():
+        for k in range(nseg):
+            libssd.ssd_gated_norm_fwd(y[sl[k]], z[sl[k]], gamma, group=group, out=out[sl[k]], stream=stream)
+        dg.zero_()
+        for k in range(nseg - 1, -1, -1):
+            libssd.ssd_gated_norm_bwd(y[sl[k]], z[sl[k]], gamma, g[sl[k]], group=group, dy=dy[sl[k]], dz=dz[sl[k]], dgamma=dg,
+                                      accumulate=True, ws=ws, stream=stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    rep.barrier()
+    run_step, per_replay = step, None
+    if args.graph:
+        side = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(side):
+            stream = torch.cuda.current_stream()
+            step()
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            nc0 = libssd.launch_count()
+            with torch.cuda.graph(graph, stream=side):
+                step()
+            per_replay = libssd.launch_count() - nc0
+        stream = torch.cuda.current_stream()
+        torch.cuda.synchronize()
+        run_step = graph.replay
+        for _ in range(3):
+            run_step()
+    sampler = ClockSampler(dev) if rep.rank == 0 else None
+    n0 = libssd.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rep.barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        run_step()
+    e1.record(stream)
+    rep.barrier()
+    ms = rep.max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    launches = per_replay * args.steps if per_replay is not None else libssd.launch_count() - n0
+    clocks = sampler.stop() if sampler else None
+    if rep.rank != 0:
+        rep.close()
+        return
+    peaks = load_peaks()
+    e = y.element_size()
+    ach = 8 * e * D * B * L / (ms * 1e-3) / 1e9           # fwd: y, z in, out out; bwd: y, z, dout in, dy, dz out
+    line = {
+        "metric": "gated_norm_fwd_bwd_segmented_tokens_per_s", "value": rep.world * B * L / (ms * 1e-3), "unit": UNIT,
+        "n_gpus": rep.world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+        "impl": "ours",
+        "config": {"workload": cfg.name + "_gated_norm", "B": B, "L": L, "channels": D, "group": group, "seg": seg,
+                   "nseg": nseg, "launch": "cuda graph replay" if args.graph else "stream launches",
+                   "l2": "inputs larger than L2", "parallelism": "replicas" if rep.world > 1 else "single"},
+        "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+        "roofline": {"kernel": "gated_norm fwd+bwd", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]},
+    }
+    print(json.dumps(line))
+    rep.close()
+
+
 # ----------------------------------------------------------------------------- the CPU oracle legs
 def _oracle_sample(cfg, inp, sample_tokens):
     """fp64 host copies of the first `sample_tokens` tokens (all heads) of the workload."""
@@ -750,6 +837,8 @@ def main():
     ap.add_argument("--stream-len", type=int, default=0, help="forward-only streaming over this many tokens "
                     "(e.g. 2097152) instead of the training step")
     ap.add_argument("--conv", action="store_true", help="time the depthwise conv + SiLU stage (forward + backward, "
+                    "segment by segment) instead of the SSD step")
+    ap.add_argument("--gated-norm", action="store_true", help="time the gated RMS normalisation stage (forward + backward, "
                     "segment by segment) instead of the SSD step")
     ap.add_argument("--layers", type=int, default=0, help="config 3: number of layers (default 64)")
     ap.add_argument("--no-graph", dest="graph", action="store_false",

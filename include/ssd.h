@@ -220,6 +220,24 @@ int ssd_conv_bwd(int B, int L, int C, int dtype, const void *u, long long u_bstr
                  float *dbias, int accumulate, void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * Gated RMS normalisation, the stage behind the SSD layer in a Mamba-2 block:
+ *     v = y * silu(z) ,   out = v * rsqrt(mean(v^2) + eps) * gamma
+ * with the mean over groups of `group` adjacent channels (D % group == 0, group % 4 == 0, group <= 8192; group = D
+ * normalises the whole row).  Token-local: a segment is a range of rows and nothing is carried across a cut.
+ *   y, z, out, dout, dy, dz  [rows, D] dense, I/O dtype (rows = B * L of the segment);  gamma, dgamma [D] fp32
+ * ssd_gated_norm_bwd writes dy, dz and dgamma (added to when `accumulate` != 0: sum over segments); `ws` holds
+ * ssd_gated_norm_workspace_bytes(rows, D) bytes of per-tile partial sums of dgamma, 256-byte aligned, added in a fixed
+ * order (deterministic).  Device pointers, enqueued on `stream`.  Returns SSD_OK or SSD_EINVAL / SSD_EUNSUPPORTED /
+ * SSD_EALIGN / SSD_EWORKSPACE / SSD_EDEVICE / SSD_ECUDA.
+ */
+size_t ssd_gated_norm_workspace_bytes(long long rows, int D);
+int ssd_gated_norm_fwd(long long rows, int D, int group, int dtype, const void *y, const void *z, const float *gamma, float eps,
+                       void *out, void *stream);
+int ssd_gated_norm_bwd(long long rows, int D, int group, int dtype, const void *y, const void *z, const float *gamma, float eps,
+                       const void *dout, void *dy, void *dz, float *dgamma, int accumulate, void *ws, size_t ws_bytes,
+                       void *stream);
+
+/*
  * Reads the status word at the start of `ws` (device memory) with a blocking copy: call it after
  * synchronising the stream.  Returns SSD_OK, SSD_ETIMEOUT if some kernel abandoned a bounded wait
  * (its outputs are then undefined), or SSD_ECUDA if the copy failed.

@@ -144,3 +144,33 @@ def conv_bwd(u, w, bias, state_in, dout, dtail=None):
     if dtail is not None:
         du[:, L - 3:, :] += _f64(dtail)
     return du, dext[:, :3, :].copy(), dw, dpre.sum(axis=(0, 1))
+
+
+def gated_norm_fwd(y, z, gamma, group=None, eps=1e-5):
+    """v = y * silu(z); out = v / sqrt(mean(v^2 over each group of `group` channels) + eps) * gamma (fp64).
+    Returns (out, v, rstd [..., D/group])."""
+    y, z, gamma = map(_f64, (y, z, gamma))
+    D = y.shape[-1]
+    group = D if group is None else group
+    v = y * z / (1.0 + np.exp(-z))
+    vg = v.reshape(v.shape[:-1] + (D // group, group))
+    rstd = 1.0 / np.sqrt((vg * vg).mean(axis=-1) + eps)
+    out = (vg * rstd[..., None]).reshape(v.shape) * gamma
+    return out, v, rstd
+
+
+def gated_norm_bwd(y, z, gamma, dout, group=None, eps=1e-5):
+    """Gradients of Loss = <out, dout>: dy, dz, dgamma (fp64)."""
+    y, z, gamma, dout = map(_f64, (y, z, gamma, dout))
+    D = y.shape[-1]
+    group = D if group is None else group
+    _, v, rstd = gated_norm_fwd(y, z, gamma, group, eps)
+    sh = v.shape[:-1] + (D // group, group)
+    xh = v.reshape(sh) * rstd[..., None]
+    dvh = (dout * gamma).reshape(sh)
+    dv = (rstd[..., None] * (dvh - xh * (dvh * xh).mean(axis=-1, keepdims=True))).reshape(v.shape)
+    sg = 1.0 / (1.0 + np.exp(-z))
+    dy = dv * z * sg
+    dz = dv * y * sg * (1.0 + z * (1.0 - sg))
+    dgamma = (dout * xh.reshape(v.shape)).reshape(-1, D).sum(axis=0)
+    return dy, dz, dgamma

@@ -24,7 +24,7 @@ static size_t g_prof_used = 0;
 
 static const char *const kKindNames[KIND_COUNT] = {
     "chunk_cumsum", "chunk_state", "state_pass_fwd", "chunk_scan_fwd", "dstate_contrib",
-    "state_pass_bwd", "bwd_dx", "bwd_dC", "bwd_dB", "bwd_finish", "reduce_dBdC", "final_dAdD", "glue", "decode_step", "bwd_dBdC", "conv1d"};
+    "state_pass_bwd", "bwd_dx", "bwd_dC", "bwd_dB", "bwd_finish", "reduce_dBdC", "final_dAdD", "glue", "decode_step", "bwd_dBdC", "conv1d", "gated_norm"};
 
 static ProfEvent *prof_begin(int kind, cudaStream_t st) {
     if (!g_prof_on) return nullptr;
@@ -673,6 +673,50 @@ int ssd_conv_bwd(int B, int L, int C, int dtype, const void *u, long long u_bstr
     cudaStream_t st = (cudaStream_t)stream;
     SSD_LAUNCH(KIND_CONV, launch_conv_bwd(dtype, u, bs, w, bias, state_in, dout, dtail, du, dstate, dw, dbias,
                                           accumulate ? 1 : 0, (float *)ws, B, L, C, st));
+    return SSD_OK;
+}
+
+static int norm_check(long long rows, int D, int group, int dtype) {
+    if (rows <= 0 || D <= 0 || group <= 0 || (D % group) || (group % 4)) return SSD_EINVAL;
+    if (group > gated_norm_max_group() || gated_norm_tiles(rows) > 2147483647ll || D / group > 65535) return SSD_EUNSUPPORTED;
+    if (dtype != SSD_DTYPE_F32 && dtype != SSD_DTYPE_BF16) return SSD_EUNSUPPORTED;
+    if (((size_t)D * (dtype == SSD_DTYPE_BF16 ? 2 : 4)) % 16) return SSD_EALIGN;
+    return SSD_OK;
+}
+
+size_t ssd_gated_norm_workspace_bytes(long long rows, int D) {
+    if (rows <= 0 || D <= 0) return 0;
+    return (size_t)gated_norm_tiles(rows) * D * sizeof(float);
+}
+
+int ssd_gated_norm_fwd(long long rows, int D, int group, int dtype, const void *y, const void *z, const float *gamma, float eps,
+                       void *out, void *stream) {
+    int rc = norm_check(rows, D, group, dtype);
+    if (rc) return rc;
+    if (!y || !z || !gamma || !out) return SSD_EINVAL;
+    if (misaligned(y) || misaligned(z) || misaligned(gamma) || misaligned(out)) return SSD_EALIGN;
+    rc = check_device();
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    SSD_LAUNCH(KIND_NORM, launch_gated_norm_fwd(dtype, y, z, gamma, eps, out, rows, D, group, st));
+    return SSD_OK;
+}
+
+int ssd_gated_norm_bwd(long long rows, int D, int group, int dtype, const void *y, const void *z, const float *gamma, float eps,
+                       const void *dout, void *dy, void *dz, float *dgamma, int accumulate, void *ws, size_t ws_bytes,
+                       void *stream) {
+    int rc = norm_check(rows, D, group, dtype);
+    if (rc) return rc;
+    if (!y || !z || !gamma || !dout || !dy || !dz || !dgamma || !ws) return SSD_EINVAL;
+    if (misaligned(y) || misaligned(z) || misaligned(gamma) || misaligned(dout) || misaligned(dy) || misaligned(dz) ||
+        misaligned(dgamma))
+        return SSD_EALIGN;
+    if (((uintptr_t)ws & 255u) || ws_bytes < ssd_gated_norm_workspace_bytes(rows, D)) return SSD_EWORKSPACE;
+    rc = check_device();
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    SSD_LAUNCH(KIND_NORM, launch_gated_norm_bwd(dtype, y, z, gamma, eps, dout, dy, dz, dgamma, accumulate ? 1 : 0, (float *)ws,
+                                                rows, D, group, st));
     return SSD_OK;
 }
 

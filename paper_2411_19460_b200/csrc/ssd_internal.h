@@ -107,6 +107,14 @@ cudaError_t launch_conv_fwd(int dtype, const void *u, long long u_bs, const floa
 cudaError_t launch_conv_bwd(int dtype, const void *u, long long u_bs, const float *w, const float *bias,
                             const void *state_in, const void *dout, const float *dtail, void *du, float *dstate,
                             float *dw, float *dbias, int accumulate, float *part, int B, int L, int C, cudaStream_t st);
+// ssd_norm.cu : gated RMS normalisation behind the SSD layer
+long long gated_norm_tiles(long long rows);
+int gated_norm_max_group();
+cudaError_t launch_gated_norm_fwd(int dtype, const void *y, const void *z, const float *gamma, float eps, void *out,
+                                  long long rows, int D, int group, cudaStream_t st);
+cudaError_t launch_gated_norm_bwd(int dtype, const void *y, const void *z, const float *gamma, float eps, const void *dout,
+                                  void *dy, void *dz, float *dgamma, int accumulate, float *part, long long rows, int D,
+                                  int group, cudaStream_t st);
 // ssd_decode.cu : one token of the recurrence, state updated in place
 cudaError_t launch_decode_step(int dtype, int N, const void *x, const float *dt, const float *A, const void *Bm,
                                const void *Cm, const float *D, float *h, void *y, int B, int H, int P, int G,
@@ -135,7 +143,7 @@ enum { STATE_MODE_FWD = 0, STATE_MODE_DSTATE = 1 };
 enum {
     KIND_CUMSUM = 0, KIND_CHUNK_STATE, KIND_STATE_PASS_FWD, KIND_SCAN_FWD, KIND_DSTATE,
     KIND_STATE_PASS_BWD, KIND_BWD_DX, KIND_BWD_DC, KIND_BWD_DB, KIND_BWD_FINISH, KIND_REDUCE_DBDC,
-    KIND_FINAL, KIND_GLUE, KIND_DECODE, KIND_BWD_DBDC, KIND_CONV, KIND_COUNT
+    KIND_FINAL, KIND_GLUE, KIND_DECODE, KIND_BWD_DBDC, KIND_CONV, KIND_NORM, KIND_COUNT
 };
 enum { MP_FWD = 0, MP_BWD_DX = 1, MP_DC = 2, MP_DB = 3 };
 

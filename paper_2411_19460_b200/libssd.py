@@ -26,7 +26,7 @@ EXPORTS = ["ssd_workspace_bytes", "ssd_boundary_bytes", "ssd_fwd", "ssd_fwd_segm
            "ssd_last_cuda_error", "ssd_launch_count", "ssd_kernel_kinds", "ssd_kernel_name",
            "ssd_profile", "ssd_profile_read", "ssd_fwd_static_ws", "ssd_glue_fwd", "ssd_glue_bwd",
            "ssd_glue_residual", "ssd_decode_step", "ssd_conv_fwd", "ssd_conv_bwd",
-           "ssd_conv_workspace_bytes"]
+           "ssd_conv_workspace_bytes", "ssd_gated_norm_fwd", "ssd_gated_norm_bwd", "ssd_gated_norm_workspace_bytes"]
 
 
 class SSDShape(ctypes.Structure):
@@ -80,6 +80,13 @@ def lib():
         L.ssd_conv_fwd.argtypes = [ci, ci, ci, ci, vp, ll, fp, fp, vp, vp, vp, vp]
         L.ssd_conv_bwd.restype = ctypes.c_int
         L.ssd_conv_bwd.argtypes = [ci, ci, ci, ci, vp, ll, fp, fp, vp, vp, fp, vp, fp, fp, fp, ci, vp, ctypes.c_size_t, vp]
+        cf = ctypes.c_float
+        L.ssd_gated_norm_workspace_bytes.restype = ctypes.c_size_t
+        L.ssd_gated_norm_workspace_bytes.argtypes = [ll, ci]
+        L.ssd_gated_norm_fwd.restype = ctypes.c_int
+        L.ssd_gated_norm_fwd.argtypes = [ll, ci, ci, ci, vp, vp, fp, cf, vp, vp]
+        L.ssd_gated_norm_bwd.restype = ctypes.c_int
+        L.ssd_gated_norm_bwd.argtypes = [ll, ci, ci, ci, vp, vp, fp, cf, vp, vp, vp, fp, ci, vp, ctypes.c_size_t, vp]
         L.ssd_decode_step.restype = ctypes.c_int
         L.ssd_decode_step.argtypes = [sp, vp, fp, fp, vp, vp, fp, fp, vp, vp]
         L.ssd_glue_residual.restype = ctypes.c_int
@@ -326,6 +333,46 @@ def ssd_conv_bwd(u, w, bias, state_in, dout, dtail=None, *, du=None, dstate=None
     if rc != SSD_OK:
         raise SSDError(rc, "ssd_conv_bwd")
     return du, dstate, dw, dbias
+
+
+def _norm_args(y):
+    if y.dtype == torch.bfloat16:
+        code = SSD_DTYPE_BF16
+    elif y.dtype == torch.float32:
+        code = SSD_DTYPE_F32
+    else:
+        raise TypeError("y must be float32 or bfloat16")
+    if not y.is_cuda or not y.is_contiguous():
+        raise ValueError("y must be a contiguous CUDA tensor [..., D]")
+    D = y.shape[-1]
+    return y.numel() // D, D, code
+
+
+def ssd_gated_norm_fwd(y, z, gamma, *, group=None, eps=1e-5, out=None, stream=None):
+    """out = RMSNorm(y * silu(z)) * gamma over groups of `group` channels (default: the whole last dimension)."""
+    rows, D, code = _norm_args(y)
+    out = torch.empty_like(y) if out is None else out
+    rc = lib().ssd_gated_norm_fwd(rows, D, D if group is None else int(group), code, _ptr(y), _ptr(z), _ptr(gamma), float(eps),
+                                  _ptr(out), _stream(stream))
+    if rc != SSD_OK:
+        raise SSDError(rc, "ssd_gated_norm_fwd")
+    return out
+
+
+def ssd_gated_norm_bwd(y, z, gamma, dout, *, group=None, eps=1e-5, dy=None, dz=None, dgamma=None, accumulate=False, ws=None,
+                       stream=None):
+    rows, D, code = _norm_args(y)
+    dy = torch.empty_like(y) if dy is None else dy
+    dz = torch.empty_like(y) if dz is None else dz
+    dgamma = torch.zeros(D, dtype=torch.float32, device=y.device) if dgamma is None else dgamma
+    nws = int(lib().ssd_gated_norm_workspace_bytes(rows, D))
+    ws = torch.empty(nws, dtype=torch.uint8, device=y.device) if ws is None else ws
+    rc = lib().ssd_gated_norm_bwd(rows, D, D if group is None else int(group), code, _ptr(y), _ptr(z), _ptr(gamma), float(eps),
+                                  _ptr(dout), _ptr(dy), _ptr(dz), _ptr(dgamma), 1 if accumulate else 0, _ptr(ws), ws.numel(),
+                                  _stream(stream))
+    if rc != SSD_OK:
+        raise SSDError(rc, "ssd_gated_norm_bwd")
+    return dy, dz, dgamma
 
 
 def _glue_shape(t):
