@@ -30,6 +30,9 @@ CASES = {
     "bf16_q128_h8": small("bf16", chunk=128, seg=384, L=1152, H=8, G=4),
     "bf16_stiff": small("bf16", a_max=64.0, dt_lo=1e-4, dt_hi=1.0, L=2048, seg=1024, H=8, G=2),
     "bf16_one_segment": small("bf16", seg=1024),
+    # head counts of the other two model sizes of Appendix C's table (d_inner 2048 and 4096: 32 and 64 heads)
+    "bf16_h32": small("bf16", H=32, L=512, seg=256),
+    "bf16_h64_g8": small("bf16", H=64, G=8, L=512, seg=512),
 }
 
 
