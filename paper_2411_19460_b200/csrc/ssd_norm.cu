@@ -5,14 +5,18 @@
 // every tensor is read once; the sums over a row meet through warp shuffles and shared memory in a fixed order; the
 // gradient of gamma is accumulated per CTA over its rows and added over the tiles by a second kernel (no atomics).
 #include "ssd_internal.h"
+#include "ssd_sm100.cuh"
 
 namespace ssd {
+
+using namespace sm100;
 
 namespace {
 
 constexpr int GN_THREADS = 256;
 constexpr int GN_MAXV = 8;        // four-channel vectors per thread, at most (the kernels are instantiated for 1, 2, 4, 5 and 8)
-constexpr int GN_ROWS = 4;        // rows per CTA
+constexpr int GN_ROWS = 16;       // rows per CTA
+constexpr int GN_STAGES = 3;      // rows in flight per CTA in the staged kernels
 
 template <typename T> __device__ __forceinline__ void gld4(const T *p, float *f);
 template <> __device__ __forceinline__ void gld4<float>(const float *p, float *f) {
@@ -174,6 +178,135 @@ __global__ void __launch_bounds__(GN_THREADS, NV <= 5 ? 2 : 1) k_gated_norm_bwd(
     }
 }
 
+// ---- staged variants: the rows of a CTA's tile stream through a ring of GN_STAGES shared-memory buffers filled by
+// bulk async copies (one per tensor and row: the channels of a group are contiguous), so that several rows per CTA
+// are in flight without holding them in registers; the arithmetic then reads a row from shared memory as often as
+// it needs to.  Used when the ring fits (bf16 rows of the model sizes do); otherwise the kernels above.
+template <typename T, int NV, bool BWD>
+__global__ void __launch_bounds__(GN_THREADS, 2) k_gated_norm_staged(const T *y, const T *z, const float *gamma, float eps,
+                                                                     const T *dout, T *out_or_dy, T *dz, float *part,
+                                                                     long long rows, int D, int group) {
+    extern __shared__ __align__(128) unsigned char gn_smem[];
+    __shared__ float red[GN_THREADS / 32];
+    __shared__ uint64_t full[GN_STAGES];
+    __shared__ uint32_t abort_flag;
+    __shared__ unsigned int status_dummy;
+    constexpr int NT = BWD ? 3 : 2;                       // tensors staged per row
+    const int gi = blockIdx.y, nv = group / 4;
+    const long long r0 = (long long)blockIdx.x * GN_ROWS;
+    const int nrows = (int)min((long long)GN_ROWS, rows - r0);
+    const uint32_t row_bytes = (uint32_t)group * sizeof(T);
+    T *ring = reinterpret_cast<T *>(gn_smem);             // [GN_STAGES][NT][group]
+    auto issue = [&](int j) {                             // thread 0: row r0 + j into stage j % GN_STAGES
+        const int st = j % GN_STAGES;
+        const size_t base = (size_t)(r0 + j) * D + (size_t)gi * group;
+        T *dst = ring + (size_t)st * NT * group;
+        mbar_arrive_expect_tx(&full[st], NT * row_bytes);
+        bulk_load(dst, y + base, row_bytes, &full[st]);
+        bulk_load(dst + group, z + base, row_bytes, &full[st]);
+        if (BWD) bulk_load(dst + 2 * (size_t)group, dout + base, row_bytes, &full[st]);
+    };
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < GN_STAGES; ++i) mbar_init(&full[i], 1);
+        abort_flag = 0;
+        status_dummy = 0;
+        fence_barrier_init();
+        for (int j = 0; j < GN_STAGES - 1 && j < nrows; ++j) issue(j);
+    }
+    float gm[NV][4], dg[NV][4];
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+        const int i = threadIdx.x + k * GN_THREADS;
+        if (i < nv) gld4(gamma + (size_t)gi * group + (size_t)i * 4, gm[k]);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) dg[k][e] = 0.f;
+    }
+    __syncthreads();
+    for (int j = 0; j < nrows; ++j) {
+        // the stage that row j + GN_STAGES - 1 goes to was read in iteration j - 1, which ended with a CTA barrier
+        if (threadIdx.x == 0 && j + GN_STAGES - 1 < nrows) issue(j + GN_STAGES - 1);
+        const int st = j % GN_STAGES;
+        mbar_wait(&full[st], (uint32_t)(j / GN_STAGES) & 1u, &abort_flag, &status_dummy);
+        const T *sy = ring + (size_t)st * NT * group, *sz = sy + group, *sg = sy + 2 * (size_t)group;
+        const size_t base = (size_t)(r0 + j) * D + (size_t)gi * group;
+        float v[NV][4];
+        float ss = 0.f;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int i = threadIdx.x + k * GN_THREADS;
+            if (i < nv) {
+                float a[4], b[4];
+                gld4(sy + (size_t)i * 4, a);
+                gld4(sz + (size_t)i * 4, b);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    v[k][e] = a[e] * b[e] * sigmoid_gn(b[e]);
+                    ss = fmaf(v[k][e], v[k][e], ss);
+                }
+            }
+        }
+        const float n = rsqrtf(block_sum(ss, red) / (float)group + eps);
+        if (!BWD) {
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int i = threadIdx.x + k * GN_THREADS;
+                if (i < nv) {
+                    float o[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) o[e] = v[k][e] * n * gm[k][e];
+                    gst4(out_or_dy + base + (size_t)i * 4, o);
+                }
+            }
+        } else {
+            // xh = v n ;  dvh = dout gamma ;  c = mean(dvh xh) ;  dv = n (dvh - xh c)
+            float dot = 0.f;
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int i = threadIdx.x + k * GN_THREADS;
+                if (i < nv) {
+                    float g[4];
+                    gld4(sg + (size_t)i * 4, g);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float xh = v[k][e] * n;
+                        dg[k][e] = fmaf(g[e], xh, dg[k][e]);
+                        dot = fmaf(g[e] * gm[k][e], xh, dot);
+                    }
+                }
+            }
+            const float cmean = block_sum(dot, red) / (float)group;
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int i = threadIdx.x + k * GN_THREADS;
+                if (i < nv) {
+                    float a[4], b[4], g[4], oy[4], oz[4];
+                    gld4(sy + (size_t)i * 4, a);
+                    gld4(sz + (size_t)i * 4, b);
+                    gld4(sg + (size_t)i * 4, g);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float xh = v[k][e] * n;
+                        const float dv = n * fmaf(-xh, cmean, g[e] * gm[k][e]);
+                        const float sgm = sigmoid_gn(b[e]);
+                        oy[e] = dv * b[e] * sgm;
+                        oz[e] = dv * a[e] * sgm * fmaf(b[e], 1.f - sgm, 1.f);
+                    }
+                    gst4(out_or_dy + base + (size_t)i * 4, oy);
+                    gst4(dz + base + (size_t)i * 4, oz);
+                }
+            }
+        }
+        __syncthreads();                                  // every thread is done with stage `st`
+    }
+    if (BWD) {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int i = threadIdx.x + k * GN_THREADS;
+            if (i < nv) gst4(part + (size_t)blockIdx.x * D + (size_t)gi * group + (size_t)i * 4, dg[k]);
+        }
+    }
+}
+
 __global__ void __launch_bounds__(128) k_gated_norm_reduce(const float *part, float *dgamma, int D, int ntiles, int accumulate) {
     const int c = blockIdx.x * 128 + threadIdx.x;
     if (c >= D) return;
@@ -192,6 +325,19 @@ static cudaError_t norm_fwd_t(const T *y, const T *z, const float *gamma, float 
                               cudaStream_t st) {
     dim3 grid((unsigned)gated_norm_tiles(rows), D / group);
     const int need = (group / 4 + GN_THREADS - 1) / GN_THREADS;
+    const size_t ring = (size_t)GN_STAGES * 2 * group * sizeof(T);
+    if (ring <= 100 * 1024 && need <= 5 && ((size_t)group * sizeof(T)) % 16 == 0) {
+#define GN_SCASE(NV)                                                                                                   \
+    do {                                                                                                               \
+        cudaError_t e = cudaFuncSetAttribute(k_gated_norm_staged<T, NV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ring); \
+        if (e != cudaSuccess) return e;                                                                                \
+        k_gated_norm_staged<T, NV, false><<<grid, GN_THREADS, ring, st>>>(y, z, gamma, eps, (const T *)nullptr, out, (T *)nullptr, \
+                                                                          (float *)nullptr, rows, D, group);            \
+    } while (0)
+        if (need <= 1) GN_SCASE(1); else if (need <= 2) GN_SCASE(2); else if (need <= 4) GN_SCASE(4); else GN_SCASE(5);
+#undef GN_SCASE
+        return cudaGetLastError();
+    }
 #define GN_CASE(NV) k_gated_norm_fwd<T, NV><<<grid, GN_THREADS, 0, st>>>(y, z, gamma, eps, out, rows, D, group)
     if (need <= 1) GN_CASE(1); else if (need <= 2) GN_CASE(2); else if (need <= 4) GN_CASE(4); else if (need <= 5) GN_CASE(5); else GN_CASE(8);
 #undef GN_CASE
@@ -202,6 +348,18 @@ static cudaError_t norm_bwd_t(const T *y, const T *z, const float *gamma, float 
                               long long rows, int D, int group, cudaStream_t st) {
     dim3 grid((unsigned)gated_norm_tiles(rows), D / group);
     const int need = (group / 4 + GN_THREADS - 1) / GN_THREADS;
+    const size_t ring = (size_t)GN_STAGES * 3 * group * sizeof(T);
+    if (ring <= 100 * 1024 && need <= 5 && ((size_t)group * sizeof(T)) % 16 == 0) {
+#define GN_SCASE(NV)                                                                                                   \
+    do {                                                                                                               \
+        cudaError_t e = cudaFuncSetAttribute(k_gated_norm_staged<T, NV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ring); \
+        if (e != cudaSuccess) return e;                                                                                \
+        k_gated_norm_staged<T, NV, true><<<grid, GN_THREADS, ring, st>>>(y, z, gamma, eps, dout, dy, dz, part, rows, D, group); \
+    } while (0)
+        if (need <= 1) GN_SCASE(1); else if (need <= 2) GN_SCASE(2); else if (need <= 4) GN_SCASE(4); else GN_SCASE(5);
+#undef GN_SCASE
+        return cudaGetLastError();
+    }
 #define GN_CASE(NV) k_gated_norm_bwd<T, NV><<<grid, GN_THREADS, 0, st>>>(y, z, gamma, eps, dout, dy, dz, part, rows, D, group)
     if (need <= 1) GN_CASE(1); else if (need <= 2) GN_CASE(2); else if (need <= 4) GN_CASE(4); else if (need <= 5) GN_CASE(5); else GN_CASE(8);
 #undef GN_CASE
