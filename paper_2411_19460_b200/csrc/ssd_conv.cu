@@ -201,6 +201,7 @@ __global__ void __launch_bounds__(CV_THREADS) k_conv_bwd(const T *u, long long u
     ld4(spu + 512, x1);
     ld4(spu + 1024, x2);
     const int ns = (int)(s_end - t_begin), nt = (int)(t_end - t_begin);
+#pragma unroll 4
     for (int j = 0; j < ns + 3; ++j) {                     // s = t_begin + j
         float dp[CV_CH];
         if (j < ns) {
@@ -310,20 +311,33 @@ __global__ void __launch_bounds__(CV_THREADS) k_conv_dstate(const T *u, long lon
     st4(ds + (size_t)2 * C, e);
 }
 
-// dw[c][k], dbias[c]: the tile partials added in tile order (then batch order), in fp64
-__global__ void __launch_bounds__(128) k_conv_reduce(const float *part, float *dw, float *dbias, int C, int ntiles, int B,
+// dw[c][k], dbias[c] from the tile partials, in fp64 and in a fixed order: a CTA owns 32 adjacent channels of one of the
+// five rows (four taps, bias); its eight warps take the tiles round-robin (coalesced 128-byte reads, several in flight),
+// then the eight partial sums are added in warp order.
+__global__ void __launch_bounds__(256) k_conv_reduce(const float *part, float *dw, float *dbias, int C, int ntiles, int B,
                                                      int accumulate) {
-    const int idx = blockIdx.x * 128 + threadIdx.x;      // (k, c), k = 0..4
-    if (idx >= 5 * C) return;
-    const int k = idx / C, c = idx % C;
+    __shared__ double red[8][32];
+    const int lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
+    const int nblk = (C + 31) / 32;
+    const int k = blockIdx.x / nblk, c = (blockIdx.x % nblk) * 32 + lane;
     double s = 0.0;
-    for (int b = 0; b < B; ++b)
-        for (int t = 0; t < ntiles; ++t) s += (double)part[(((size_t)b * ntiles + t) * 5 + k) * C + c];
-    if (k < 4) {
-        float *d = dw + (size_t)c * 4 + k;
-        *d = accumulate ? *d + (float)s : (float)s;
-    } else {
-        dbias[c] = accumulate ? dbias[c] + (float)s : (float)s;
+    if (c < C) {
+        const long long total = (long long)B * ntiles;
+#pragma unroll 4
+        for (long long t = wp; t < total; t += 8) s += (double)part[((size_t)t * 5 + k) * C + c];
+    }
+    red[wp][lane] = s;
+    __syncthreads();
+    if (wp == 0 && c < C) {
+        double tot = 0.0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) tot += red[i][lane];
+        if (k < 4) {
+            float *d = dw + (size_t)c * 4 + k;
+            *d = accumulate ? *d + (float)tot : (float)tot;
+        } else {
+            dbias[c] = accumulate ? dbias[c] + (float)tot : (float)tot;
+        }
     }
 }
 
@@ -380,7 +394,7 @@ cudaError_t launch_conv_bwd(int dtype, const void *u, long long u_bs, const floa
         e = conv_bwd_t<__nv_bfloat16>((const __nv_bfloat16 *)u, u_bs, w, bias, (const __nv_bfloat16 *)state_in,
                                       (const __nv_bfloat16 *)dout, dtail, (__nv_bfloat16 *)du, dstate, part, B, L, C, st);
     if (e != cudaSuccess) return e;
-    k_conv_reduce<<<(5 * C + 127) / 128, 128, 0, st>>>(part, dw, dbias, C, conv_tiles(L), B, accumulate);
+    k_conv_reduce<<<5 * ((C + 31) / 32), 256, 0, st>>>(part, dw, dbias, C, conv_tiles(L), B, accumulate);
     return cudaGetLastError();
 }
 
