@@ -307,12 +307,25 @@ __global__ void __launch_bounds__(GN_THREADS, 2) k_gated_norm_staged(const T *y,
     }
 }
 
-__global__ void __launch_bounds__(128) k_gated_norm_reduce(const float *part, float *dgamma, int D, int ntiles, int accumulate) {
-    const int c = blockIdx.x * 128 + threadIdx.x;
-    if (c >= D) return;
+// dgamma from the tile partials, in fp64 and in a fixed order: a CTA owns 32 adjacent channels; its eight warps take the
+// tiles round-robin (coalesced reads, several in flight), then the eight partial sums are added in warp order.
+__global__ void __launch_bounds__(256) k_gated_norm_reduce(const float *part, float *dgamma, int D, int ntiles, int accumulate) {
+    __shared__ double red[8][32];
+    const int lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
+    const int c = blockIdx.x * 32 + lane;
     double s = 0.0;
-    for (int t = 0; t < ntiles; ++t) s += (double)part[(size_t)t * D + c];
-    dgamma[c] = accumulate ? dgamma[c] + (float)s : (float)s;
+    if (c < D) {
+#pragma unroll 4
+        for (int t = wp; t < ntiles; t += 8) s += (double)part[(size_t)t * D + c];
+    }
+    red[wp][lane] = s;
+    __syncthreads();
+    if (wp == 0 && c < D) {
+        double tot = 0.0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) tot += red[i][lane];
+        dgamma[c] = accumulate ? dgamma[c] + (float)tot : (float)tot;
+    }
 }
 
 }  // namespace
@@ -384,7 +397,7 @@ cudaError_t launch_gated_norm_bwd(int dtype, const void *y, const void *z, const
         e = norm_bwd_t<__nv_bfloat16>((const __nv_bfloat16 *)y, (const __nv_bfloat16 *)z, gamma, eps, (const __nv_bfloat16 *)dout,
                                       (__nv_bfloat16 *)dy, (__nv_bfloat16 *)dz, part, rows, D, group, st);
     if (e != cudaSuccess) return e;
-    k_gated_norm_reduce<<<(D + 127) / 128, 128, 0, st>>>(part, dgamma, D, (int)gated_norm_tiles(rows), accumulate);
+    k_gated_norm_reduce<<<(D + 31) / 32, 256, 0, st>>>(part, dgamma, D, (int)gated_norm_tiles(rows), accumulate);
     return cudaGetLastError();
 }
 
