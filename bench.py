@@ -95,7 +95,7 @@ def load_peaks():
 # to the timed workload by tokens x heads per launch (the traffic of these kernels grows in proportion).
 NCU_TRAFFIC_CFG1 = {
     # kernel kind: (bytes per launch, source file, sha256 of that file at capture time)
-    "bwd_dBdC": (20.55e6, "ssd_tc_bcf.cu", "859295b23fee1e4bd90f5ad8d9328f5793795a8a7698b9087b2286f5d42b35af"),
+    "bwd_dBdC": (20.54e6, "ssd_tc_bcf.cu", "79a49e539bef6a7f64c2774cd24e04bff53cde132d380ea03f4d4eb0743ba242"),
     "bwd_dx": (17.23e6, "ssd_tc_scan.cu", "3ea5757da6501f0ea6a699499461cb3b9279fc57cceda76140ade8c4444a5dcd"),
     "chunk_scan_fwd": (10.94e6, "ssd_tc_scan.cu", "3ea5757da6501f0ea6a699499461cb3b9279fc57cceda76140ade8c4444a5dcd"),
     "chunk_state": (7.04e6, "ssd_tc.cu", "476c275026f7e136b96cec13cc7c617ea7c59d6fc34edbe9bc79467efbc16aee"),
