@@ -45,7 +45,10 @@ static void prof_end(ProfEvent *ev, cudaStream_t st) {
 
 struct Layout {
     size_t status, cs, dtT, Hst, Hbf, hcarry, Gst, Gbf, gcarry, ghdot, ddt_dir, rho, rho2, psi, psi2, pB, pC, dAp, dDp;
-    size_t dtT_b, rho2_b, ghdot_b, rhob, psib;   // second copies: a segment's finishing kernels overlap the next segment's first ones
+    size_t rhob, psib;
+    // second copies (tensor-core path, more than one segment): the state chain of a segment runs on a helper
+    // stream while the large kernels of its neighbour still read the first copies
+    size_t cs_b, dtT_b, Hbf_b, Gbf_b, rho2_b, ghdot_b;
     size_t total;
 };
 
@@ -174,6 +177,10 @@ static void make_layout(const Plan &pl, int op, Layout &lo) {
     lo.Hst = take(st * sizeof(float));
     lo.Hbf = take(pl.use_tc ? st * 2 : 0);
     lo.hcarry = take(BH * PN * sizeof(float));
+    const bool twin = pl.use_tc && pl.nseg > 1;
+    lo.cs_b = take(twin ? vec : 0);
+    lo.dtT_b = take(twin ? vec : 0);
+    lo.Hbf_b = take(twin ? st * 2 : 0);
     if (bwd) {
         lo.Gst = take(st * sizeof(float));
         lo.Gbf = take(pl.use_tc ? st * 2 : 0);
@@ -190,9 +197,9 @@ static void make_layout(const Plan &pl, int op, Layout &lo) {
         lo.pC = take(part);
         lo.dAp = take(BH * pl.nct * sizeof(float));
         lo.dDp = take(BH * pl.nct * 16 * sizeof(float));
-        lo.dtT_b = take(pl.use_tc ? vec : 0);
-        lo.rho2_b = take(pl.use_tc ? vec : 0);
-        lo.ghdot_b = take(pl.use_tc ? BH * pl.ncs * 8 * sizeof(float) : 0);
+        lo.Gbf_b = take(twin ? st * 2 : 0);
+        lo.rho2_b = take(twin ? vec : 0);
+        lo.ghdot_b = take(twin ? BH * pl.ncs * 8 * sizeof(float) : 0);
         lo.rhob = take(pl.use_tc ? vec : 0);
         lo.psib = take(pl.use_tc ? vec : 0);
     }
@@ -217,14 +224,16 @@ static int check_device() {
     return cached_ok ? SSD_OK : SSD_EDEVICE;
 }
 
-// Two helper streams per (host thread, device) for the backward's independent kernels, with the events
-// that fork them off the caller's stream and join them back.  Created on first use, never destroyed
-// (they hold no device memory); the caller's stream stays the only one the caller has to order against.
+// Three helper streams per (host thread, device) with the events that fork them off the caller's stream and
+// join them back: s[0] runs the state chain of a segment (chunk states, state passes), s[1] the dB/dC kernel
+// beside dx on the caller's stream, s[2] a segment's two finishing kernels.  Created on first use, never
+// destroyed (they hold no device memory); the caller's stream stays the only one the caller has to order
+// against.  Events indexed [2] alternate with the segment, like the second copies of the scratch regions.
 struct SideStreams {
     int dev = -1;
     cudaStream_t s[3] = {nullptr, nullptr, nullptr};
-    cudaEvent_t fork[2] = {nullptr, nullptr}, join[2] = {nullptr, nullptr};
-    cudaEvent_t tail_go = nullptr, tail_done = nullptr;
+    cudaEvent_t start = nullptr, join = nullptr, tail_go = nullptr;
+    cudaEvent_t chain_done[2] = {nullptr, nullptr}, big_done[2] = {nullptr, nullptr}, tail_done[2] = {nullptr, nullptr};
 };
 static SideStreams *side_streams() {
     static thread_local std::vector<SideStreams> all;
@@ -236,12 +245,10 @@ static SideStreams *side_streams() {
     a.dev = dev;
     for (int i = 0; i < 3; ++i)
         if (cudaStreamCreateWithFlags(&a.s[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-    for (int i = 0; i < 2; ++i) {
-        if (cudaEventCreateWithFlags(&a.fork[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
-        if (cudaEventCreateWithFlags(&a.join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
-    }
-    if (cudaEventCreateWithFlags(&a.tail_go, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-    if (cudaEventCreateWithFlags(&a.tail_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    cudaEvent_t *evs[] = {&a.start, &a.join, &a.tail_go, &a.chain_done[0], &a.chain_done[1], &a.big_done[0],
+                          &a.big_done[1], &a.tail_done[0], &a.tail_done[1]};
+    for (cudaEvent_t *ev : evs)
+        if (cudaEventCreateWithFlags(ev, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     all.push_back(a);
     return &all.back();
 }
@@ -306,10 +313,23 @@ static void set_segment(const Plan &pl, int k, SegParams &sp) {
     sp.nsplit_scan = best_head_split(sp.nc, pl.G, pl.B, pl.hpg, pl.hpg >= 2 ? pl.hpg / 2 : 1);
 }
 
+// Points the kernels at the first or the second copy of the scratch regions that exist twice.
+static void select_copy(const Layout &lo, void *ws, bool second, bool bwd, SegParams &sp) {
+    char *w = (char *)ws;
+    sp.cs = (float *)(w + (second ? lo.cs_b : lo.cs));
+    sp.dtT = (float *)(w + (second ? lo.dtT_b : lo.dtT));
+    sp.Hbf = (__nv_bfloat16 *)(w + (second ? lo.Hbf_b : lo.Hbf));
+    if (bwd) {
+        sp.Gbf = (__nv_bfloat16 *)(w + (second ? lo.Gbf_b : lo.Gbf));
+        sp.rho2 = (float *)(w + (second ? lo.rho2_b : lo.rho2));
+        sp.ghdot = (float *)(w + (second ? lo.ghdot_b : lo.ghdot));
+    }
+}
+
 static int forward_impl(const ssd_shape_t *shape, const void *x, const float *dt, const float *A,
                         const void *Bm, const void *Cm, const float *D, const float *h0, void *y,
                         float *h_final, float *boundary, bool need_boundary, void *ws,
-                        size_t ws_bytes, void *stream) {
+                        size_t ws_bytes, void *stream, bool may_use_helper_stream = true) {
     Plan pl;
     int rc = make_plan(shape, pl);
     if (rc) return rc;
@@ -333,6 +353,40 @@ static int forward_impl(const ssd_shape_t *shape, const void *x, const float *dt
     TcMaps maps;
     if (pl.use_tc && !tc_make_maps(sp, maps)) return SSD_ECUDA;
     const long long PN = (long long)pl.P * pl.N;
+    if (pl.use_tc && pl.nseg > 1 && may_use_helper_stream && !(shape->flags & SSD_FLAG_SERIAL) && !g_prof_on) {
+        // Algorithm 1 with the state chain one segment ahead: chunk states and state pass of segment k run on a
+        // helper stream while the caller's stream still computes y of segment k-1, whose last, partly idle wave
+        // they fill.  What both touch (cumulative sums, dt per chunk, bf16 chunk states) exists twice and
+        // alternates; the fp32 chunk sums and the carried state belong to the chain alone.
+        SideStreams *side = side_streams();
+        if (!side) { g_last_cuda = (int)cudaGetLastError(); return SSD_ECUDA; }
+        TcMaps maps_b;
+        select_copy(lo, ws, true, false, sp);
+        if (!tc_make_maps(sp, maps_b)) return SSD_ECUDA;
+        cudaStream_t chain = side->s[0];
+        SSD_TRY(cudaEventRecord(side->start, st));
+        SSD_TRY(cudaStreamWaitEvent(chain, side->start, 0));
+        for (int k = 0; k < pl.nseg; ++k) {
+            const int par = k & 1;
+            set_segment(pl, k, sp);
+            select_copy(lo, ws, par != 0, false, sp);
+            const TcMaps &mk = par ? maps_b : maps;
+            if (k >= 2) SSD_TRY(cudaStreamWaitEvent(chain, side->big_done[par], 0));   // y of segment k-2 has read this copy
+            {
+                cudaStream_t st = chain;
+                SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_tc(sp, mk, STATE_MODE_FWD, st));
+                const float *init = (k == 0) ? h0 : sp.hcarry;
+                float *bnd = boundary ? boundary + (size_t)k * pl.H * PN : nullptr;
+                SSD_LAUNCH(KIND_STATE_PASS_FWD, launch_state_pass_fwd(sp, init, (long long)pl.H * PN, bnd, (long long)pl.nseg * pl.H * PN,
+                                              (k == pl.nseg - 1) ? h_final : nullptr, true, st));
+                SSD_TRY(cudaEventRecord(side->chain_done[par], st));
+            }
+            SSD_TRY(cudaStreamWaitEvent(st, side->chain_done[par], 0));
+            SSD_LAUNCH(KIND_SCAN_FWD, launch_scan_tc(sp, mk, SC_FWD, st));
+            if (k + 2 < pl.nseg) SSD_TRY(cudaEventRecord(side->big_done[par], st));
+        }
+        return SSD_OK;
+    }
     for (int k = 0; k < pl.nseg; ++k) {
         set_segment(pl, k, sp);
         if (pl.use_tc) {   // the tensor-core chunk-state kernel computes the chunk cumsum itself
@@ -422,7 +476,7 @@ int ssd_fwd_static_ws(const ssd_shape_t *shape, const void *x, const float *dt, 
     // forward_impl zeroes the status word on the stream and writes every other scratch region
     // before reading it, so stale contents of the shared array cannot leak into the outputs.
     return forward_impl(shape, x, dt, A, Bm, Cm, D, h0, y, h_final, nullptr, false, ws,
-                        (size_t)SSD_STATIC_WS_BYTES, stream);
+                        (size_t)SSD_STATIC_WS_BYTES, stream, false);
 }
 
 int ssd_fwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, const float *A,
@@ -462,10 +516,6 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
     TcMaps maps;
     if (pl.use_tc && !tc_make_maps(sp, maps)) return SSD_ECUDA;
     const long long PN = (long long)pl.P * pl.N;
-    // The dC kernel needs only the recomputed states, the dB and dx kernels also the state gradients; the
-    // three do not depend on one another.  Unless told otherwise they run on side streams forked off the
-    // caller's stream and joined back before the segment's finishing kernels, so that one kernel's tail
-    // (its last, partly idle wave) is filled by the next one's CTAs.
     const bool fused_bc = pl.use_tc && !(shape->flags & SSD_FLAG_SPLIT_BC);
     if (fused_bc) {
         sp.nsl = pl.nslf;
@@ -478,88 +528,107 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
         side = side_streams();
         if (!side) { g_last_cuda = (int)cudaGetLastError(); return SSD_ECUDA; }
     }
-    // With the helper streams, a segment's two finishing kernels (which are short and latency-bound) run on
-    // a third one while the caller's stream already recomputes the next segment; what they read and the
-    // next segment's first kernels rewrite (dt per chunk, rho2, <G,H>) alternates between two copies.
-    bool tail_pending = false;
-    for (int k = pl.nseg - 1; k >= 0; --k) {
-        set_segment(pl, k, sp);
-        if (side) {
-            const bool odd = ((pl.nseg - 1 - k) & 1) != 0;
-            sp.dtT = (float *)((char *)ws + (odd ? lo.dtT_b : lo.dtT));
-            sp.rho2 = (float *)((char *)ws + (odd ? lo.rho2_b : lo.rho2));
-            sp.ghdot = (float *)((char *)ws + (odd ? lo.ghdot_b : lo.ghdot));
+    if (side) {
+        // Algorithm 2 as three pipelines that meet through events.  Segment k (right to left) needs
+        //   chain(k): Recompute_Forward (chunk states, forward state pass), the state-gradient contributions and
+        //             the backward state pass -- all it takes from segment k+1 is the state gradient handed left;
+        //   big(k)  : dx on the caller's stream beside dB/dC on a second one -- they read what chain(k) left;
+        //   tail(k) : the two short finishing kernels.
+        // chain(k-1) runs on its own stream while big(k) is busy and fills the SMs that big(k)'s last, partly
+        // idle wave leaves free; tail(k) runs under big(k-1)'s predecessors likewise.  What chain(k-1) writes and
+        // big(k) / tail(k) read exists twice and alternates with the segment (cumulative sums, dt per chunk, both
+        // bf16 state copies, rho2, <G,H>); the fp32 chunk sums and the carried gradient belong to the chain alone.
+        const bool twin = pl.nseg > 1;
+        TcMaps maps_b;
+        if (twin) {
+            select_copy(lo, ws, true, true, sp);
+            if (!tc_make_maps(sp, maps_b)) return SSD_ECUDA;
         }
-        // Recompute_Forward: chunk-entry states of segment k from the stored boundary state
-        if (pl.use_tc) {   // the tensor-core chunk-state kernel computes the chunk cumsum itself
-            SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_tc(sp, maps, STATE_MODE_FWD, st));
-        } else {
-            SSD_LAUNCH(KIND_CUMSUM, launch_chunk_cumsum(sp, st));
-            SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
-        }
-        SSD_LAUNCH(KIND_STATE_PASS_FWD, launch_state_pass_fwd(sp, boundary + (size_t)k * pl.H * PN, (long long)pl.nseg * pl.H * PN,
-                                      nullptr, 0, nullptr, pl.use_tc, st));
-        if (side && !fused_bc) {
-            SSD_TRY(cudaEventRecord(side->fork[0], st));
-            SSD_TRY(cudaStreamWaitEvent(side->s[0], side->fork[0], 0));
-            if (tail_pending) SSD_TRY(cudaStreamWaitEvent(side->s[0], side->tail_done, 0));
+        cudaStream_t chain = side->s[0], bcs = side->s[1], tails = side->s[2];
+        SSD_TRY(cudaEventRecord(side->start, st));
+        SSD_TRY(cudaStreamWaitEvent(chain, side->start, 0));
+        int par = 0;
+        for (int k = pl.nseg - 1; k >= 0; --k) {
+            par = (pl.nseg - 1 - k) & 1;
+            set_segment(pl, k, sp);
+            select_copy(lo, ws, par != 0, true, sp);
+            const TcMaps &mk = par ? maps_b : maps;
+            // ---- chain(k); its copy was last read by big(k+2) and tail(k+2)
+            if (k + 2 <= pl.nseg - 1) SSD_TRY(cudaStreamWaitEvent(chain, side->tail_done[par], 0));
             {
-                cudaStream_t st = side->s[0];
-                SSD_LAUNCH(KIND_BWD_DC, launch_grad_bc_tc(sp, maps, GB_DC, st));
-                SSD_TRY(cudaEventRecord(side->join[0], st));
+                cudaStream_t st = chain;
+                SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_tc(sp, mk, STATE_MODE_FWD, st));
+                SSD_LAUNCH(KIND_STATE_PASS_FWD, launch_state_pass_fwd(sp, boundary + (size_t)k * pl.H * PN, (long long)pl.nseg * pl.H * PN,
+                                              nullptr, 0, nullptr, true, st));
+                SSD_LAUNCH(KIND_DSTATE, launch_chunk_state_tc(sp, mk, STATE_MODE_DSTATE, st));
+                const float *ginit = (k == pl.nseg - 1) ? dh_final : sp.gcarry;
+                float *gleft = (k == 0 && dh0) ? dh0 : sp.gcarry;
+                SSD_LAUNCH(KIND_STATE_PASS_BWD, launch_state_pass_bwd(sp, ginit, gleft, true, st));
+                SSD_TRY(cudaEventRecord(side->chain_done[par], st));
             }
-        }
-        // Backward through the segment; dh enters from the right, leaves to the left
-        if (pl.use_tc) SSD_LAUNCH(KIND_DSTATE, launch_chunk_state_tc(sp, maps, STATE_MODE_DSTATE, st));
-        else SSD_LAUNCH(KIND_DSTATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_DSTATE, st));
-        const float *ginit = (k == pl.nseg - 1) ? dh_final : sp.gcarry;
-        float *gleft = (k == 0 && dh0) ? dh0 : sp.gcarry;
-        SSD_LAUNCH(KIND_STATE_PASS_BWD, launch_state_pass_bwd(sp, ginit, gleft, pl.use_tc, st));
-        if (side) {
-            SSD_TRY(cudaEventRecord(side->fork[1], st));
-            SSD_TRY(cudaStreamWaitEvent(side->s[1], side->fork[1], 0));
-            if (tail_pending) {
-                SSD_TRY(cudaStreamWaitEvent(side->s[1], side->tail_done, 0));
-                SSD_TRY(cudaStreamWaitEvent(st, side->tail_done, 0));
-                tail_pending = false;
+            // ---- big(k); its outputs (direct ddt, rho, psi, partial dB/dC slices) are read by tail(k+1)
+            SSD_TRY(cudaStreamWaitEvent(st, side->chain_done[par], 0));
+            SSD_TRY(cudaStreamWaitEvent(bcs, side->chain_done[par], 0));
+            if (k < pl.nseg - 1) {
+                SSD_TRY(cudaStreamWaitEvent(st, side->tail_done[par ^ 1], 0));
+                SSD_TRY(cudaStreamWaitEvent(bcs, side->tail_done[par ^ 1], 0));
             }
             {
-                cudaStream_t st = side->s[1];
-                if (fused_bc) SSD_LAUNCH(KIND_BWD_DBDC, launch_grad_bc_fused(sp, maps, st));
-                else SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_tc(sp, maps, GB_DB, st));
-                SSD_TRY(cudaEventRecord(side->join[1], st));
+                cudaStream_t st = bcs;
+                if (fused_bc) {
+                    SSD_LAUNCH(KIND_BWD_DBDC, launch_grad_bc_fused(sp, mk, st));
+                } else {
+                    SSD_LAUNCH(KIND_BWD_DC, launch_grad_bc_tc(sp, mk, GB_DC, st));
+                    SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_tc(sp, mk, GB_DB, st));
+                }
+                SSD_TRY(cudaEventRecord(side->join, st));
             }
-        }
-        if (pl.use_tc) SSD_LAUNCH(KIND_BWD_DX, launch_scan_tc(sp, maps, SC_DX, st));
-        else SSD_LAUNCH(KIND_BWD_DX, launch_masked_product_simt(sp, pl.dtype, MP_BWD_DX, st));
-        if (side) {
-            if (!fused_bc) SSD_TRY(cudaStreamWaitEvent(st, side->join[0], 0));
-            SSD_TRY(cudaStreamWaitEvent(st, side->join[1], 0));
-        } else if (fused_bc) {
-            SSD_LAUNCH(KIND_BWD_DBDC, launch_grad_bc_fused(sp, maps, st));
-        } else if (pl.use_tc) {
-            SSD_LAUNCH(KIND_BWD_DC, launch_grad_bc_tc(sp, maps, GB_DC, st));
-            SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_tc(sp, maps, GB_DB, st));
-        } else {
-            SSD_LAUNCH(KIND_BWD_DC, launch_masked_product_simt(sp, pl.dtype, MP_DC, st));
-            SSD_LAUNCH(KIND_BWD_DB, launch_masked_product_simt(sp, pl.dtype, MP_DB, st));
-        }
-        if (side) {
+            SSD_LAUNCH(KIND_BWD_DX, launch_scan_tc(sp, mk, SC_DX, st));
+            SSD_TRY(cudaStreamWaitEvent(st, side->join, 0));
+            // ---- tail(k)
             SSD_TRY(cudaEventRecord(side->tail_go, st));
-            SSD_TRY(cudaStreamWaitEvent(side->s[2], side->tail_go, 0));
+            SSD_TRY(cudaStreamWaitEvent(tails, side->tail_go, 0));
             {
-                cudaStream_t st = side->s[2];
+                cudaStream_t st = tails;
                 SSD_LAUNCH(KIND_BWD_FINISH, launch_bwd_finish(sp, st));
                 SSD_LAUNCH(KIND_REDUCE_DBDC, launch_reduce_dbdc(sp, pl.dtype, st));
-                SSD_TRY(cudaEventRecord(side->tail_done, st));
+                SSD_TRY(cudaEventRecord(side->tail_done[par], st));
             }
-            tail_pending = true;
-        } else {
+        }
+        SSD_TRY(cudaStreamWaitEvent(st, side->tail_done[par], 0));   // the finishing stream is in order: this covers every segment
+    } else {
+        for (int k = pl.nseg - 1; k >= 0; --k) {
+            set_segment(pl, k, sp);
+            // Recompute_Forward: chunk-entry states of segment k from the stored boundary state
+            if (pl.use_tc) {   // the tensor-core chunk-state kernel computes the chunk cumsum itself
+                SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_tc(sp, maps, STATE_MODE_FWD, st));
+            } else {
+                SSD_LAUNCH(KIND_CUMSUM, launch_chunk_cumsum(sp, st));
+                SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_FWD, st));
+            }
+            SSD_LAUNCH(KIND_STATE_PASS_FWD, launch_state_pass_fwd(sp, boundary + (size_t)k * pl.H * PN, (long long)pl.nseg * pl.H * PN,
+                                          nullptr, 0, nullptr, pl.use_tc, st));
+            // Backward through the segment; dh enters from the right, leaves to the left
+            if (pl.use_tc) SSD_LAUNCH(KIND_DSTATE, launch_chunk_state_tc(sp, maps, STATE_MODE_DSTATE, st));
+            else SSD_LAUNCH(KIND_DSTATE, launch_chunk_state_simt(sp, pl.dtype, STATE_MODE_DSTATE, st));
+            const float *ginit = (k == pl.nseg - 1) ? dh_final : sp.gcarry;
+            float *gleft = (k == 0 && dh0) ? dh0 : sp.gcarry;
+            SSD_LAUNCH(KIND_STATE_PASS_BWD, launch_state_pass_bwd(sp, ginit, gleft, pl.use_tc, st));
+            if (pl.use_tc) SSD_LAUNCH(KIND_BWD_DX, launch_scan_tc(sp, maps, SC_DX, st));
+            else SSD_LAUNCH(KIND_BWD_DX, launch_masked_product_simt(sp, pl.dtype, MP_BWD_DX, st));
+            if (fused_bc) {
+                SSD_LAUNCH(KIND_BWD_DBDC, launch_grad_bc_fused(sp, maps, st));
+            } else if (pl.use_tc) {
+                SSD_LAUNCH(KIND_BWD_DC, launch_grad_bc_tc(sp, maps, GB_DC, st));
+                SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_tc(sp, maps, GB_DB, st));
+            } else {
+                SSD_LAUNCH(KIND_BWD_DC, launch_masked_product_simt(sp, pl.dtype, MP_DC, st));
+                SSD_LAUNCH(KIND_BWD_DB, launch_masked_product_simt(sp, pl.dtype, MP_DB, st));
+            }
             SSD_LAUNCH(KIND_BWD_FINISH, launch_bwd_finish(sp, st));
             SSD_LAUNCH(KIND_REDUCE_DBDC, launch_reduce_dbdc(sp, pl.dtype, st));
         }
     }
-    if (tail_pending) SSD_TRY(cudaStreamWaitEvent(st, side->tail_done, 0));
     SSD_LAUNCH(KIND_FINAL, launch_final_dAdD(sp, dA, dD, (shape->flags & SSD_FLAG_ACCUM_PARAM_GRADS) != 0, st));
     return SSD_OK;
 }
