@@ -14,7 +14,9 @@
 // heads of the CTA and leave once, as fp32 partial slices that a later kernel adds in a fixed order.
 // Shared memory holds the C rows of the t-block and the B rows of the s-block for the whole CTA (operands
 // of CB, and the MN-major B operands of the two products), and per head the dy / x rows (double buffered),
-// the masked tile, one buffer for the scaled rows of an inter-chunk term, and the two bf16 chunk states.
+// one buffer for the scaled rows of an inter-chunk term, and the two bf16 chunk states (double buffered: the
+// second copies live where the head sum of W goes at the very end, which is free until then, so a state's
+// load has a whole head of time to land).
 // The inter-chunk terms are spread over the tiles: (0,0) adds dC's for t-block 0, (1,0) dB's for s-block 0,
 // (1,1) dC's for t-block 1 and then dB's for s-block 1.
 //   warp 0 producer (TMA) | warp 1 MMA issuer | warps 2..17 mask warps | warp 18 per-head vectors
@@ -31,9 +33,9 @@ constexpr int GF_THREADS = 608;
 constexpr uint32_t GF_OFF_CT = 0;          // 32 KB  C rows of the t-block  [n-half][128 rows][128 B]
 constexpr uint32_t GF_OFF_BT = 32768;      // 32 KB  B rows of the s-block
 constexpr uint32_t GF_OFF_R = 65536;       // 2 x (dy rows of the t-block 16 KB | x rows of the s-block 16 KB)
-constexpr uint32_t GF_OFF_W = 131072;      // 32 KB  masked tile [s-half][128 t rows][128 B]
+constexpr uint32_t GF_OFF_W = 131072;      // 32 KB  head sum of the masked tiles [s-half][128 t rows][128 B]; until then: states of odd heads
 constexpr uint32_t GF_OFF_SC = 163840;     // 16 KB  scaled rows of an inter-chunk term
-constexpr uint32_t GF_OFF_ST = 180224;     // 2 x 16 KB  bf16 chunk states (entering: H, gradient leaving: G)
+constexpr uint32_t GF_OFF_ST = 180224;     // 2 x 16 KB  bf16 chunk states (entering: H, gradient leaving: G) of even heads
 constexpr uint32_t GF_OFF_VEC = 212992;    // per-head vectors, double buffered
 constexpr uint32_t GF_VEC_FLOATS = 256 * 3 + 64;
 constexpr uint32_t GF_OFF_PART = GF_OFF_VEC + 2 * GF_VEC_FLOATS * 4;   // [head parity][rho: 4 slices x 128 rows | psi: 4 quarters x 128 cols]
@@ -64,8 +66,8 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
                 const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmG) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ uint64_t bar_ld, bar_cb, rfull[2], rempty[2], sfull, sempty, wfull, scfull, scempty, hfull, hempty,
-        gfull, gempty, accfull, vfull[2], vempty[2], pfull[2], pempty[2];
+    __shared__ uint64_t bar_ld, bar_cb, rfull[2], rempty[2], sfull, sempty, wfull, scfull, scempty, hfull[2], hempty[2],
+        gfull[2], gempty[2], stdone, accfull, vfull[2], vempty[2], pfull[2], pempty[2];
     __shared__ uint32_t tmem_base, abort_flag;
 
     // 1-D grid: all full tiles first (they have the most mask work), then the two diagonal kinds
@@ -95,16 +97,17 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
             mbar_init(&vempty[i], 16);
             mbar_init(&pfull[i], 16);         // the mask warps' partial sums of rho / psi of a head
             mbar_init(&pempty[i], 1);
+            mbar_init(&hfull[i], 1);
+            mbar_init(&hempty[i], 1);
+            mbar_init(&gfull[i], 1);
+            mbar_init(&gempty[i], 1);
         }
         mbar_init(&sfull, 1);
         mbar_init(&sempty, 16);
         mbar_init(&wfull, 16);
         mbar_init(&scfull, 16);
         mbar_init(&scempty, 1);
-        mbar_init(&hfull, 1);
-        mbar_init(&hempty, 1);
-        mbar_init(&gfull, 1);
-        mbar_init(&gempty, 1);
+        mbar_init(&stdone, 1);
         mbar_init(&accfull, 1);
         abort_flag = 0;
         fence_barrier_init();
@@ -133,17 +136,18 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
                 mbar_arrive_expect_tx(&rfull[rbuf], 32768);
                 tma_load_3d(smem + GF_OFF_R + rbuf * 32768, &tmDy, &rfull[rbuf], h * 64, tok0 + tb * 128, b);
                 tma_load_3d(smem + GF_OFF_R + rbuf * 32768 + 16384, &tmX, &rfull[rbuf], h * 64, tok0 + sb * 128, b);
+                unsigned char *stb = smem + (rbuf ? GF_OFF_W : GF_OFF_ST);   // states of odd heads: the spare buffer
                 if (doC) {
-                    if (hi >= 1) mbar_wait(&hempty, (hi - 1) & 1, abortp, p.status);
-                    mbar_arrive_expect_tx(&hfull, 16384);
-                    tma_load_3d(smem + GF_OFF_ST, &tmH, &hfull, 0, (rowH + h) * 64, 0);
-                    tma_load_3d(smem + GF_OFF_ST + 8192, &tmH, &hfull, 64, (rowH + h) * 64, 0);
+                    if (hi >= 2) mbar_wait(&hempty[rbuf], ((hi >> 1) - 1) & 1, abortp, p.status);
+                    mbar_arrive_expect_tx(&hfull[rbuf], 16384);
+                    tma_load_3d(stb, &tmH, &hfull[rbuf], 0, (rowH + h) * 64, 0);
+                    tma_load_3d(stb + 8192, &tmH, &hfull[rbuf], 64, (rowH + h) * 64, 0);
                 }
                 if (doB) {
-                    if (hi >= 1) mbar_wait(&gempty, (hi - 1) & 1, abortp, p.status);
-                    mbar_arrive_expect_tx(&gfull, 16384);
-                    tma_load_3d(smem + GF_OFF_ST + 16384, &tmG, &gfull, 0, (rowG + h) * 64, 0);
-                    tma_load_3d(smem + GF_OFF_ST + 16384 + 8192, &tmG, &gfull, 64, (rowG + h) * 64, 0);
+                    if (hi >= 2) mbar_wait(&gempty[rbuf], ((hi >> 1) - 1) & 1, abortp, p.status);
+                    mbar_arrive_expect_tx(&gfull[rbuf], 16384);
+                    tma_load_3d(stb + 16384, &tmG, &gfull[rbuf], 0, (rowG + h) * 64, 0);
+                    tma_load_3d(stb + 16384 + 8192, &tmG, &gfull[rbuf], 64, (rowG + h) * 64, 0);
                 }
             }
         }
@@ -160,10 +164,11 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
             const uint64_t dWk = umma_desc_sw128(smem_u32(smem + GF_OFF_W), 16, 1024), dWm = umma_desc_sw128(smem_u32(smem + GF_OFF_W), 16384, 1024);
             const uint64_t dSk = umma_desc_sw128(smem_u32(smem + GF_OFF_SC), 16, 1024);
             const uint64_t dSt = umma_desc_sw128(smem_u32(smem + GF_OFF_ST), 8192, 1024);
+            const uint64_t dSt1 = umma_desc_sw128(smem_u32(smem + GF_OFF_W), 8192, 1024);    // states of odd heads
             const uint32_t loCk = (uint32_t)dCk, hiK = (uint32_t)(dCk >> 32), loBk = (uint32_t)dBk;
             const uint32_t loCm = (uint32_t)dCm, hiM = (uint32_t)(dCm >> 32), loBm = (uint32_t)dBm;
             const uint32_t loRk = (uint32_t)dRk, loWk = (uint32_t)dWk, loWm = (uint32_t)dWm, loSk = (uint32_t)dSk;
-            const uint32_t loSt = (uint32_t)dSt, hiSt = (uint32_t)(dSt >> 32);
+            const uint32_t loSt0 = (uint32_t)dSt, loSt1 = (uint32_t)dSt1, hiSt = (uint32_t)(dSt >> 32);
 
             // CB tile, once
             mbar_wait(&bar_ld, 0, abortp, p.status);
@@ -195,8 +200,9 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
                 // inter-chunk terms: scaled rows (K = p) times a chunk state.  A tile's first one is published by the
                 // mask warps before they mask the head, so it is issued first: the scaled-rows buffer is free again
                 // by the time tile (1,1) wants it for its second one.
+                const uint32_t loSt = (hi & 1) ? loSt1 : loSt0;
                 auto inter_dC = [&]() {   // dC += (e^{cs_t} dy_t) H_in
-                    mbar_wait(&hfull, hi & 1, abortp, p.status);
+                    mbar_wait(&hfull[hi & 1], (hi >> 1) & 1, abortp, p.status);
                     mbar_wait(&scfull, scuse & 1, abortp, p.status);
                     ++scuse;
                     tc_fence_after_sync();
@@ -207,10 +213,10 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
                         else umma_bf16_fixed<true>(tm + TF_ACCC, ad, bd, idKM);
                     }
                     umma_commit(&scempty);
-                    umma_commit(&hempty);
+                    umma_commit(&hempty[hi & 1]);
                 };
                 auto inter_dB = [&](bool first_into_acc) {   // dB += (dt_s e^{cs_last-cs_s} x_s) Gout
-                    mbar_wait(&gfull, hi & 1, abortp, p.status);
+                    mbar_wait(&gfull[hi & 1], (hi >> 1) & 1, abortp, p.status);
                     mbar_wait(&scfull, scuse & 1, abortp, p.status);
                     ++scuse;
                     tc_fence_after_sync();
@@ -221,7 +227,7 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
                         else umma_bf16_fixed<true>(tm + TF_ACCB, ad, bd, idKM);
                     }
                     umma_commit(&scempty);
-                    umma_commit(&gempty);
+                    umma_commit(&gempty[hi & 1]);
                 };
                 if (doC) inter_dC();
                 else inter_dB(hi == 0);
@@ -234,6 +240,7 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
                 if (doC && doB) inter_dB(hi == 0);
                 umma_commit(&rempty[hi & 1]);
             }
+            umma_commit(&stdone);     // every product that read a chunk state is done: the spare buffer may take the head sum
             // the head sum of the masked tiles (made in fp32 by the mask warps, rounded once): both products
             mbar_wait(&wfull, 0, abortp, p.status);
             tc_fence_after_sync();
@@ -471,7 +478,8 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
         }
 
         // ---- the head sum of W, rounded once to bf16: [s-half w][row][128 B], this thread's 16 columns of a
-        // half = chunks quar * 2, quar * 2 + 1
+        // half = chunks quar * 2, quar * 2 + 1.  The buffer held chunk states until the last head's products ended.
+        mbar_wait(&stdone, 0, abortp, p.status);
 #pragma unroll
         for (int w = 0; w < 2; ++w) {
             unsigned char *mrow = smem + GF_OFF_W + w * 16384 + rl * 128;
