@@ -57,6 +57,29 @@ template <> __device__ __forceinline__ void st4<__nv_bfloat16>(__nv_bfloat16 *p,
     *reinterpret_cast<uint2 *>(p) = v;
 }
 
+// The same four channels as two pairs, for the packed two-lane fp32 instructions of the backward kernel.
+template <typename T> __device__ __forceinline__ void ld2x2(const T *p, float2 &a, float2 &b);
+template <> __device__ __forceinline__ void ld2x2<float>(const float *p, float2 &a, float2 &b) {
+    const float4 v = *reinterpret_cast<const float4 *>(p);
+    a = make_float2(v.x, v.y);
+    b = make_float2(v.z, v.w);
+}
+template <> __device__ __forceinline__ void ld2x2<__nv_bfloat16>(const __nv_bfloat16 *p, float2 &a, float2 &b) {
+    const uint2 v = *reinterpret_cast<const uint2 *>(p);
+    a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&v.x));
+    b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&v.y));
+}
+__device__ __forceinline__ float2 sigmoid_fast2(float2 x) {
+    const float2 t = __fmul2_rn(x, make_float2(-1.4426950408889634f, -1.4426950408889634f));
+    float2 e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.x) : "f"(t.x));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.y) : "f"(t.y));
+    const float2 d = __fadd2_rn(e, make_float2(1.f, 1.f));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r.x) : "f"(d.x));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r.y) : "f"(d.y));
+    return r;
+}
+
 // Stage rows [t_first, t_last) of a [L, C] tensor (channels cbase .. cbase + nch) into shared memory, row r of the
 // stage = token t_first + r, 512 channels of room per row.  Tokens in front of the segment come from the carried
 // state (3 rows) or are zero-filled; called by one thread, completion on `bar`.
@@ -176,66 +199,76 @@ __global__ void __launch_bounds__(CV_THREADS) k_conv_bwd(const T *u, long long u
         stage_rows(sg, gb, (const T *)nullptr, t_begin, s_end, C, cbase, nch, &bar);
     }
     const bool active = c0 < C;
-    float wk[CV_CH][4], bs[CV_CH];
+    // two channel pairs per thread: every quantity below is a float2 over (c, c + 1), so that the multiply-adds
+    // issue as packed two-lane instructions (the kernel is bound by instruction issue as much as by memory)
+    constexpr int NP = CV_CH / 2;
+    float2 wk[NP][4], bs[NP];
     if (active) {
 #pragma unroll
-        for (int i = 0; i < CV_CH; ++i) {
-            const float4 wv = *reinterpret_cast<const float4 *>(w + (size_t)(c0 + i) * 4);
-            wk[i][0] = wv.x; wk[i][1] = wv.y; wk[i][2] = wv.z; wk[i][3] = wv.w;
-            bs[i] = bias[c0 + i];
+        for (int i = 0; i < NP; ++i) {
+            const float4 wa = *reinterpret_cast<const float4 *>(w + (size_t)(c0 + 2 * i) * 4);
+            const float4 wb = *reinterpret_cast<const float4 *>(w + (size_t)(c0 + 2 * i + 1) * 4);
+            wk[i][0] = make_float2(wa.x, wb.x); wk[i][1] = make_float2(wa.y, wb.y);
+            wk[i][2] = make_float2(wa.z, wb.z); wk[i][3] = make_float2(wa.w, wb.w);
+            bs[i] = make_float2(bias[c0 + 2 * i], bias[c0 + 2 * i + 1]);
         }
     }
     mbar_wait(&bar, 0, &abort_flag, &status_dummy);
     if (!active) return;
     const T *spu = su + threadIdx.x * CV_CH, *spg = sg + threadIdx.x * CV_CH;
-    float x0[CV_CH], x1[CV_CH], x2[CV_CH], x3[CV_CH];
-    float d0[CV_CH], d1[CV_CH], d2[CV_CH], d3[CV_CH];     // dpre[t], dpre[t+1], dpre[t+2], dpre[t+3] while emitting du[t]
-    float aw[CV_CH][4], ab[CV_CH];
+    const float2 zero2 = make_float2(0.f, 0.f), one2 = make_float2(1.f, 1.f), mone2 = make_float2(-1.f, -1.f);
+    float2 x0[NP], x1[NP], x2[NP], x3[NP];
+    float2 d0[NP], d1[NP], d2[NP], d3[NP];     // dpre[t], dpre[t+1], dpre[t+2], dpre[t+3] while emitting du[t]
+    float2 aw[NP][4], ab[NP];
 #pragma unroll
-    for (int i = 0; i < CV_CH; ++i) {
-        aw[i][0] = aw[i][1] = aw[i][2] = aw[i][3] = 0.f;
-        ab[i] = 0.f;
-        d0[i] = d1[i] = d2[i] = d3[i] = 0.f;
+    for (int i = 0; i < NP; ++i) {
+        aw[i][0] = aw[i][1] = aw[i][2] = aw[i][3] = zero2;
+        ab[i] = zero2;
+        d0[i] = d1[i] = d2[i] = d3[i] = zero2;
     }
-    ld4(spu, x0);
-    ld4(spu + 512, x1);
-    ld4(spu + 1024, x2);
+    ld2x2(spu, x0[0], x0[1]);
+    ld2x2(spu + 512, x1[0], x1[1]);
+    ld2x2(spu + 1024, x2[0], x2[1]);
     const int ns = (int)(s_end - t_begin), nt = (int)(t_end - t_begin);
 #pragma unroll 4
     for (int j = 0; j < ns + 3; ++j) {                     // s = t_begin + j
-        float dp[CV_CH];
+        float2 dp[NP];
         if (j < ns) {
-            float g[CV_CH];
-            ld4(spu + (size_t)(j + 3) * 512, x3);
-            ld4(spg + (size_t)j * 512, g);
+            float2 g[NP];
+            ld2x2(spu + (size_t)(j + 3) * 512, x3[0], x3[1]);
+            ld2x2(spg + (size_t)j * 512, g[0], g[1]);
 #pragma unroll
-            for (int i = 0; i < CV_CH; ++i) {
-                const float pre = fmaf(wk[i][3], x3[i], fmaf(wk[i][2], x2[i], fmaf(wk[i][1], x1[i], fmaf(wk[i][0], x0[i], bs[i]))));
-                const float sgm = sigmoid_fast(pre);
-                dp[i] = g[i] * sgm * fmaf(pre, 1.f - sgm, 1.f);
+            for (int i = 0; i < NP; ++i) {
+                const float2 pre = __ffma2_rn(wk[i][3], x3[i], __ffma2_rn(wk[i][2], x2[i], __ffma2_rn(wk[i][1], x1[i], __ffma2_rn(wk[i][0], x0[i], bs[i]))));
+                const float2 sgm = sigmoid_fast2(pre);
+                // dpre = dout * silu'(pre),  silu'(z) = s (1 + z (1 - s))
+                dp[i] = __fmul2_rn(__fmul2_rn(g[i], sgm), __ffma2_rn(pre, __ffma2_rn(sgm, mone2, one2), one2));
                 if (j < nt) {   // the tile's own tokens: weight and bias gradients
-                    aw[i][0] = fmaf(dp[i], x0[i], aw[i][0]);
-                    aw[i][1] = fmaf(dp[i], x1[i], aw[i][1]);
-                    aw[i][2] = fmaf(dp[i], x2[i], aw[i][2]);
-                    aw[i][3] = fmaf(dp[i], x3[i], aw[i][3]);
-                    ab[i] += dp[i];
+                    aw[i][0] = __ffma2_rn(dp[i], x0[i], aw[i][0]);
+                    aw[i][1] = __ffma2_rn(dp[i], x1[i], aw[i][1]);
+                    aw[i][2] = __ffma2_rn(dp[i], x2[i], aw[i][2]);
+                    aw[i][3] = __ffma2_rn(dp[i], x3[i], aw[i][3]);
+                    ab[i] = __fadd2_rn(ab[i], dp[i]);
                 }
                 x0[i] = x1[i]; x1[i] = x2[i]; x2[i] = x3[i];
             }
         } else {
 #pragma unroll
-            for (int i = 0; i < CV_CH; ++i) dp[i] = 0.f;
+            for (int i = 0; i < NP; ++i) dp[i] = zero2;
         }
         // shift the dpre window; after it d3 = dpre[s], d0 = dpre[s-3]: du[s-3] is complete
 #pragma unroll
-        for (int i = 0; i < CV_CH; ++i) { d0[i] = d1[i]; d1[i] = d2[i]; d2[i] = d3[i]; d3[i] = dp[i]; }
+        for (int i = 0; i < NP; ++i) { d0[i] = d1[i]; d1[i] = d2[i]; d2[i] = d3[i]; d3[i] = dp[i]; }
         const int jt = j - 3;
         if (jt >= 0 && jt < nt) {
             const long long t = t_begin + jt;
             float o[CV_CH];
 #pragma unroll
-            for (int i = 0; i < CV_CH; ++i)
-                o[i] = fmaf(wk[i][3], d0[i], fmaf(wk[i][2], d1[i], fmaf(wk[i][1], d2[i], wk[i][0] * d3[i])));
+            for (int i = 0; i < NP; ++i) {
+                const float2 v = __ffma2_rn(wk[i][3], d0[i], __ffma2_rn(wk[i][2], d1[i], __ffma2_rn(wk[i][1], d2[i], __fmul2_rn(wk[i][0], d3[i]))));
+                o[2 * i] = v.x;
+                o[2 * i + 1] = v.y;
+            }
             if (dtail && t >= (long long)L - 3) {
                 float e[CV_CH];
                 ld4(dtail + ((size_t)b * 3 + (size_t)(t - ((long long)L - 3))) * C + c0, e);
@@ -252,10 +285,12 @@ __global__ void __launch_bounds__(CV_THREADS) k_conv_bwd(const T *u, long long u
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
 #pragma unroll
-            for (int i = 0; i < CV_CH; ++i) col[i] = aw[i][k];
+            for (int i = 0; i < NP; ++i) { col[2 * i] = aw[i][k].x; col[2 * i + 1] = aw[i][k].y; }
             st4(pp + (size_t)k * C, col);
         }
-        st4(pp + (size_t)4 * C, ab);
+#pragma unroll
+        for (int i = 0; i < NP; ++i) { col[2 * i] = ab[i].x; col[2 * i + 1] = ab[i].y; }
+        st4(pp + (size_t)4 * C, col);
     }
 }
 
