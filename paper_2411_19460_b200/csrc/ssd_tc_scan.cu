@@ -47,6 +47,7 @@ constexpr uint32_t OFF_XR = 196608;       // 16 KB  SC_DX: the head's x rows of 
 constexpr uint32_t OFF_VEC = 212992;      // per-head vectors, double buffered
 constexpr uint32_t VEC_FLOATS = 256 * 3 + 64;
 constexpr uint32_t SC_SMEM = OFF_VEC + 2 * VEC_FLOATS * 4 + 1024;
+constexpr int PF_AHEAD = 3;               // L2 prefetch distance of the producer, in heads
 
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -162,6 +163,18 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                     if (hi >= 1) mbar_wait(&xrempty, (hi - 1) & 1, abortp, p.status);
                     mbar_arrive_expect_tx(&xrfull, 16384);
                     tma_load_3d(smem + OFF_XR, &tmXr, &xrfull, h * 64, tok0 + rb * 128, b);
+                }
+                // A value stage is held until the head's output has left it, so its next load can be issued only
+                // about one head before it is needed.  Ask for the tiles of the head three ahead (and the state two
+                // ahead) in L2 now; the later loads then take an L2 hit's time.
+                if (hi + PF_AHEAD < nheads) {
+                    const int hp = h + PF_AHEAD;
+                    for (int r0 = 0; r0 < ncols; r0 += 128) tma_prefetch_3d(&tmV, hp * 64, tok0 + colbase + r0, b);
+                    if (!FWD) tma_prefetch_3d(&tmXr, hp * 64, tok0 + rb * 128, b);
+                }
+                if (hi + PF_AHEAD - 1 < nheads) {
+                    tma_prefetch_3d(&tmSt, 0, (strow + h + PF_AHEAD - 1) * 64, 0);
+                    tma_prefetch_3d(&tmSt, 64, (strow + h + PF_AHEAD - 1) * 64, 0);
                 }
             }
         }
