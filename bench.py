@@ -95,9 +95,9 @@ def load_peaks():
 # to the timed workload by tokens x heads per launch (the traffic of these kernels grows in proportion).
 NCU_TRAFFIC_CFG1 = {
     # kernel kind: (bytes per launch, source file, sha256 of that file at capture time)
-    "bwd_dBdC": (20.54e6, "ssd_tc_bcf.cu", "79a49e539bef6a7f64c2774cd24e04bff53cde132d380ea03f4d4eb0743ba242"),
-    "bwd_dx": (17.23e6, "ssd_tc_scan.cu", "3ea5757da6501f0ea6a699499461cb3b9279fc57cceda76140ade8c4444a5dcd"),
-    "chunk_scan_fwd": (10.94e6, "ssd_tc_scan.cu", "3ea5757da6501f0ea6a699499461cb3b9279fc57cceda76140ade8c4444a5dcd"),
+    "bwd_dBdC": (20.55e6, "ssd_tc_bcf.cu", "86cbdbf8df5a575ff65e77851460b110f53d2ae5c0ef203bece4e8ba5cb8f8ee"),
+    "bwd_dx": (17.24e6, "ssd_tc_scan.cu", "f42132f3fb6c9558b719a6414f8431eb3af4548abcafdc0fcd79735a277d7f32"),
+    "chunk_scan_fwd": (10.94e6, "ssd_tc_scan.cu", "f42132f3fb6c9558b719a6414f8431eb3af4548abcafdc0fcd79735a277d7f32"),
     "chunk_state": (7.04e6, "ssd_tc.cu", "476c275026f7e136b96cec13cc7c617ea7c59d6fc34edbe9bc79467efbc16aee"),
     "dstate_contrib": (7.04e6, "ssd_tc.cu", "476c275026f7e136b96cec13cc7c617ea7c59d6fc34edbe9bc79467efbc16aee"),
 }

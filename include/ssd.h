@@ -59,10 +59,13 @@ enum {
     SSD_FLAG_SPLIT_BC = 8,         /* ssd_bwd_segmented, tensor-core path: dB and dC by two kernels that each mask the
                                       score tiles themselves, instead of the one that masks them once for both (a
                                       cross-check; the same values up to the order of the fp32 head sums) */
-    SSD_FLAG_SERIAL = 4            /* ssd_bwd_segmented: launch every kernel on `stream` itself, in order.  By default
-                                      the tensor-core path runs its three mutually independent gradient kernels of a
-                                      segment on two library-owned helper streams forked off `stream` and joined back
-                                      into it before the call returns to the next segment; results are the same bits */
+    SSD_FLAG_SERIAL = 4            /* ssd_fwd / ssd_fwd_segmented / ssd_bwd_segmented: launch every kernel on `stream`
+                                      itself, in order.  By default the tensor-core path, when there is more than one
+                                      segment, runs a segment's state chain (chunk sums, state passes) one segment ahead
+                                      of the large kernels, and the backward's dB/dC kernel and finishing kernels beside
+                                      dx, on library-owned helper streams forked off `stream` and joined back into it
+                                      before the call's last kernel; results are the same bits.  ssd_fwd_static_ws
+                                      always runs in order on `stream` */
 };
 
 /* `op` of ssd_workspace_bytes */

@@ -125,3 +125,9 @@ def test_helper_streams_change_no_bit_and_respect_caller_stream():
     for k, v in g.items():
         if v is not None:
             assert torch.equal(v, ref[k]), k
+    # the forward with its state chain one segment ahead on a helper stream, same check
+    with torch.cuda.stream(s):
+        y, h_final, boundary = libssd.ssd_fwd_segmented(inp["x"], inp["dt"], inp["A"], inp["Bm"], inp["Cm"], inp["D"],
+                                                        inp["h0"], chunk=cfg.chunk, seg=cfg.seg, stream=s)
+    s.synchronize()
+    assert torch.equal(y, ref["y"]) and torch.equal(h_final, ref["h_final"]) and torch.equal(boundary, ref["boundary"])
