@@ -23,7 +23,6 @@ namespace {
 constexpr int CV_THREADS = 128;   // x 4 channels = 512 channels per CTA
 constexpr int CV_CH = 4;          // channels per thread: one 8-byte bf16 vector (16 bytes in fp32)
 constexpr int CV_TILE_F = 32;     // tokens per CTA, forward
-constexpr int CV_TILE_B = 32;     // tokens per CTA, backward (it stages u and dout, with three more tokens of each)
 
 // 1 / (1 + e^-x) from one ex2.approx and one rcp.approx (relative error of the order of 1e-7; the kernels are bound
 // by instruction issue, not by memory, and an IEEE division alone would cost as much as the rest of an element)
@@ -107,6 +106,8 @@ __global__ void __launch_bounds__(CV_THREADS) k_conv_fwd(const T *u, long long u
     __shared__ uint32_t abort_flag;
     __shared__ unsigned int status_dummy;
     T *su = reinterpret_cast<T *>(cv_smem);                       // [CV_TILE_F + 3][512]
+    pdl_launch_dependents();
+    pdl_wait();       // the previous kernel of the stream (a neighbouring segment's) has finished
     const int cbase = blockIdx.x * 512, nch = min(512, C - cbase);
     const int c0 = cbase + threadIdx.x * CV_CH;
     const int b = blockIdx.z;
@@ -164,45 +165,90 @@ __global__ void __launch_bounds__(CV_THREADS) k_conv_fwd(const T *u, long long u
     }
 }
 
-// Backward over one token tile.  dpre[t] = dout[t] * silu'(pre[t]);  du[t] = sum_k w[k] dpre[t+3-k], so a tile also
-// forms dpre of the three tokens to its right (for du only); past the end of the segment they are not formed: their
-// effect on the last three tokens arrives as `dtail`.  dw, dbias: the tile's own tokens.
+// Backward over a range of consecutive tokens.  dpre[t] = dout[t] * silu'(pre[t]);  du[t] = sum_k w[k] dpre[t+3-k].
+// A CTA owns 512 channels and walks its range front to back with the last three inputs and the last four dpre in
+// registers, so nothing is staged or formed twice inside the range; only at its end does it form dpre of the three
+// tokens behind it (for its own last du's; past the end of the segment they are not formed: their effect arrives
+// as `dtail`).  The rows of u and dout stream through a ring of 8-token stages filled by a producer warp with one
+// bulk copy per row, so the loads of later stages are in flight while a stage is being consumed.
+// dw, dbias: one partial per range, the range's own tokens.
+constexpr int CV_STG_TOK = 8;
+constexpr int CV_STAGES = 3;
+constexpr int CV_BWD_THREADS = CV_THREADS + 32;   // four compute warps and the producer warp
+
 template <typename T>
-__global__ void __launch_bounds__(CV_THREADS) k_conv_bwd(const T *u, long long u_bs, const float *w, const float *bias,
-                                                         const T *state_in, const T *dout, const float *dtail, T *du,
-                                                         float *part, int L, int C) {
+__global__ void __launch_bounds__(CV_BWD_THREADS, 4)
+k_conv_bwd(const T *u, long long u_bs, const float *w, const float *bias, const T *state_in, const T *dout,
+           const float *dtail, T *du, float *dstate, float *part, int L, int C, int RL) {
     extern __shared__ __align__(128) unsigned char cv_smem[];
-    __shared__ uint64_t bar;
+    __shared__ uint64_t full[CV_STAGES], empty[CV_STAGES];
     __shared__ uint32_t abort_flag;
     __shared__ unsigned int status_dummy;
-    T *su = reinterpret_cast<T *>(cv_smem);                       // [CV_TILE_B + 6][512]  u rows t_begin-3 .. s_end
-    T *sg = su + (size_t)(CV_TILE_B + 6) * 512;                   // [CV_TILE_B + 3][512]  dout rows t_begin .. s_end
+    T *ring = reinterpret_cast<T *>(cv_smem);                     // [stage][u rows | dout rows][512]
+    pdl_launch_dependents();
+    pdl_wait();
     const int cbase = blockIdx.x * 512, nch = min(512, C - cbase);
-    const int c0 = cbase + threadIdx.x * CV_CH;
     const int b = blockIdx.z;
-    const long long t_begin = (long long)blockIdx.y * CV_TILE_B, t_end = min(t_begin + (long long)CV_TILE_B, (long long)L);
-    const long long s_end = min(t_end + 3, (long long)L);
+    const long long r_begin = (long long)blockIdx.y * RL, r_end = min(r_begin + (long long)RL, (long long)L);
+    const int ntok = (int)(r_end - r_begin), nst = (ntok + CV_STG_TOK - 1) / CV_STG_TOK;
     const T *ub = u + (size_t)b * u_bs, *gb = dout + (size_t)b * u_bs;
     const T *sb = state_in ? state_in + (size_t)b * 3 * C : nullptr;
     T *dub = du + (size_t)b * u_bs;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        mbar_init(&bar, 2);
+        for (int i = 0; i < CV_STAGES; ++i) {
+            mbar_init(&full[i], 1);
+            mbar_init(&empty[i], CV_THREADS / 32);    // one arrival per compute warp
+        }
         abort_flag = 0;
         status_dummy = 0;
         fence_barrier_init();
     }
-    if (!sb && t_begin < 3)
-        for (int i = threadIdx.x; i < (int)(3 - t_begin) * 512; i += CV_THREADS) su[i] = (T)0.f;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        stage_rows(su, ub, sb, t_begin - 3, s_end, C, cbase, nch, &bar);
-        stage_rows(sg, gb, (const T *)nullptr, t_begin, s_end, C, cbase, nch, &bar);
+    if (warp == CV_THREADS / 32) {
+        // ---- producer
+        if (lane == 0) {
+            const uint32_t row_bytes = (uint32_t)nch * sizeof(T);
+            for (int i = 0; i < nst; ++i) {
+                const int slot = i % CV_STAGES;
+                if (i >= CV_STAGES) mbar_wait(&empty[slot], ((i / CV_STAGES) - 1) & 1, &abort_flag, &status_dummy);
+                const long long t0 = r_begin + (long long)i * CV_STG_TOK;
+                const int n = (int)min((long long)CV_STG_TOK, r_end - t0);
+                mbar_arrive_expect_tx(&full[slot], 2u * (uint32_t)n * row_bytes);
+                T *su = ring + (size_t)slot * (2 * CV_STG_TOK * 512), *sg = su + CV_STG_TOK * 512;
+                for (int j = 0; j < n; ++j) {
+                    bulk_load(su + (size_t)j * 512, ub + (size_t)(t0 + j) * C + cbase, row_bytes, &full[slot]);
+                    bulk_load(sg + (size_t)j * 512, gb + (size_t)(t0 + j) * C + cbase, row_bytes, &full[slot]);
+                }
+            }
+        }
+        return;
     }
-    const bool active = c0 < C;
+    const int c0 = cbase + threadIdx.x * CV_CH;
+    const bool active = c0 < C;      // inactive threads (past the last channel) still take part in the hand-overs
     // two channel pairs per thread: every quantity below is a float2 over (c, c + 1), so that the multiply-adds
-    // issue as packed two-lane instructions (the kernel is bound by instruction issue as much as by memory)
+    // issue as packed two-lane instructions
     constexpr int NP = CV_CH / 2;
+    const float2 zero2 = make_float2(0.f, 0.f), one2 = make_float2(1.f, 1.f), mone2 = make_float2(-1.f, -1.f);
     float2 wk[NP][4], bs[NP];
+    float2 x0[NP], x1[NP], x2[NP], x3[NP];
+    float2 d0[NP], d1[NP], d2[NP], d3[NP];     // dpre[t], dpre[t+1], dpre[t+2], dpre[t+3] while emitting du[t]
+    float2 aw[NP][4], ab[NP];
+    const bool head_range = (dstate != nullptr) && blockIdx.y == 0;
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+        aw[i][0] = aw[i][1] = aw[i][2] = aw[i][3] = zero2;
+        ab[i] = zero2;
+        d0[i] = d1[i] = d2[i] = d3[i] = zero2;
+        x0[i] = x1[i] = x2[i] = x3[i] = zero2;
+        wk[i][0] = wk[i][1] = wk[i][2] = wk[i][3] = bs[i] = zero2;
+    }
+    // the input at token t of the segment; in front of it the carried state, or zeros
+    auto ld_u = [&](long long t, float2 *v) {
+        if (t >= 0) ld2x2(ub + (size_t)t * C + c0, v[0], v[1]);
+        else if (sb) ld2x2(sb + (size_t)(3 + t) * C + c0, v[0], v[1]);
+        else v[0] = v[1] = zero2;
+    };
     if (active) {
 #pragma unroll
         for (int i = 0; i < NP; ++i) {
@@ -212,38 +258,22 @@ __global__ void __launch_bounds__(CV_THREADS) k_conv_bwd(const T *u, long long u
             wk[i][2] = make_float2(wa.z, wb.z); wk[i][3] = make_float2(wa.w, wb.w);
             bs[i] = make_float2(bias[c0 + 2 * i], bias[c0 + 2 * i + 1]);
         }
+        ld_u(r_begin - 3, x0);
+        ld_u(r_begin - 2, x1);
+        ld_u(r_begin - 1, x2);
     }
-    mbar_wait(&bar, 0, &abort_flag, &status_dummy);
-    if (!active) return;
-    const T *spu = su + threadIdx.x * CV_CH, *spg = sg + threadIdx.x * CV_CH;
-    const float2 zero2 = make_float2(0.f, 0.f), one2 = make_float2(1.f, 1.f), mone2 = make_float2(-1.f, -1.f);
-    float2 x0[NP], x1[NP], x2[NP], x3[NP];
-    float2 d0[NP], d1[NP], d2[NP], d3[NP];     // dpre[t], dpre[t+1], dpre[t+2], dpre[t+3] while emitting du[t]
-    float2 aw[NP][4], ab[NP];
-#pragma unroll
-    for (int i = 0; i < NP; ++i) {
-        aw[i][0] = aw[i][1] = aw[i][2] = aw[i][3] = zero2;
-        ab[i] = zero2;
-        d0[i] = d1[i] = d2[i] = d3[i] = zero2;
-    }
-    ld2x2(spu, x0[0], x0[1]);
-    ld2x2(spu + 512, x1[0], x1[1]);
-    ld2x2(spu + 1024, x2[0], x2[1]);
-    const int ns = (int)(s_end - t_begin), nt = (int)(t_end - t_begin);
-#pragma unroll 4
-    for (int j = 0; j < ns + 3; ++j) {                     // s = t_begin + j
+    // dpre of token s from its input x3 (the window x0..x2 holds the three before it) and g = dout[s]; own tokens
+    // also feed the weight and bias gradients.  Then the windows move on and du[s - 3] is complete.
+    auto token = [&](long long s, const float2 *g, bool own, bool formed) {
         float2 dp[NP];
-        if (j < ns) {
-            float2 g[NP];
-            ld2x2(spu + (size_t)(j + 3) * 512, x3[0], x3[1]);
-            ld2x2(spg + (size_t)j * 512, g[0], g[1]);
 #pragma unroll
-            for (int i = 0; i < NP; ++i) {
+        for (int i = 0; i < NP; ++i) {
+            if (formed) {
                 const float2 pre = __ffma2_rn(wk[i][3], x3[i], __ffma2_rn(wk[i][2], x2[i], __ffma2_rn(wk[i][1], x1[i], __ffma2_rn(wk[i][0], x0[i], bs[i]))));
                 const float2 sgm = sigmoid_fast2(pre);
                 // dpre = dout * silu'(pre),  silu'(z) = s (1 + z (1 - s))
                 dp[i] = __fmul2_rn(__fmul2_rn(g[i], sgm), __ffma2_rn(pre, __ffma2_rn(sgm, mone2, one2), one2));
-                if (j < nt) {   // the tile's own tokens: weight and bias gradients
+                if (own) {
                     aw[i][0] = __ffma2_rn(dp[i], x0[i], aw[i][0]);
                     aw[i][1] = __ffma2_rn(dp[i], x1[i], aw[i][1]);
                     aw[i][2] = __ffma2_rn(dp[i], x2[i], aw[i][2]);
@@ -251,17 +281,38 @@ __global__ void __launch_bounds__(CV_THREADS) k_conv_bwd(const T *u, long long u
                     ab[i] = __fadd2_rn(ab[i], dp[i]);
                 }
                 x0[i] = x1[i]; x1[i] = x2[i]; x2[i] = x3[i];
+            } else {
+                dp[i] = zero2;
             }
-        } else {
-#pragma unroll
-            for (int i = 0; i < NP; ++i) dp[i] = zero2;
+            d0[i] = d1[i]; d1[i] = d2[i]; d2[i] = d3[i]; d3[i] = dp[i];
         }
-        // shift the dpre window; after it d3 = dpre[s], d0 = dpre[s-3]: du[s-3] is complete
+        if (head_range && s == 2) {
+            // What the first three dpre rows of the segment (now d1, d2, d3) send to the three tokens in front of it:
+            // token -3 feeds pre[0] through w[0]; token -2: pre[0] w[1], pre[1] w[0]; token -1: pre[0] w[2], pre[1] w[1],
+            // pre[2] w[0].
+            float *ds = dstate + (size_t)b * 3 * C + c0;
+            float e[CV_CH];
 #pragma unroll
-        for (int i = 0; i < NP; ++i) { d0[i] = d1[i]; d1[i] = d2[i]; d2[i] = d3[i]; d3[i] = dp[i]; }
-        const int jt = j - 3;
-        if (jt >= 0 && jt < nt) {
-            const long long t = t_begin + jt;
+            for (int i = 0; i < NP; ++i) {
+                const float2 v = __fmul2_rn(wk[i][0], d1[i]);
+                e[2 * i] = v.x; e[2 * i + 1] = v.y;
+            }
+            st4(ds, e);
+#pragma unroll
+            for (int i = 0; i < NP; ++i) {
+                const float2 v = __ffma2_rn(wk[i][0], d2[i], __fmul2_rn(wk[i][1], d1[i]));
+                e[2 * i] = v.x; e[2 * i + 1] = v.y;
+            }
+            st4(ds + (size_t)C, e);
+#pragma unroll
+            for (int i = 0; i < NP; ++i) {
+                const float2 v = __ffma2_rn(wk[i][0], d3[i], __ffma2_rn(wk[i][1], d2[i], __fmul2_rn(wk[i][2], d1[i])));
+                e[2 * i] = v.x; e[2 * i + 1] = v.y;
+            }
+            st4(ds + (size_t)2 * C, e);
+        }
+        const long long t = s - 3;
+        if (t >= r_begin) {
             float o[CV_CH];
 #pragma unroll
             for (int i = 0; i < NP; ++i) {
@@ -277,8 +328,38 @@ __global__ void __launch_bounds__(CV_THREADS) k_conv_bwd(const T *u, long long u
             }
             st4(dub + (size_t)t * C + c0, o);
         }
+    };
+    for (int i = 0; i < nst; ++i) {
+        const int slot = i % CV_STAGES;
+        mbar_wait(&full[slot], (i / CV_STAGES) & 1, &abort_flag, &status_dummy);
+        if (active) {
+            const T *spu = ring + (size_t)slot * (2 * CV_STG_TOK * 512) + threadIdx.x * CV_CH, *spg = spu + CV_STG_TOK * 512;
+            const long long t0 = r_begin + (long long)i * CV_STG_TOK;
+            const int n = (int)min((long long)CV_STG_TOK, r_end - t0);
+#pragma unroll 4
+            for (int j = 0; j < n; ++j) {
+                float2 g[NP];
+                ld2x2(spu + (size_t)j * 512, x3[0], x3[1]);
+                ld2x2(spg + (size_t)j * 512, g[0], g[1]);
+                token(t0 + j, g, true, true);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[slot]);      // this warp has read the stage
     }
-    // partial weight / bias gradients of this tile: part[b][tile][5][C]
+    if (!active) return;
+    // the three tokens behind the range complete its last du's (plain loads: 16 bytes per thread and token)
+    for (int k = 0; k < 3; ++k) {
+        const long long s = r_end + k;
+        float2 g[NP] = {zero2, zero2};
+        const bool formed = s < (long long)L;
+        if (formed) {
+            ld2x2(ub + (size_t)s * C + c0, x3[0], x3[1]);
+            ld2x2(gb + (size_t)s * C + c0, g[0], g[1]);
+        }
+        token(s, g, false, formed);
+    }
+    // partial weight / bias gradients of this range: part[b][range][5][C]
     {
         float *pp = part + (((size_t)b * gridDim.y + blockIdx.y) * 5) * C + c0;
         float col[CV_CH];
@@ -294,64 +375,14 @@ __global__ void __launch_bounds__(CV_THREADS) k_conv_bwd(const T *u, long long u
     }
 }
 
-// What the first three dpre rows of the segment send to the three tokens in front of it (their dpre is recomputed
-// here: three tokens per channel, plain loads).
-template <typename T>
-__global__ void __launch_bounds__(CV_THREADS) k_conv_dstate(const T *u, long long u_bs, const float *w, const float *bias,
-                                                            const T *state_in, const T *dout, float *dstate, int L, int C) {
-    const int c0 = (blockIdx.x * CV_THREADS + threadIdx.x) * CV_CH;
-    if (c0 >= C) return;
-    const int b = blockIdx.z;
-    const T *ub = u + (size_t)b * u_bs, *gb = dout + (size_t)b * u_bs;
-    const T *sb = state_in ? state_in + (size_t)b * 3 * C : nullptr;
-    float wk[CV_CH][4], bs[CV_CH];
-#pragma unroll
-    for (int i = 0; i < CV_CH; ++i) {
-        const float4 wv = *reinterpret_cast<const float4 *>(w + (size_t)(c0 + i) * 4);
-        wk[i][0] = wv.x; wk[i][1] = wv.y; wk[i][2] = wv.z; wk[i][3] = wv.w;
-        bs[i] = bias[c0 + i];
-    }
-    float y0[CV_CH], y1[CV_CH], y2[CV_CH], y3[CV_CH], q[3][CV_CH];
-#pragma unroll
-    for (int i = 0; i < CV_CH; ++i) y0[i] = y1[i] = y2[i] = 0.f;
-    if (sb) {
-        ld4(sb + c0, y0);
-        ld4(sb + (size_t)C + c0, y1);
-        ld4(sb + (size_t)2 * C + c0, y2);
-    }
-#pragma unroll
-    for (int s = 0; s < 3; ++s) {
-        float g[CV_CH];
-        ld4(ub + (size_t)s * C + c0, y3);
-        ld4(gb + (size_t)s * C + c0, g);
-#pragma unroll
-        for (int i = 0; i < CV_CH; ++i) {
-            const float pre = fmaf(wk[i][3], y3[i], fmaf(wk[i][2], y2[i], fmaf(wk[i][1], y1[i], fmaf(wk[i][0], y0[i], bs[i]))));
-            const float sgm = sigmoid_fast(pre);
-            q[s][i] = g[i] * sgm * fmaf(pre, 1.f - sgm, 1.f);
-            y0[i] = y1[i]; y1[i] = y2[i]; y2[i] = y3[i];
-        }
-    }
-    // token -3 feeds pre[0] through w[0]; token -2: pre[0] w[1], pre[1] w[0]; token -1: pre[0] w[2], pre[1] w[1], pre[2] w[0]
-    float e[CV_CH];
-    float *ds = dstate + (size_t)b * 3 * C + c0;
-#pragma unroll
-    for (int i = 0; i < CV_CH; ++i) e[i] = wk[i][0] * q[0][i];
-    st4(ds, e);
-#pragma unroll
-    for (int i = 0; i < CV_CH; ++i) e[i] = fmaf(wk[i][0], q[1][i], wk[i][1] * q[0][i]);
-    st4(ds + (size_t)C, e);
-#pragma unroll
-    for (int i = 0; i < CV_CH; ++i) e[i] = fmaf(wk[i][0], q[2][i], fmaf(wk[i][1], q[1][i], wk[i][2] * q[0][i]));
-    st4(ds + (size_t)2 * C, e);
-}
-
 // dw[c][k], dbias[c] from the tile partials, in fp64 and in a fixed order: a CTA owns 32 adjacent channels of one of the
 // five rows (four taps, bias); its eight warps take the tiles round-robin (coalesced 128-byte reads, several in flight),
 // then the eight partial sums are added in warp order.
 __global__ void __launch_bounds__(256) k_conv_reduce(const float *part, float *dw, float *dbias, int C, int ntiles, int B,
                                                      int accumulate) {
     __shared__ double red[8][32];
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
     const int nblk = (C + 31) / 32;
     const int k = blockIdx.x / nblk, c = (blockIdx.x % nblk) * 32 + lane;
@@ -383,31 +414,34 @@ cudaError_t conv_fwd_t(const T *u, long long u_bs, const float *w, const float *
     cudaError_t e = cudaFuncSetAttribute(k_conv_fwd<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     dim3 grid((C + 511) / 512, (L + CV_TILE_F - 1) / CV_TILE_F, B);
-    k_conv_fwd<T><<<grid, CV_THREADS, smem, st>>>(u, u_bs, w, bias, state_in, out, state_out, L, C);
-    return cudaGetLastError();
+    return launch_pdl(k_conv_fwd<T>, grid, dim3(CV_THREADS), (size_t)smem, st, u, u_bs, w, bias, state_in, out, state_out, L, C);
+}
+
+// Tokens per CTA of the backward: about four CTAs per SM over the whole launch, whole stages, and never
+// more ranges than conv_tiles() promises scratch for.
+static int conv_range_len(int B, int L, int C) {
+    const int nblk = (C + 511) / 512;
+    int want = (4 * 148) / (nblk * B);
+    if (want < 1) want = 1;
+    int rl = ((L + want - 1) / want + CV_STG_TOK - 1) / CV_STG_TOK * CV_STG_TOK;
+    if (rl < 32) rl = 32;
+    return rl;
 }
 
 template <typename T>
 cudaError_t conv_bwd_t(const T *u, long long u_bs, const float *w, const float *bias, const T *state_in, const T *dout,
-                       const float *dtail, T *du, float *dstate, float *part, int B, int L, int C, cudaStream_t st) {
-    const int smem = (2 * CV_TILE_B + 9) * 512 * (int)sizeof(T);
+                       const float *dtail, T *du, float *dstate, float *part, int B, int L, int C, int RL, cudaStream_t st) {
+    const int smem = CV_STAGES * 2 * CV_STG_TOK * 512 * (int)sizeof(T);
     cudaError_t e = cudaFuncSetAttribute(k_conv_bwd<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    dim3 grid((C + 511) / 512, (L + CV_TILE_B - 1) / CV_TILE_B, B);
-    k_conv_bwd<T><<<grid, CV_THREADS, smem, st>>>(u, u_bs, w, bias, state_in, dout, dtail, du, part, L, C);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    if (dstate) {
-        dim3 g1((C / CV_CH + CV_THREADS - 1) / CV_THREADS, 1, B);
-        k_conv_dstate<T><<<g1, CV_THREADS, 0, st>>>(u, u_bs, w, bias, state_in, dout, dstate, L, C);
-        e = cudaGetLastError();
-    }
-    return e;
+    dim3 grid((C + 511) / 512, (L + RL - 1) / RL, B);
+    return launch_pdl(k_conv_bwd<T>, grid, dim3(CV_BWD_THREADS), (size_t)smem, st, u, u_bs, w, bias, state_in, dout, dtail, du, dstate,
+                      part, L, C, RL);
 }
 
 }  // namespace
 
-int conv_tiles(int L) { return (L + CV_TILE_B - 1) / CV_TILE_B; }
+int conv_tiles(int L) { return (L + 31) / 32; }
 
 cudaError_t launch_conv_fwd(int dtype, const void *u, long long u_bs, const float *w, const float *bias,
                             const void *state_in, void *out, void *state_out, int B, int L, int C, cudaStream_t st) {
@@ -421,16 +455,17 @@ cudaError_t launch_conv_fwd(int dtype, const void *u, long long u_bs, const floa
 cudaError_t launch_conv_bwd(int dtype, const void *u, long long u_bs, const float *w, const float *bias,
                             const void *state_in, const void *dout, const float *dtail, void *du, float *dstate,
                             float *dw, float *dbias, int accumulate, float *part, int B, int L, int C, cudaStream_t st) {
+    const int RL = conv_range_len(B, L, C);
     cudaError_t e;
     if (dtype == SSD_DTYPE_F32)
         e = conv_bwd_t<float>((const float *)u, u_bs, w, bias, (const float *)state_in, (const float *)dout, dtail, (float *)du,
-                              dstate, part, B, L, C, st);
+                              dstate, part, B, L, C, RL, st);
     else
         e = conv_bwd_t<__nv_bfloat16>((const __nv_bfloat16 *)u, u_bs, w, bias, (const __nv_bfloat16 *)state_in,
-                                      (const __nv_bfloat16 *)dout, dtail, (__nv_bfloat16 *)du, dstate, part, B, L, C, st);
+                                      (const __nv_bfloat16 *)dout, dtail, (__nv_bfloat16 *)du, dstate, part, B, L, C, RL, st);
     if (e != cudaSuccess) return e;
-    k_conv_reduce<<<5 * ((C + 31) / 32), 256, 0, st>>>(part, dw, dbias, C, conv_tiles(L), B, accumulate);
-    return cudaGetLastError();
+    return launch_pdl(k_conv_reduce, dim3(5 * ((C + 31) / 32)), dim3(256), (size_t)0, st, (const float *)part, dw, dbias, C,
+                      (L + RL - 1) / RL, B, accumulate);
 }
 
 }  // namespace ssd
