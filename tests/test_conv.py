@@ -67,7 +67,8 @@ def test_oracle_conv_is_invariant_to_segmentation():
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("dtype,B,L,C", [("fp32", 2, 300, 40), ("bf16", 2, 300, 40), ("bf16", 1, 1024, 5376)])
+@pytest.mark.parametrize("dtype,B,L,C", [("fp32", 2, 300, 40), ("bf16", 2, 300, 40), ("bf16", 1, 1024, 5376),
+                                         ("bf16", 6, 1536, 2560)])   # the last: 88 tokens (11 ring stages) per backward CTA
 def test_conv_matches_oracle_whole_and_segmented(dtype, B, L, C):
     from paper_2411_19460_b200 import libssd
     from tests.parity_util import TOL, relerr
