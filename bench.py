@@ -876,7 +876,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="config 3: number of layers (default 64)")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="time plain stream launches instead of the replay of the step captured in a CUDA graph")
-    ap.add_argument("--serial", action="store_true", help="backward: no helper streams, every kernel in order on one stream")
+    ap.add_argument("--serial", action="store_true", help="no helper streams: every kernel of the forward and the backward in order on one stream")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-tokens", type=int, default=32768, help="tokens in the cpu_baseline sample")

@@ -5,12 +5,12 @@
 // the next one; backward walks the segments right to left and hands the gradient that reaches the three
 // tokens in front of a segment to the segment on its left.
 //     pre[t,c] = bias[c] + sum_{k<4} w[c,k] u[t-3+k, c]        out = pre * sigmoid(pre)
-// Bandwidth-shaped kernels: a CTA owns (a block of up to 512 adjacent channels) x (a tile of tokens); one thread
-// brings the tile's rows (plus the three-token halo) into shared memory with bulk async copies, one per token row
-// (the channels of a row are contiguous: up to 1 KB), so that many kilobytes per SM are in flight without holding
-// registers; then a thread owns 4 adjacent channels and walks the tile with a sliding window in registers, writing
-// its results straight to global memory (8 or 16 bytes per thread, coalesced over the channels).  Weight and bias
-// gradients: one partial per token tile, then a fixed-order sum (no atomics).
+// Bandwidth-shaped kernels over 512 adjacent channels per CTA, a thread owning 4 of them with a sliding window in
+// registers; rows reach shared memory by bulk async copies, one per token row (the channels of a row are contiguous:
+// up to 1 KB), so that many kilobytes per SM are in flight without holding registers, and results go straight to
+// global memory (8 or 16 bytes per thread, coalesced over the channels).  Forward: one 32-token tile per CTA, staged
+// whole (plus the three-token halo).  Backward: a range of tokens per CTA streamed through a ring of 8-token stages.
+// Weight and bias gradients: one partial per backward CTA, then a fixed-order sum (no atomics).
 #include "ssd_internal.h"
 #include "ssd_sm100.cuh"
 
