@@ -49,6 +49,9 @@ struct Layout {
     // second copies (tensor-core path, more than one segment): the state chain of a segment runs on a helper
     // stream while the large kernels of its neighbour still read the first copies
     size_t cs_b, dtT_b, Hbf_b, Gbf_b, rho2_b, ghdot_b;
+    // and of what the large kernels of the backward leave for a segment's finishing kernels, so that the next
+    // segment's large kernels need not wait for those
+    size_t ddt_dir_b, rho_b, rhob_b, psi_b, psib_b, psi2_b, pB_b, pC_b;
     size_t total;
 };
 
@@ -202,6 +205,14 @@ static void make_layout(const Plan &pl, int op, Layout &lo) {
         lo.ghdot_b = take(twin ? BH * pl.ncs * 8 * sizeof(float) : 0);
         lo.rhob = take(pl.use_tc ? vec : 0);
         lo.psib = take(pl.use_tc ? vec : 0);
+        lo.ddt_dir_b = take(twin ? vec : 0);
+        lo.rho_b = take(twin ? vec : 0);
+        lo.rhob_b = take(twin ? vec : 0);
+        lo.psi_b = take(twin ? vec : 0);
+        lo.psib_b = take(twin ? vec : 0);
+        lo.psi2_b = take(twin ? vec : 0);
+        lo.pB_b = take(twin ? part : 0);
+        lo.pC_b = take(twin ? part : 0);
     }
     lo.total = o;
 }
@@ -323,6 +334,16 @@ static void select_copy(const Layout &lo, void *ws, bool second, bool bwd, SegPa
         sp.Gbf = (__nv_bfloat16 *)(w + (second ? lo.Gbf_b : lo.Gbf));
         sp.rho2 = (float *)(w + (second ? lo.rho2_b : lo.rho2));
         sp.ghdot = (float *)(w + (second ? lo.ghdot_b : lo.ghdot));
+        sp.ddt_dir = (float *)(w + (second ? lo.ddt_dir_b : lo.ddt_dir));
+        sp.rho = (float *)(w + (second ? lo.rho_b : lo.rho));
+        sp.psi = (float *)(w + (second ? lo.psi_b : lo.psi));
+        sp.psi2 = (float *)(w + (second ? lo.psi2_b : lo.psi2));
+        sp.pB = (float *)(w + (second ? lo.pB_b : lo.pB));
+        sp.pC = (float *)(w + (second ? lo.pC_b : lo.pC));
+        if (sp.rhob) {   // the fused dB/dC kernel is in use
+            sp.rhob = (float *)(w + (second ? lo.rhob_b : lo.rhob));
+            sp.psib = (float *)(w + (second ? lo.psib_b : lo.psib));
+        }
     }
 }
 
@@ -566,13 +587,10 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
                 SSD_LAUNCH(KIND_STATE_PASS_BWD, launch_state_pass_bwd(sp, ginit, gleft, true, st));
                 SSD_TRY(cudaEventRecord(side->chain_done[par], st));
             }
-            // ---- big(k); its outputs (direct ddt, rho, psi, partial dB/dC slices) are read by tail(k+1)
+            // ---- big(k); what it leaves for tail(k) (direct ddt, rho, psi, partial dB/dC slices) alternates too, and
+            // chain(k) has already waited for tail(k+2), the last reader of this copy
             SSD_TRY(cudaStreamWaitEvent(st, side->chain_done[par], 0));
             SSD_TRY(cudaStreamWaitEvent(bcs, side->chain_done[par], 0));
-            if (k < pl.nseg - 1) {
-                SSD_TRY(cudaStreamWaitEvent(st, side->tail_done[par ^ 1], 0));
-                SSD_TRY(cudaStreamWaitEvent(bcs, side->tail_done[par ^ 1], 0));
-            }
             {
                 cudaStream_t st = bcs;
                 if (fused_bc) {
