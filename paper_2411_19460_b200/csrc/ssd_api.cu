@@ -55,6 +55,11 @@ struct Layout {
     size_t total;
 };
 
+// Second copies of the per-segment scratch (and with them the state chain running one segment ahead) pay only when
+// there are segments enough to pipeline; with two or three long segments they would cost a third more scratch for
+// a per cent or two.
+static const int kMinSegmentsForTwins = 4;
+
 struct Plan {
     int B, L, H, P, N, G, Q, seg, nseg, ncs, nct, hpg, nsl, nslf, dtype;
     bool use_tc;
@@ -180,7 +185,7 @@ static void make_layout(const Plan &pl, int op, Layout &lo) {
     lo.Hst = take(st * sizeof(float));
     lo.Hbf = take(pl.use_tc ? st * 2 : 0);
     lo.hcarry = take(BH * PN * sizeof(float));
-    const bool twin = pl.use_tc && pl.nseg > 1;
+    const bool twin = pl.use_tc && pl.nseg >= kMinSegmentsForTwins;
     lo.cs_b = take(twin ? vec : 0);
     lo.dtT_b = take(twin ? vec : 0);
     lo.Hbf_b = take(twin ? st * 2 : 0);
@@ -374,7 +379,7 @@ static int forward_impl(const ssd_shape_t *shape, const void *x, const float *dt
     TcMaps maps;
     if (pl.use_tc && !tc_make_maps(sp, maps)) return SSD_ECUDA;
     const long long PN = (long long)pl.P * pl.N;
-    if (pl.use_tc && pl.nseg > 1 && may_use_helper_stream && !(shape->flags & SSD_FLAG_SERIAL) && !g_prof_on) {
+    if (pl.use_tc && pl.nseg >= kMinSegmentsForTwins && may_use_helper_stream && !(shape->flags & SSD_FLAG_SERIAL) && !g_prof_on) {
         // Algorithm 1 with the state chain one segment ahead: chunk states and state pass of segment k run on a
         // helper stream while the caller's stream still computes y of segment k-1, whose last, partly idle wave
         // they fill.  What both touch (cumulative sums, dt per chunk, bf16 chunk states) exists twice and
@@ -559,7 +564,7 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
         // idle wave leaves free; tail(k) runs under big(k-1)'s predecessors likewise.  What chain(k-1) writes and
         // big(k) / tail(k) read exists twice and alternates with the segment (cumulative sums, dt per chunk, both
         // bf16 state copies, rho2, <G,H>); the fp32 chunk sums and the carried gradient belong to the chain alone.
-        const bool twin = pl.nseg > 1;
+        const bool twin = pl.nseg >= kMinSegmentsForTwins;    // else one copy: chain(k) then also waits for tail(k+1)
         TcMaps maps_b;
         if (twin) {
             select_copy(lo, ws, true, true, sp);
@@ -570,12 +575,12 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
         SSD_TRY(cudaStreamWaitEvent(chain, side->start, 0));
         int par = 0;
         for (int k = pl.nseg - 1; k >= 0; --k) {
-            par = (pl.nseg - 1 - k) & 1;
+            par = twin ? ((pl.nseg - 1 - k) & 1) : 0;
             set_segment(pl, k, sp);
             select_copy(lo, ws, par != 0, true, sp);
             const TcMaps &mk = par ? maps_b : maps;
-            // ---- chain(k); its copy was last read by big(k+2) and tail(k+2)
-            if (k + 2 <= pl.nseg - 1) SSD_TRY(cudaStreamWaitEvent(chain, side->tail_done[par], 0));
+            // ---- chain(k); its copy was last read by big(k+2) and tail(k+2) (of k+1 when there is one copy only)
+            if (k + (twin ? 2 : 1) <= pl.nseg - 1) SSD_TRY(cudaStreamWaitEvent(chain, side->tail_done[par], 0));
             {
                 cudaStream_t st = chain;
                 SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_tc(sp, mk, STATE_MODE_FWD, st));

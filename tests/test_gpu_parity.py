@@ -110,10 +110,11 @@ def test_status_word_clean():
 
 
 @pytest.mark.gpu
-def test_helper_streams_change_no_bit_and_respect_caller_stream():
+@pytest.mark.parametrize("seg", [512, 768, 1024, 2048])   # 4 segments (second scratch copies), 3 (ragged), 2, 1
+def test_helper_streams_change_no_bit_and_respect_caller_stream(seg):
     """The backward's forked helper streams (default) against SSD_FLAG_SERIAL: the same bits, also when the
     caller's stream is not the default one and is the only thing the caller synchronises."""
-    cfg = small(B=2, L=2048, H=8, G=2, seg=512)
+    cfg = small(B=2, L=2048, H=8, G=2, seg=seg)
     inp = make_inputs(cfg, "cuda")
     ref = pu.run_gpu(cfg, inp, flags=libssd.SSD_FLAG_SERIAL)
     s = torch.cuda.Stream()
