@@ -46,7 +46,10 @@ def test_stack_matches_oracle_layer_by_layer():
     inp = make_inputs(cfg, "cuda")
     sp = make_stack_params(cfg, "cuda")
     st = LayerStack(inp["x"], inp["dt"], inp["Bm"], inp["Cm"], sp["A"], sp["D"], sp["W"], chunk=cfg.chunk, seg=cfg.seg)
-    h0 = [torch.randn(cfg.B, cfg.H, cfg.P, cfg.N, device="cuda") * 0.1 for _ in range(cfg.layers)]
+    # seeded: the case must not vary from run to run (dA of four heads over 1 024 tokens is a heavily cancelled sum,
+    # so its relative error swings with how small the sum happens to be: 3e-4 to 6e-3 over the first five seeds)
+    gen = torch.Generator(device="cuda").manual_seed(cfg.seed + 1)
+    h0 = [torch.randn(cfg.B, cfg.H, cfg.P, cfg.N, device="cuda", generator=gen) * 0.1 for _ in range(cfg.layers)]
     for j in range(cfg.layers):
         st.set_h0(j, h0[j])
     st.forward()
@@ -99,7 +102,10 @@ def test_layer_interval_changes_no_bit(interval):
     cfg = CONFIGS[3].scaled(L=1024, H=4, seg=256, layers=4, dh_std=0.0)
     inp = make_inputs(cfg, "cuda")
     sp = make_stack_params(cfg, "cuda")
-    h0 = [torch.randn(cfg.B, cfg.H, cfg.P, cfg.N, device="cuda") * 0.1 for _ in range(cfg.layers)]
+    # seeded: the case must not vary from run to run (dA of four heads over 1 024 tokens is a heavily cancelled sum,
+    # so its relative error swings with how small the sum happens to be: 3e-4 to 6e-3 over the first five seeds)
+    gen = torch.Generator(device="cuda").manual_seed(cfg.seed + 1)
+    h0 = [torch.randn(cfg.B, cfg.H, cfg.P, cfg.N, device="cuda", generator=gen) * 0.1 for _ in range(cfg.layers)]
 
     def run(l):
         st = LayerStack(inp["x"], inp["dt"], inp["Bm"], inp["Cm"], sp["A"], sp["D"], sp["W"], chunk=cfg.chunk,
