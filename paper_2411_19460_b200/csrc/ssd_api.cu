@@ -240,16 +240,18 @@ static int check_device() {
     return cached_ok ? SSD_OK : SSD_EDEVICE;
 }
 
-// Three helper streams per (host thread, device) with the events that fork them off the caller's stream and
-// join them back: s[0] runs the state chain of a segment (chunk states, state passes), s[1] the dB/dC kernel
-// beside dx on the caller's stream, s[2] a segment's two finishing kernels.  Created on first use, never
+// Helper streams per (host thread, device) with the events that fork them off the caller's stream and join them
+// back: s[4] recomputes a segment's chunk states (in the forward: the whole state chain is on s[0]), s[0] runs the
+// state-gradient part of the chain, s[1] / s[3] the dB/dC kernel of even / odd segments beside dx on the caller's
+// stream, s[2] a segment's two finishing kernels.  Created on first use, never
 // destroyed (they hold no device memory); the caller's stream stays the only one the caller has to order
 // against.  Events indexed [2] alternate with the segment, like the second copies of the scratch regions.
 struct SideStreams {
     int dev = -1;
-    cudaStream_t s[3] = {nullptr, nullptr, nullptr};
-    cudaEvent_t start = nullptr, join = nullptr, tail_go = nullptr;
+    cudaStream_t s[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // gradient chain | dB/dC, even | tails | dB/dC, odd | recompute
+    cudaEvent_t start = nullptr;
     cudaEvent_t chain_done[2] = {nullptr, nullptr}, big_done[2] = {nullptr, nullptr}, tail_done[2] = {nullptr, nullptr};
+    cudaEvent_t rec_done[2] = {nullptr, nullptr}, join[2] = {nullptr, nullptr}, dx_done[2] = {nullptr, nullptr};
 };
 static SideStreams *side_streams() {
     static thread_local std::vector<SideStreams> all;
@@ -259,10 +261,10 @@ static SideStreams *side_streams() {
         if (a.dev == dev) return &a;
     SideStreams a;
     a.dev = dev;
-    for (int i = 0; i < 3; ++i)
+    for (int i = 0; i < 5; ++i)
         if (cudaStreamCreateWithFlags(&a.s[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-    cudaEvent_t *evs[] = {&a.start, &a.join, &a.tail_go, &a.chain_done[0], &a.chain_done[1], &a.big_done[0],
-                          &a.big_done[1], &a.tail_done[0], &a.tail_done[1]};
+    cudaEvent_t *evs[] = {&a.start, &a.chain_done[0], &a.chain_done[1], &a.big_done[0], &a.big_done[1], &a.tail_done[0],
+                          &a.tail_done[1], &a.rec_done[0], &a.rec_done[1], &a.join[0], &a.join[1], &a.dx_done[0], &a.dx_done[1]};
     for (cudaEvent_t *ev : evs)
         if (cudaEventCreateWithFlags(ev, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     all.push_back(a);
@@ -570,22 +572,31 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
             select_copy(lo, ws, true, true, sp);
             if (!tc_make_maps(sp, maps_b)) return SSD_ECUDA;
         }
-        cudaStream_t chain = side->s[0], bcs = side->s[1], tails = side->s[2];
+        cudaStream_t grads = side->s[0], recomp = side->s[4], tails = side->s[2];
         SSD_TRY(cudaEventRecord(side->start, st));
-        SSD_TRY(cudaStreamWaitEvent(chain, side->start, 0));
+        SSD_TRY(cudaStreamWaitEvent(recomp, side->start, 0));
+        SSD_TRY(cudaStreamWaitEvent(grads, side->start, 0));
         int par = 0;
         for (int k = pl.nseg - 1; k >= 0; --k) {
             par = twin ? ((pl.nseg - 1 - k) & 1) : 0;
             set_segment(pl, k, sp);
             select_copy(lo, ws, par != 0, true, sp);
             const TcMaps &mk = par ? maps_b : maps;
-            // ---- chain(k); its copy was last read by big(k+2) and tail(k+2) (of k+1 when there is one copy only)
-            if (k + (twin ? 2 : 1) <= pl.nseg - 1) SSD_TRY(cudaStreamWaitEvent(chain, side->tail_done[par], 0));
+            // ---- chain(k), first half: Recompute_Forward.  Its copy was last read by big(k+2) and tail(k+2) (of k+1
+            // when there is one copy only); the fp32 chunk sums belong to this stream alone.
+            if (k + (twin ? 2 : 1) <= pl.nseg - 1) SSD_TRY(cudaStreamWaitEvent(recomp, side->tail_done[par], 0));
             {
-                cudaStream_t st = chain;
+                cudaStream_t st = recomp;
                 SSD_LAUNCH(KIND_CHUNK_STATE, launch_chunk_state_tc(sp, mk, STATE_MODE_FWD, st));
                 SSD_LAUNCH(KIND_STATE_PASS_FWD, launch_state_pass_fwd(sp, boundary + (size_t)k * pl.H * PN, (long long)pl.nseg * pl.H * PN,
                                               nullptr, 0, nullptr, true, st));
+                SSD_TRY(cudaEventRecord(side->rec_done[par], st));
+            }
+            // ---- chain(k), second half: the state gradients, which alone wait for segment k+1 (stream order: the
+            // gradient handed left, and the fp32 contributions that belong to this stream alone)
+            SSD_TRY(cudaStreamWaitEvent(grads, side->rec_done[par], 0));
+            {
+                cudaStream_t st = grads;
                 SSD_LAUNCH(KIND_DSTATE, launch_chunk_state_tc(sp, mk, STATE_MODE_DSTATE, st));
                 const float *ginit = (k == pl.nseg - 1) ? dh_final : sp.gcarry;
                 float *gleft = (k == 0 && dh0) ? dh0 : sp.gcarry;
@@ -593,7 +604,9 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
                 SSD_TRY(cudaEventRecord(side->chain_done[par], st));
             }
             // ---- big(k); what it leaves for tail(k) (direct ddt, rho, psi, partial dB/dC slices) alternates too, and
-            // chain(k) has already waited for tail(k+2), the last reader of this copy
+            // chain(k) has already waited for tail(k+2), the last reader of this copy.  The dB/dC kernels of
+            // neighbouring segments are on different streams: with short segments one alone does not fill the GPU.
+            cudaStream_t bcs = side->s[par ? 3 : 1];
             SSD_TRY(cudaStreamWaitEvent(st, side->chain_done[par], 0));
             SSD_TRY(cudaStreamWaitEvent(bcs, side->chain_done[par], 0));
             {
@@ -604,13 +617,13 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
                     SSD_LAUNCH(KIND_BWD_DC, launch_grad_bc_tc(sp, mk, GB_DC, st));
                     SSD_LAUNCH(KIND_BWD_DB, launch_grad_bc_tc(sp, mk, GB_DB, st));
                 }
-                SSD_TRY(cudaEventRecord(side->join, st));
+                SSD_TRY(cudaEventRecord(side->join[par], st));
             }
             SSD_LAUNCH(KIND_BWD_DX, launch_scan_tc(sp, mk, SC_DX, st));
-            SSD_TRY(cudaStreamWaitEvent(st, side->join, 0));
-            // ---- tail(k)
-            SSD_TRY(cudaEventRecord(side->tail_go, st));
-            SSD_TRY(cudaStreamWaitEvent(tails, side->tail_go, 0));
+            SSD_TRY(cudaEventRecord(side->dx_done[par], st));
+            // ---- tail(k), after both
+            SSD_TRY(cudaStreamWaitEvent(tails, side->dx_done[par], 0));
+            SSD_TRY(cudaStreamWaitEvent(tails, side->join[par], 0));
             {
                 cudaStream_t st = tails;
                 SSD_LAUNCH(KIND_BWD_FINISH, launch_bwd_finish(sp, st));
