@@ -472,7 +472,7 @@ def run_stack(args, rep, dev):
     inp = make_inputs(cfg, dev, seed=cfg.seed + rep.rank)
     sp = make_stack_params(cfg, dev)
     st = LayerStack(inp["x"], inp["dt"], inp["Bm"], inp["Cm"], sp["A"], sp["D"], sp["W"], chunk=cfg.chunk, seg=cfg.seg,
-                    layer_interval=args.layer_interval)
+                    layer_interval=args.layer_interval, flags=(libssd.SSD_FLAG_SERIAL if args.serial else 0))
     out = dict(dx0=torch.empty_like(inp["x"]), dA=torch.zeros(cfg.layers, cfg.H, device=dev),
                dD=torch.zeros(cfg.layers, cfg.H, device=dev))
     stream = torch.cuda.current_stream()

@@ -2,7 +2,11 @@
 // and 2 of the paper keep only each layer's INPUT along the layer axis): layer j maps x_j to
 // y_j = SSD_j(x_j) and hands x_{j+1} = W (y_j + x_j) to the next layer, W a fixed P x P mixing matrix
 // applied per (batch, step, head).  Backward: dz = W^T g_{j+1}; dy_j = dz; dx_j = (SSD backward) + dz.
-// Bandwidth-shaped CUDA-core kernels; bf16 or fp32 I/O, fp32 arithmetic.
+// Bandwidth-shaped kernels; bf16 or fp32 I/O.  fp32: CUDA cores, fp32 arithmetic.  bf16: the 64 x 64 product runs on
+// the tensor cores through warp-level mma (W rounded to bf16 once per CTA, fp32 accumulation): at 4096 multiply-adds
+// per 128-byte row the CUDA-core version was five times over its memory time.
+#include <mma.h>
+
 #include "ssd_internal.h"
 
 namespace ssd {
@@ -83,6 +87,89 @@ __global__ void __launch_bounds__(128) k_glue(const T *a, const T *b, const floa
     }
 }
 
+// The same product for bf16 rows on the tensor cores.  A warp owns 16 consecutive rows (one contiguous 2 KB block of
+// the row-major [rows][64] tensor): it fetches them with 16-byte loads that cover whole 512-byte spans per instruction,
+// forms Z = a (+ b) in bf16 and parks it in a padded shared-memory tile, multiplies it by the bf16 copy of W with
+// 4 x 4 warp-level mma steps (fp32 accumulation), and sends the 16 result rows out the same way, through a padded
+// fp32 staging tile.  Row strides of 72 elements keep the fragment accesses off one bank.
+constexpr int GL_LD = 72;
+template <bool TRANSPOSE>
+__global__ void __launch_bounds__(128) k_glue_bf16_mma(const __nv_bfloat16 *a, const __nv_bfloat16 *b, const float *W,
+                                                       __nv_bfloat16 *out, long long rows_per_batch, long long bstride, int B) {
+    using namespace nvcuda;
+    __shared__ __align__(32) __nv_bfloat16 Wb[64 * GL_LD];
+    __shared__ __align__(32) __nv_bfloat16 zs[4][16 * GL_LD];
+    __shared__ __align__(32) float stage[4][16 * GL_LD];
+    for (int idx = threadIdx.x; idx < 4096; idx += 128) Wb[(idx >> 6) * GL_LD + (idx & 63)] = __float2bfloat16_rn(W[idx]);
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long ntiles = rows_per_batch * B / 16;
+    for (long long t = (long long)blockIdx.x * 4 + warp; t < ntiles; t += (long long)gridDim.x * 4) {
+        const long long row0 = t * 16, bb = row0 / rows_per_batch, rr = row0 % rows_per_batch;
+        const size_t off = (size_t)bb * bstride + (size_t)rr * 64;
+        // 16-byte chunk c of the block (128 of them): row c / 8, columns (c % 8) * 8 ..
+        uint4 va[4], vb[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) va[q] = __ldg(reinterpret_cast<const uint4 *>(a + off) + q * 32 + lane);
+        if (b) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) vb[q] = __ldg(reinterpret_cast<const uint4 *>(b + off) + q * 32 + lane);
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            uint4 z = va[q];
+            if (b) {
+                __nv_bfloat162 *zp = reinterpret_cast<__nv_bfloat162 *>(&z);
+                const __nv_bfloat162 *bp = reinterpret_cast<const __nv_bfloat162 *>(&vb[q]);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) zp[i] = __hadd2(zp[i], bp[i]);
+            }
+            const int c = q * 32 + lane;
+            *reinterpret_cast<uint4 *>(&zs[warp][(c >> 3) * GL_LD + (c & 7) * 8]) = z;
+        }
+        __syncwarp();
+        wmma::fragment<wmma::matrix_a, 16, 16, 16, __nv_bfloat16, wmma::row_major> za[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) wmma::load_matrix_sync(za[k], zs[warp] + k * 16, GL_LD);
+        // out[row, i] = sum_j M[i][j] z[j]: the B operand is element (k = j, n = i) = M[i][j].  M = W: W[n][k], i.e. W
+        // read column-major; M = W^T: W[k][n], row-major.
+#pragma unroll
+        for (int n = 0; n < 4; ++n) {
+            wmma::fragment<wmma::accumulator, 16, 16, 16, float> acc;
+            wmma::fill_fragment(acc, 0.f);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (TRANSPOSE) {
+                    wmma::fragment<wmma::matrix_b, 16, 16, 16, __nv_bfloat16, wmma::row_major> mb;
+                    wmma::load_matrix_sync(mb, Wb + (k * 16) * GL_LD + n * 16, GL_LD);
+                    wmma::mma_sync(acc, za[k], mb, acc);
+                } else {
+                    wmma::fragment<wmma::matrix_b, 16, 16, 16, __nv_bfloat16, wmma::col_major> mb;
+                    wmma::load_matrix_sync(mb, Wb + (n * 16) * GL_LD + k * 16, GL_LD);
+                    wmma::mma_sync(acc, za[k], mb, acc);
+                }
+            }
+            wmma::store_matrix_sync(stage[warp] + n * 16, acc, GL_LD, wmma::mem_row_major);
+        }
+        __syncwarp();
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int c = q * 32 + lane;
+            const float *src = stage[warp] + (c >> 3) * GL_LD + (c & 7) * 8;
+            const float4 v0 = *reinterpret_cast<const float4 *>(src), v1 = *reinterpret_cast<const float4 *>(src + 4);
+            __nv_bfloat162 p0 = __floats2bfloat162_rn(v0.x, v0.y), p1 = __floats2bfloat162_rn(v0.z, v0.w);
+            __nv_bfloat162 p2 = __floats2bfloat162_rn(v1.x, v1.y), p3 = __floats2bfloat162_rn(v1.z, v1.w);
+            uint4 pk;
+            pk.x = *reinterpret_cast<unsigned int *>(&p0);
+            pk.y = *reinterpret_cast<unsigned int *>(&p1);
+            pk.z = *reinterpret_cast<unsigned int *>(&p2);
+            pk.w = *reinterpret_cast<unsigned int *>(&p3);
+            *(reinterpret_cast<uint4 *>(out + off) + c) = pk;
+        }
+        __syncwarp();      // both tiles are reused by the warp's next 16 rows
+    }
+}
+
 // dst += src, elementwise over [B][rows_per_batch * 64]
 template <typename T>
 __global__ void __launch_bounds__(256) k_residual(T *dst, const T *src, long long n_per_batch, long long bstride, int B) {
@@ -117,6 +204,11 @@ cudaError_t launch_glue(int dtype, bool transpose, const void *a, const void *b,
     if (dtype == SSD_DTYPE_F32) {
         if (transpose) k_glue<float, true><<<blocks, 128, 0, st>>>((const float *)a, (const float *)b, W, (float *)out, rows_per_batch, bstride, B);
         else k_glue<float, false><<<blocks, 128, 0, st>>>((const float *)a, (const float *)b, W, (float *)out, rows_per_batch, bstride, B);
+    } else if (rows_per_batch % 16 == 0) {
+        const long long tiles = total / 16;
+        const unsigned mblocks = (unsigned)((tiles + 3) / 4 < 148 * 8 ? (tiles + 3) / 4 : 148 * 8);
+        if (transpose) k_glue_bf16_mma<true><<<mblocks, 128, 0, st>>>((const __nv_bfloat16 *)a, (const __nv_bfloat16 *)b, W, (__nv_bfloat16 *)out, rows_per_batch, bstride, B);
+        else k_glue_bf16_mma<false><<<mblocks, 128, 0, st>>>((const __nv_bfloat16 *)a, (const __nv_bfloat16 *)b, W, (__nv_bfloat16 *)out, rows_per_batch, bstride, B);
     } else {
         if (transpose) k_glue<__nv_bfloat16, true><<<blocks, 128, 0, st>>>((const __nv_bfloat16 *)a, (const __nv_bfloat16 *)b, W, (__nv_bfloat16 *)out, rows_per_batch, bstride, B);
         else k_glue<__nv_bfloat16, false><<<blocks, 128, 0, st>>>((const __nv_bfloat16 *)a, (const __nv_bfloat16 *)b, W, (__nv_bfloat16 *)out, rows_per_batch, bstride, B);
