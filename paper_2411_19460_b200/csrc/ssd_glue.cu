@@ -104,17 +104,25 @@ __global__ void __launch_bounds__(128) k_glue_bf16_mma(const __nv_bfloat16 *a, c
     __syncthreads();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long ntiles = rows_per_batch * B / 16;
-    for (long long t = (long long)blockIdx.x * 4 + warp; t < ntiles; t += (long long)gridDim.x * 4) {
+    auto tile_offset = [&](long long t) {
         const long long row0 = t * 16, bb = row0 / rows_per_batch, rr = row0 % rows_per_batch;
-        const size_t off = (size_t)bb * bstride + (size_t)rr * 64;
-        // 16-byte chunk c of the block (128 of them): row c / 8, columns (c % 8) * 8 ..
-        uint4 va[4], vb[4];
+        return (size_t)bb * bstride + (size_t)rr * 64;
+    };
+    // 16-byte chunk c of a tile's block (128 of them): row c / 8, columns (c % 8) * 8 ..; the next tile's rows are
+    // requested as soon as the current ones have been parked in shared memory
+    uint4 va[4], vb[4];
+    auto fetch = [&](size_t off) {
 #pragma unroll
         for (int q = 0; q < 4; ++q) va[q] = __ldg(reinterpret_cast<const uint4 *>(a + off) + q * 32 + lane);
         if (b) {
 #pragma unroll
             for (int q = 0; q < 4; ++q) vb[q] = __ldg(reinterpret_cast<const uint4 *>(b + off) + q * 32 + lane);
         }
+    };
+    const long long t_first = (long long)blockIdx.x * 4 + warp, t_step = (long long)gridDim.x * 4;
+    if (t_first < ntiles) fetch(tile_offset(t_first));
+    for (long long t = t_first; t < ntiles; t += t_step) {
+        const size_t off = tile_offset(t);
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             uint4 z = va[q];
@@ -127,6 +135,7 @@ __global__ void __launch_bounds__(128) k_glue_bf16_mma(const __nv_bfloat16 *a, c
             const int c = q * 32 + lane;
             *reinterpret_cast<uint4 *>(&zs[warp][(c >> 3) * GL_LD + (c & 7) * 8]) = z;
         }
+        if (t + t_step < ntiles) fetch(tile_offset(t + t_step));
         __syncwarp();
         wmma::fragment<wmma::matrix_a, 16, 16, 16, __nv_bfloat16, wmma::row_major> za[4];
 #pragma unroll
@@ -206,7 +215,7 @@ cudaError_t launch_glue(int dtype, bool transpose, const void *a, const void *b,
         else k_glue<float, false><<<blocks, 128, 0, st>>>((const float *)a, (const float *)b, W, (float *)out, rows_per_batch, bstride, B);
     } else if (rows_per_batch % 16 == 0) {
         const long long tiles = total / 16;
-        const unsigned mblocks = (unsigned)((tiles + 3) / 4 < 148 * 8 ? (tiles + 3) / 4 : 148 * 8);
+        const unsigned mblocks = (unsigned)((tiles + 3) / 4 < 148 * 6 ? (tiles + 3) / 4 : 148 * 6);   // six 37 KB CTAs fit an SM: one wave
         if (transpose) k_glue_bf16_mma<true><<<mblocks, 128, 0, st>>>((const __nv_bfloat16 *)a, (const __nv_bfloat16 *)b, W, (__nv_bfloat16 *)out, rows_per_batch, bstride, B);
         else k_glue_bf16_mma<false><<<mblocks, 128, 0, st>>>((const __nv_bfloat16 *)a, (const __nv_bfloat16 *)b, W, (__nv_bfloat16 *)out, rows_per_batch, bstride, B);
     } else {
