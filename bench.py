@@ -505,7 +505,7 @@ def run_stack(args, rep, dev):
         return
     peaks = load_peaks()
     fl, by = step_model(cfg, cfg.seg)
-    glue_bytes = 2 * (3 + 3) * cfg.H * cfg.P              # forward x, y -> x_next; backward g -> dz, dx += dz
+    glue_bytes = 2 * (3 + 2) * cfg.H * cfg.P              # forward x, y -> x_next; backward g -> dz (dx += dz is folded into the dx kernel)
     t_roof = cfg.layers * cfg.L * max(fl / (peaks["bf16_tflops"] * 1e12), (by + glue_bytes) / (peaks["hbm_gbs"] * 1e9))
     value = rep.world * cfg.L / (ms * 1e-3)
     line = {

@@ -56,6 +56,9 @@ enum {
     SSD_FLAG_FORCE_SIMT = 1,       /* bf16 I/O: use the CUDA-core kernels instead of the tensor-core ones */
     SSD_FLAG_ACCUM_PARAM_GRADS = 2,/* ssd_bwd_segmented: dA and dD are added to, not overwritten (a driver that
                                       back-propagates one grid cell at a time sums them over the cells) */
+    SSD_FLAG_SKIP_GRAD = 16,       /* ssd_bwd_segmented: dx += dy, the gradient that a skip connection around the layer
+                                      (next input = f(y + x)) sends straight to x; folded into the dx kernel's output
+                                      (one rounding), instead of a separate read-add-write pass over dx */
     SSD_FLAG_SPLIT_BC = 8,         /* ssd_bwd_segmented, tensor-core path: dB and dC by two kernels that each mask the
                                       score tiles themselves, instead of the one that masks them once for both (a
                                       cross-check; the same values up to the order of the fp32 head sums) */

@@ -539,6 +539,7 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
     fill_params(pl, lo, ws, sp);
     sp.x = x; sp.dt = dt; sp.A = A; sp.Bm = Bm; sp.Cm = Cm; sp.D = D; sp.dy = dy;
     sp.dx = dx; sp.ddt = ddt; sp.dB = dB; sp.dC = dC;
+    sp.dx_skip = (shape->flags & SSD_FLAG_SKIP_GRAD) ? 1.f : 0.f;
     if (pl.use_tc) sp.rho2 = (float *)((char *)ws + lo.rho2);
     SSD_TRY(cudaMemsetAsync(sp.status, 0, 256, st));
     TcMaps maps;

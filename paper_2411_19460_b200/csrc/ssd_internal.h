@@ -46,6 +46,7 @@ struct SegParams {
     int bc_fused;  // 1: the fused dB/dC kernel wrote them: two slots per slice (see ssd_tc_bcf.cu), second parts of rho/psi
     int ndd;          // partial sums of dD per (head, chunk) that the kernels of this path write (<= 16)
     int nsplit_scan;  // head ranges per group in the tensor-core scan kernels (no effect on results)
+    float dx_skip;    // 1 when dx also takes dy (a skip connection around the layer), else 0
     int64_t x_bs, dt_bs, bc_bs;  // batch strides, elements
 
     // caller tensors

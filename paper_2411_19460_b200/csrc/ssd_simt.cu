@@ -505,7 +505,7 @@ __global__ void __launch_bounds__(256) k_masked_product_simt(SegParams p) {
                 stf(yb + (size_t)r * HP + pp, fmaf(Dh, xv, acc[i][j]));
             }
     } else if (MODE == MP_BWD_DX) {
-        const float Dh = __ldg(p.D + h);
+        const float Dh = __ldg(p.D + h) + p.dx_skip;      // D dy, plus dy itself under a skip connection
         T *dxb = (T *)p.dx + (size_t)b * p.x_bs + tok0 * HP + (size_t)h * 64;
         float dsum = 0.f;
 #pragma unroll

@@ -388,6 +388,7 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             __syncwarp();
             if (lane == 0) mbar_arrive(&vempty[buf]);
             const float Dh = __ldg(p.D + h);
+            const float Dx = Dh + (FWD ? 0.f : p.dx_skip);       // dx: D dy, plus dy itself under a skip connection
             mbar_wait(&xfull[xs], xuse & 1, abortp, p.status);
             if (!FWD) mbar_wait(&xrfull, hi & 1, abortp, p.status);
             unsigned char *blockbase = smem + OFF_X + xs * 32768 + ((FWD ? rb * 128 : 0) + q * 32) * 128;
@@ -423,7 +424,7 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                             dd2 = fmaf(xv[e + 1], a2[i + 1], dd2);
                             dsum = fmaf(vv[e], xv[e], dsum);
                             dsum = fmaf(vv[e + 1], xv[e + 1], dsum);
-                            ow[e >> 1] = pack2(fmaf(Dh, vv[e], dtr * u0), fmaf(Dh, vv[e + 1], dtr * u1));
+                            ow[e >> 1] = pack2(fmaf(Dx, vv[e], dtr * u0), fmaf(Dx, vv[e + 1], dtr * u1));
                         }
                     }
                     *reinterpret_cast<uint4 *>(vrow + off) = o;

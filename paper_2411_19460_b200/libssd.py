@@ -15,6 +15,7 @@ SSD_FLAG_FORCE_SIMT = 1
 SSD_FLAG_ACCUM_PARAM_GRADS = 2
 SSD_FLAG_SERIAL = 4
 SSD_FLAG_SPLIT_BC = 8
+SSD_FLAG_SKIP_GRAD = 16
 SSD_OP_FWD, SSD_OP_FWD_SEG, SSD_OP_BWD_SEG = 0, 1, 2
 SSD_OK, SSD_EINVAL, SSD_EUNSUPPORTED, SSD_EALIGN = 0, -1, -2, -3
 SSD_EWORKSPACE, SSD_EDEVICE, SSD_ECUDA, SSD_ETIMEOUT = -4, -5, -6, -7

@@ -10,7 +10,7 @@ back-propagated layer by layer and hands dx down the stack and dh to the segment
 
 Layer j: y_j = SSD_j(x_j), x_{j+1} = W (y_j + x_j).  B, C, dt are shared by the layers; A, D are per layer.
 This module only marshals: every arithmetic step is a libssd call (ssd_fwd, ssd_bwd_segmented with
-one segment per call, ssd_glue_*).  torch allocates the buffers.
+one segment per call and the skip-branch gradient folded in, ssd_glue_*).  torch allocates the buffers.
 """
 import torch
 
@@ -96,7 +96,8 @@ class LayerStack:
             for j, t in enumerate(dh_final):
                 if t is not None:
                     self.dh[j, 0].copy_(t)
-        flags = self.flags | libssd.SSD_FLAG_ACCUM_PARAM_GRADS
+        # dx of a layer = (SSD backward of dz) + dz, the skip branch: the dx kernel adds it itself
+        flags = self.flags | libssd.SSD_FLAG_ACCUM_PARAM_GRADS | libssd.SSD_FLAG_SKIP_GRAD
         for k in range(self.nseg - 1, -1, -1):
             cur = (self.nseg - 1 - k) & 1              # dh[j, cur] enters from the right, dh[j, 1-cur] leaves
             g_in = self._sl(g_top, k)
@@ -110,7 +111,6 @@ class LayerStack:
                 libssd.ssd_bwd_segmented(xs, self._dts[k], self.A[j], self._Bs[k],
                                          self._Cs[k], self.D[j], self._bin[j][k], self.dz, self.dh[j, cur],
                                          chunk=self.chunk, seg=self.seg, flags=flags, out=cell, ws=self.ws_b)
-                libssd.ssd_glue_residual(dx, self.dz)
                 if on_cell is not None:
                     on_cell(j, k, dict(cell, dy=self.dz))
                 g_in = dx

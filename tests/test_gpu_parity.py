@@ -132,3 +132,21 @@ def test_helper_streams_change_no_bit_and_respect_caller_stream(seg):
                                                         inp["h0"], chunk=cfg.chunk, seg=cfg.seg, stream=s)
     s.synchronize()
     assert torch.equal(y, ref["y"]) and torch.equal(h_final, ref["h_final"]) and torch.equal(boundary, ref["boundary"])
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_skip_gradient_flag_adds_dy_to_dx(dtype):
+    """SSD_FLAG_SKIP_GRAD: dx = (plain dx) + dy with one rounding; every other output unchanged."""
+    cfg = small(dtype=dtype, B=2, L=1024, H=8, G=2, seg=512) if dtype == "bf16" else CASES["fp32_q256"]
+    inp = make_inputs(cfg, "cuda")
+    ref = pu.run_gpu(cfg, inp)
+    g = libssd.ssd_bwd_segmented(inp["x"], inp["dt"], inp["A"], inp["Bm"], inp["Cm"], inp["D"], ref["boundary"],
+                                 inp["dy"], inp["dh_final"], chunk=cfg.chunk, seg=cfg.seg, flags=libssd.SSD_FLAG_SKIP_GRAD)
+    torch.cuda.synchronize()
+    want = ref["dx"].float() + inp["dy"].float()
+    err = (g["dx"].float() - want).abs().max().item() / want.abs().max().item()
+    assert err <= (8e-3 if dtype == "bf16" else 1e-6), err
+    for k, v in g.items():
+        if v is not None and k != "dx":
+            assert torch.equal(v, ref[k]), k
