@@ -176,7 +176,8 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
  * with batch stride x_bstride; only B, L, H, P, dtype and x_bstride of `shape` are read (P must be 64).
  *   ssd_glue_fwd      : x_next = W (y + x)
  *   ssd_glue_bwd      : dz = W^T g_next     (dz is the dy of the layer's SSD backward)
- *   ssd_glue_residual : dx += dz            (the skip branch; call after ssd_bwd_segmented wrote dx)
+ *   ssd_glue_residual : dx += dz            (the skip branch; call after ssd_bwd_segmented wrote dx -- or pass
+ *                                            SSD_FLAG_SKIP_GRAD to ssd_bwd_segmented, which then adds dy itself)
  * Device pointers, enqueued on `stream`, no scratch.  Returns SSD_OK or SSD_EINVAL / SSD_EUNSUPPORTED /
  * SSD_EALIGN / SSD_ECUDA.
  */
