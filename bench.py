@@ -236,6 +236,9 @@ def run_ours(args):
     if args.heads:
         cfg = cfg.scaled(H=args.heads, name="%s_h%d" % (cfg.name, args.heads))
         CONFIGS[args.config] = cfg
+    if args.len:
+        cfg = cfg.scaled(L=args.len, name="%s_L%d" % (cfg.name, args.len))
+        CONFIGS[args.config] = cfg
     if args.stream_len:
         return run_stream(args, rep, dev)
     if args.conv:
@@ -873,6 +876,8 @@ def main():
     ap.add_argument("--gated-norm", action="store_true", help="time the gated RMS normalisation stage (forward + backward, "
                     "segment by segment) instead of the SSD step")
     ap.add_argument("--heads", type=int, default=0, help="override the head count (32 / 64: the 370M / 1.3B model sizes)")
+    ap.add_argument("--len", type=int, default=0, help="override the sequence length (a short prefix of the workload, "
+                    "e.g. for a profiler capture of one kernel at the workload's launch geometry)")
     ap.add_argument("--layers", type=int, default=0, help="config 3: number of layers (default 64)")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="time plain stream launches instead of the replay of the step captured in a CUDA graph")
