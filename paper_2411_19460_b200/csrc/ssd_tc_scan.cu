@@ -38,7 +38,10 @@ using namespace sm100;
 
 namespace {
 
-constexpr int SC_THREADS = 736;           // warp 0 producer, 1 MMA, 2..17 mask, 18 vectors, 19..22 epilogue
+// warp 0 producer, 1 MMA, 2..17 mask, 18 vectors, 19.. epilogue: one warp per TMEM lane quarter for y, two for dx,
+// whose epilogue (three row sums besides the output) set the pace of the kernel with one
+__host__ __device__ constexpr int sc_epilogue_warps(int mode) { return mode == SC_FWD ? 4 : 8; }
+__host__ __device__ constexpr int sc_threads(int mode) { return (19 + sc_epilogue_warps(mode)) * 32; }
 constexpr uint32_t OFF_ROWS = 0;          // 32 KB  [n-half][128 rows][128 B]
 constexpr uint32_t OFF_X = 32768;         // 3 x 32 KB value stages; first the score-columns operand (<= 64 KB)
 constexpr uint32_t OFF_M = 131072;        // 2 x 16 KB ring of masked pieces
@@ -70,10 +73,14 @@ __device__ __forceinline__ void unpack8(const uint4 &q, float *f) {
     }
 }
 
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
 }  // namespace
 
 template <int MODE>
-__global__ void __launch_bounds__(SC_THREADS, 1)
+__global__ void __launch_bounds__(sc_threads(MODE), 1)
 k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
           const __grid_constant__ CUtensorMap tmCol, const __grid_constant__ CUtensorMap tmV,
           const __grid_constant__ CUtensorMap tmSt, const __grid_constant__ CUtensorMap tmOut,
@@ -83,8 +90,10 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
     __shared__ uint64_t bar_ab, bar_s, xfull[3], xempty[3], hfull[2], hempty[2], xrfull, xrempty, mfull[2], mempty[2],
         accfull[2], accempty[2], vfull[2], vempty[2];
     __shared__ uint32_t tmem_base, abort_flag;
+    __shared__ float epx[2][128][2], epd[2][4];    // SC_DX: row sums handed from one epilogue warp of a pair to the other
 
     constexpr bool FWD = (MODE == SC_FWD);
+    constexpr int EPW = sc_epilogue_warps(MODE), NPP = 16 / EPW;   // epilogue warps; 16-column passes per warp
     // 1-D grid; the first half are the long CTAs (the row block with the larger column range), so the
     // tail of the launch is filled with short ones
     const int nc = p.nc, ny = nsplit * p.G;
@@ -118,12 +127,12 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             mbar_init(&mfull[i], 8);           // one arrival per warp (lane 0, after __syncwarp()) of the slot's eight
             mbar_init(&mempty[i], 1);
             mbar_init(&accfull[i], 1);
-            mbar_init(&accempty[i], 4);
+            mbar_init(&accempty[i], EPW);
             mbar_init(&vfull[i], 1);
-            mbar_init(&vempty[i], 16 + 4);
+            mbar_init(&vempty[i], 16 + EPW);
         }
         mbar_init(&xrfull, 1);
-        mbar_init(&xrempty, 4);
+        mbar_init(&xrempty, EPW);
         abort_flag = 0;
         fence_barrier_init();
     }
@@ -369,11 +378,13 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             if (lane == 0) mbar_arrive(&vempty[hi & 1]);
         }
     } else if (warp >= 19) {
-        // ------------------------------------------------------------ epilogue warps (one per TMEM lane quarter)
+        // ------------------------------------------------------------ epilogue warps (one or two per TMEM lane quarter)
         // x (and dy) come from the tiles TMA already brought to shared memory; the output overwrites the
         // rows just read, in place (the MMAs of the head are done with the stage), and leaves by one TMA
-        // store per warp (32 rows x 64 columns), after which the warp releases the stage.
+        // store per lane quarter (32 rows x 64 columns), after which the stage is released.  With two warps per
+        // quarter each takes 32 of the 64 output columns.
         const int q = warp & 3;
+        const int ech = (warp - 19) >> 2;          // which 32 output columns
         const int rl = q * 32 + lane;              // row inside the 128-row block
         const int r = rb * 128 + rl;               // row inside the chunk
         const uint32_t tlane = (uint32_t)(q * 32) << 16;
@@ -398,10 +409,13 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
             tc_fence_after_sync();
             float dd = 0.f, dd2 = 0.f, dsum = 0.f;
 #pragma unroll
-            for (int pass = 0; pass < 4; ++pass) {
+            for (int pp = 0; pp < NPP; ++pp) {
+                const int pass = ech * NPP + pp;
                 float a1[16], a2[16];
-                tmem_ld16(tm + tlane + 256 + buf * 128 + pass * 16, a1);
-                tmem_ld16(tm + tlane + 320 + buf * 128 + pass * 16, a2);
+                tmem_ld16_nowait(tm + tlane + 256 + buf * 128 + pass * 16, a1);
+                tmem_ld16_nowait(tm + tlane + 320 + buf * 128 + pass * 16, a2);
+                tmem_ld_wait16(a1);
+                tmem_ld_wait16(a2);
 #pragma unroll
                 for (int c2 = 0; c2 < 2; ++c2) {
                     const uint32_t off = (uint32_t)((2 * pass + c2) ^ (rl & 7)) << 4;
@@ -430,26 +444,43 @@ k_scan_tc(SegParams p, int nsplit, const __grid_constant__ CUtensorMap tmRow,
                     *reinterpret_cast<uint4 *>(vrow + off) = o;
                 }
             }
+            if (!FWD) {
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, off);
+                if (EPW == 8 && ech == 1) {      // the upper columns' sums go to the other warp of the quarter (buffers alternate by head)
+                    epx[buf][rl][0] = dd;
+                    epx[buf][rl][1] = dd2;
+                    if (lane == 0) epd[buf][q] = dsum;
+                }
+            }
             tc_fence_before_sync();
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(&accempty[buf]);
                 if (!FWD) mbar_arrive(&xrempty);
-                tma_store_3d(&tmOut, blockbase, h * 64, tok0 + rb * 128 + q * 32, b);
-                tma_store_commit();
-                tma_store_wait_read();              // the store has read the block: the stage may be refilled
-                mbar_arrive(&xempty[xs]);
             }
-            if (!FWD) {
-                const size_t vo = ((((size_t)b * p.H + h) * p.ncs + c) << 8) + r;
-                p.ddt_dir[vo] = dd;
-                // psi2_s = B_s . (inter-chunk part of this head's dB_s) = dt_s e^{cs_last-cs_s} x_s . (Gout B_s)
-                p.psi2[vo] = dtr * offs * dd2;
-                // dy.x of this warp's 32 rows: one of 8 partials per (head, chunk), summed later in a fixed order
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, off);
-                if (lane == 0) p.dDp[((((size_t)b * p.H + h) * p.nct + p.c0 + c) << 4) + rb * 4 + q] = dsum;
+            if (EPW == 8) named_bar_sync(1 + q, 64);          // both halves of the quarter's 32 x 64 block are in place
+            if (ech == 0) {
+                if (lane == 0) {
+                    tma_store_3d(&tmOut, blockbase, h * 64, tok0 + rb * 128 + q * 32, b);
+                    tma_store_commit();
+                    tma_store_wait_read();              // the store has read the block: the stage may be refilled
+                    mbar_arrive(&xempty[xs]);
+                }
+                if (!FWD) {
+                    if (EPW == 8) {
+                        dd += epx[buf][rl][0];
+                        dd2 += epx[buf][rl][1];
+                        dsum += epd[buf][q];
+                    }
+                    const size_t vo = ((((size_t)b * p.H + h) * p.ncs + c) << 8) + r;
+                    p.ddt_dir[vo] = dd;
+                    // psi2_s = B_s . (inter-chunk part of this head's dB_s) = dt_s e^{cs_last-cs_s} x_s . (Gout B_s)
+                    p.psi2[vo] = dtr * offs * dd2;
+                    // dy.x of this quarter's 32 rows: one of 8 partials per (head, chunk), summed later in a fixed order
+                    if (lane == 0) p.dDp[((((size_t)b * p.H + h) * p.nct + p.c0 + c) << 4) + rb * 4 + q] = dsum;
+                }
             }
         }
         if (lane == 0) tma_store_wait_all();
@@ -470,11 +501,11 @@ cudaError_t launch_scan_tc(const SegParams &p, const TcMaps &m, int mode, cudaSt
     if (mode == SC_FWD) {
         e = cudaFuncSetAttribute(k_scan_tc<SC_FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SC_SMEM);
         if (e != cudaSuccess) return e;
-        return launch_pdl(k_scan_tc<SC_FWD>, grid, dim3(SC_THREADS), (size_t)SC_SMEM, st, p, nsplit, m.Cm, m.Bm, m.x, m.Hbf, m.y, m.x);
+        return launch_pdl(k_scan_tc<SC_FWD>, grid, dim3(sc_threads(SC_FWD)), (size_t)SC_SMEM, st, p, nsplit, m.Cm, m.Bm, m.x, m.Hbf, m.y, m.x);
     } else {
         e = cudaFuncSetAttribute(k_scan_tc<SC_DX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SC_SMEM);
         if (e != cudaSuccess) return e;
-        return launch_pdl(k_scan_tc<SC_DX>, grid, dim3(SC_THREADS), (size_t)SC_SMEM, st, p, nsplit, m.Bm, m.Cm, m.dy, m.Gbf, m.dx, m.x);
+        return launch_pdl(k_scan_tc<SC_DX>, grid, dim3(sc_threads(SC_DX)), (size_t)SC_SMEM, st, p, nsplit, m.Bm, m.Cm, m.dy, m.Gbf, m.dx, m.x);
     }
     return cudaGetLastError();
 }
