@@ -103,7 +103,11 @@ typedef struct ssd_shape {
 
 /* Bytes of scratch `ws` that `op` needs for this shape (0 on an invalid shape).  Grows with
  * seg/chunk (the per-segment chunk states: the "grid cell" term of Eq. 4), not with L, apart from
- * 8 bytes per (batch, head, chunk) of dA/dD partial sums in the backward. */
+ * 8 bytes per (batch, head, chunk) of dA/dD partial sums in the backward.  With four segments or more
+ * the tensor-core path keeps second copies of what neighbouring segments' kernels touch at the same
+ * time, unless shape->flags has SSD_FLAG_SERIAL: size the buffer with the flags the call will use.
+ * Whether the tensor-core path is taken depends on the CUDA driver being present (it resolves the
+ * tensor-map encoder at run time), so the answer is the one for the machine the query runs on. */
 size_t ssd_workspace_bytes(const ssd_shape_t *shape, int op);
 
 /* Bytes of the `boundary` buffer: B * ceil(L/seg) * H * P * N * 4 (the S_ckpt of Algorithm 1). */
@@ -131,9 +135,10 @@ int ssd_fwd(const ssd_shape_t *shape, const void *x, const float *dt, const floa
  * The call itself performs no allocation of any kind; inputs and outputs are still the caller's.
  *
  * Same arguments and results as ssd_fwd (bit-identical outputs), minus ws / ws_bytes.
- *  - Returns SSD_ETOOLARGE, with nothing enqueued, when ssd_workspace_bytes(shape, SSD_OP_FWD)
- *    exceeds SSD_STATIC_WS_BYTES: shrink `seg` (scratch grows with seg/chunk, not with L) or use
- *    ssd_fwd with your own buffer.
+ *  - Every kernel runs in order on `stream`, so the scratch is laid out as for SSD_FLAG_SERIAL (no
+ *    second copies).  Returns SSD_ETOOLARGE, with nothing enqueued, when that layout --
+ *    ssd_workspace_bytes(shape with SSD_FLAG_SERIAL set, SSD_OP_FWD) -- exceeds SSD_STATIC_WS_BYTES:
+ *    shrink `seg` (scratch grows with seg/chunk, not with L) or use ssd_fwd with your own buffer.
  *  - The first call on each device looks up the device address of the built-in array (with that
  *    device current).  Make that first call outside any CUDA stream capture.
  *  - All calls on one device share the one array, and it keeps whatever the previous call left

@@ -62,7 +62,7 @@ static const int kMinSegmentsForTwins = 4;
 
 struct Plan {
     int B, L, H, P, N, G, Q, seg, nseg, ncs, nct, hpg, nsl, nslf, dtype;
-    bool use_tc;
+    bool use_tc, serial;
     int64_t x_bs, dt_bs, bc_bs;
     size_t esz;
 };
@@ -156,6 +156,7 @@ static int make_plan(const ssd_shape_t *s, Plan &pl) {
     if (((size_t)s->H * s->P * pl.esz) % 16 || ((size_t)s->G * s->N * pl.esz) % 16 ||
         ((size_t)pl.x_bs * pl.esz) % 16 || ((size_t)pl.bc_bs * pl.esz) % 16)
         return SSD_EALIGN;
+    pl.serial = (s->flags & SSD_FLAG_SERIAL) != 0;
     pl.use_tc = tc_supported(s->dtype, s->flags, s->P, s->N, s->chunk, pl.hpg);
     // Partial slices of the dB/dC head sums.  CUDA-core kernels: one head per slice.  Tensor-core
     // kernels: one slice per CTA head range, chosen for a reference launch of 16 chunks (at least 4
@@ -171,7 +172,9 @@ static int make_plan(const ssd_shape_t *s, Plan &pl) {
     return SSD_OK;
 }
 
-static void make_layout(const Plan &pl, int op, Layout &lo) {
+// `twins`: whether the second copies may exist at all (not for callers that keep every kernel in order on one
+// stream: SSD_FLAG_SERIAL and the built-in scratch of ssd_fwd_static_ws).
+static void make_layout(const Plan &pl, int op, Layout &lo, bool twins) {
     const size_t PN = (size_t)pl.P * pl.N, BH = (size_t)pl.B * pl.H;
     const size_t vec = BH * pl.ncs * pl.Q * sizeof(float);
     const size_t st = (size_t)pl.B * (pl.ncs + 1) * pl.H * PN;
@@ -185,7 +188,7 @@ static void make_layout(const Plan &pl, int op, Layout &lo) {
     lo.Hst = take(st * sizeof(float));
     lo.Hbf = take(pl.use_tc ? st * 2 : 0);
     lo.hcarry = take(BH * PN * sizeof(float));
-    const bool twin = pl.use_tc && pl.nseg >= kMinSegmentsForTwins;
+    const bool twin = twins && pl.use_tc && pl.nseg >= kMinSegmentsForTwins;
     lo.cs_b = take(twin ? vec : 0);
     lo.dtT_b = take(twin ? vec : 0);
     lo.Hbf_b = take(twin ? st * 2 : 0);
@@ -368,7 +371,7 @@ static int forward_impl(const ssd_shape_t *shape, const void *x, const float *dt
         (boundary && misaligned(boundary)))
         return SSD_EALIGN;
     Layout lo;
-    make_layout(pl, need_boundary ? SSD_OP_FWD_SEG : SSD_OP_FWD, lo);
+    make_layout(pl, need_boundary ? SSD_OP_FWD_SEG : SSD_OP_FWD, lo, may_use_helper_stream && !pl.serial);
     if (((uintptr_t)ws & 255u) || ws_bytes < lo.total) return SSD_EWORKSPACE;
     rc = check_device();
     if (rc) return rc;
@@ -381,7 +384,7 @@ static int forward_impl(const ssd_shape_t *shape, const void *x, const float *dt
     TcMaps maps;
     if (pl.use_tc && !tc_make_maps(sp, maps)) return SSD_ECUDA;
     const long long PN = (long long)pl.P * pl.N;
-    if (pl.use_tc && pl.nseg >= kMinSegmentsForTwins && may_use_helper_stream && !(shape->flags & SSD_FLAG_SERIAL) && !g_prof_on) {
+    if (pl.use_tc && pl.nseg >= kMinSegmentsForTwins && may_use_helper_stream && !pl.serial && !g_prof_on) {
         // Algorithm 1 with the state chain one segment ahead: chunk states and state pass of segment k run on a
         // helper stream while the caller's stream still computes y of segment k-1, whose last, partly idle wave
         // they fill.  What both touch (cumulative sums, dt per chunk, bf16 chunk states) exists twice and
@@ -470,7 +473,7 @@ size_t ssd_workspace_bytes(const ssd_shape_t *shape, int op) {
     if (make_plan(shape, pl)) return 0;
     if (op != SSD_OP_FWD && op != SSD_OP_FWD_SEG && op != SSD_OP_BWD_SEG) return 0;
     Layout lo;
-    make_layout(pl, op, lo);
+    make_layout(pl, op, lo, !pl.serial);
     return lo.total;
 }
 
@@ -493,7 +496,7 @@ int ssd_fwd_static_ws(const ssd_shape_t *shape, const void *x, const float *dt, 
     int rc = make_plan(shape, pl);
     if (rc) return rc;
     Layout lo;
-    make_layout(pl, SSD_OP_FWD, lo);
+    make_layout(pl, SSD_OP_FWD, lo, false);      // in order on one stream: no second copies
     if (lo.total > (size_t)SSD_STATIC_WS_BYTES) return SSD_ETOOLARGE;
     if (!x || !dt || !A || !Bm || !Cm || !D || !y) return SSD_EINVAL;
     rc = check_device();
@@ -529,7 +532,7 @@ int ssd_bwd_segmented(const ssd_shape_t *shape, const void *x, const float *dt, 
         misaligned(dD) || (dh0 && misaligned(dh0)))
         return SSD_EALIGN;
     Layout lo;
-    make_layout(pl, SSD_OP_BWD_SEG, lo);
+    make_layout(pl, SSD_OP_BWD_SEG, lo, !pl.serial);
     if (((uintptr_t)ws & 255u) || ws_bytes < lo.total) return SSD_EWORKSPACE;
     rc = check_device();
     if (rc) return rc;

@@ -17,6 +17,21 @@ def relerr(gpu, ref):
     return float(np.max(np.abs(g - ref))) / den
 
 
+# Outputs that belong to one head each, with the axis that indexes the head.  For these the error is also measured
+# head by head, max over heads of max|gpu_h - ref_h| / max(max|ref_h|, HEAD_FLOOR * max|ref|): with stiff decays the
+# heads differ by orders of magnitude, and a wrong result in a small head would vanish in the whole-tensor measure.
+# The floor keeps a head whose reference is (almost) zero from turning rounding noise into a large ratio.
+HEAD_AXIS = {"y": 2, "dx": 2, "ddt": 2, "h_final": 1, "dh0": 1, "boundary": 2}
+HEAD_FLOOR = 0.05
+
+
+def relerr_per_head(gpu, ref, axis):
+    g = gpu.detach().to("cpu", torch.float64).numpy() if isinstance(gpu, torch.Tensor) else np.asarray(gpu)
+    other = tuple(i for i in range(ref.ndim) if i != axis)
+    den = np.maximum(np.max(np.abs(ref), axis=other), HEAD_FLOOR * max(float(np.max(np.abs(ref))), 1e-30))
+    return float(np.max(np.max(np.abs(g - ref), axis=other) / den))
+
+
 def run_gpu(cfg, inp, seg=None, flags=0, want=("fwd", "bwd")):
     seg = cfg.seg if seg is None else seg
     out = {}
@@ -44,6 +59,7 @@ def check_all(cfg, gpu, ref, keys=None, tol=None):
     tol = TOL[cfg.dtype] if tol is None else tol
     keys = [k for k in ref if k in gpu] if keys is None else keys
     errs = {k: relerr(gpu[k], ref[k]) for k in keys}
+    errs.update({k + "/head": relerr_per_head(gpu[k], ref[k], HEAD_AXIS[k]) for k in keys if k in HEAD_AXIS})
     bad = {k: v for k, v in errs.items() if not (v <= tol)}
     assert not bad, "parity failure (limit %g): %s  | all: %s" % (tol, bad, errs)
     return errs

@@ -39,6 +39,8 @@ def _sampled_head_parity(cfg, heads):
     errs = {}
     for k in PER_HEAD:
         errs[k] = pu.relerr(_slice_heads(k, gpu[k], heads), ref[k])
+        if k in pu.HEAD_AXIS:
+            errs[k + "/head"] = pu.relerr_per_head(_slice_heads(k, gpu[k], heads), ref[k], pu.HEAD_AXIS[k])
     bad = {k: v for k, v in errs.items() if not (v <= pu.TOL[cfg.dtype])}
     assert not bad, "parity failure at full size: %s | all %s" % (bad, errs)
     return errs
@@ -46,6 +48,15 @@ def _sampled_head_parity(cfg, heads):
 
 def test_config2_full_size_sampled_heads():
     print(_sampled_head_parity(CONFIGS[2], heads=[0, 37, 79]))
+
+
+def test_config2_launch_geometry_all_outputs_on_a_prefix():
+    """Config 2's per-launch geometry (80 heads in one group, 4096-token segments, default path) on its first
+    16384 tokens: EVERY output against the oracle, dB and dC included -- the sums over 80 heads that the fused
+    kernel forms in three head ranges and rounds once."""
+    cfg = CONFIGS[2].scaled(L=16384)
+    errs = pu.full_parity(cfg)
+    print(errs)
 
 
 def test_config1_full_size_all_outputs():

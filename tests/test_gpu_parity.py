@@ -55,6 +55,25 @@ def test_parity_two_kernel_dB_dC_path(name):
     pu.full_parity(cfg, flags=libssd.SSD_FLAG_SPLIT_BC)
 
 
+@pytest.mark.parametrize("name", ["bf16_ragged_g2_b2", "bf16_stiff", "bf16_h64_g8"])
+def test_tensor_core_path_against_cuda_core_path(name):
+    """The two GPU paths on the same bf16 inputs, at half the oracle tolerance: both round their outputs to bf16
+    (or sum bf16 products in fp32), so they differ by a rounding step at most, wherever a head is large or small."""
+    cfg = CASES[name]
+    inp = make_inputs(cfg, "cuda")
+    tc = pu.run_gpu(cfg, inp, flags=0)
+    cc = pu.run_gpu(cfg, inp, flags=SIMT)
+    errs = {}
+    for k in ("y", "h_final", "dx", "ddt", "dA", "dB", "dC", "dD", "dh0"):
+        ref = cc[k].detach().to("cpu", torch.float64).numpy()
+        errs[k] = pu.relerr(tc[k], ref)
+        if k in pu.HEAD_AXIS:
+            errs[k + "/head"] = pu.relerr_per_head(tc[k], ref, pu.HEAD_AXIS[k])
+    bad = {k: v for k, v in errs.items() if not (v <= 1e-2)}
+    assert not bad, "paths disagree (limit 1e-2): %s | all %s" % (bad, errs)
+    print(name, errs)
+
+
 @pytest.mark.parametrize("flags", [SIMT, 0, libssd.SSD_FLAG_SPLIT_BC])
 @pytest.mark.parametrize("name", ["cfg0_fp32", "bf16_ragged_g2_b2", "bf16_stiff"])
 def test_segmented_backward_bit_exact_vs_unsegmented(name, flags):

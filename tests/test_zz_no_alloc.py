@@ -46,3 +46,16 @@ def test_static_scratch_forward_matches_ssd_fwd_on_two_calls_in_a_row():
         assert relerr(y, ry) <= tol, (seed, relerr(y, ry))
         assert relerr(hf, rh) <= tol, (seed, relerr(hf, rh))
         assert torch.isfinite(y.float()).all() and torch.isfinite(hf).all()
+        # the header promises more than the tolerance: the same kernels on the same inputs, so the same bits
+        assert torch.equal(y, y_ref) and torch.equal(hf, h_ref), seed
+
+
+def test_static_scratch_is_sized_without_the_second_copies():
+    # four segments or more: ssd_fwd's default layout doubles some regions for its helper streams, the in-order
+    # layout of the built-in scratch does not, so a shape can fit the latter and not the former
+    ssd_build.build()
+    L = libssd.lib()
+    mk = lambda flags: libssd.SSDShape(1, 8192, 8, 64, 128, 1, 256, 1024, libssd.SSD_DTYPE_BF16, flags, 0, 0, 0)
+    serial = libssd.workspace_bytes(mk(libssd.SSD_FLAG_SERIAL), libssd.SSD_OP_FWD)
+    default = libssd.workspace_bytes(mk(0), libssd.SSD_OP_FWD)
+    assert 0 < serial <= default
