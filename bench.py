@@ -476,6 +476,8 @@ def run_stack(args, rep, dev):
     sp = make_stack_params(cfg, dev)
     st = LayerStack(inp["x"], inp["dt"], inp["Bm"], inp["Cm"], sp["A"], sp["D"], sp["W"], chunk=cfg.chunk, seg=cfg.seg,
                     layer_interval=args.layer_interval, flags=(libssd.SSD_FLAG_SERIAL if args.serial else 0))
+    for j in range(cfg.layers):          # every layer starts from its own N(0, h0_std^2) state, as the workload says
+        st.set_h0(j, sp["h0"][j])
     out = dict(dx0=torch.empty_like(inp["x"]), dA=torch.zeros(cfg.layers, cfg.H, device=dev),
                dD=torch.zeros(cfg.layers, cfg.H, device=dev))
     stream = torch.cuda.current_stream()

@@ -124,16 +124,18 @@ def make_stack_params(cfg: SSDConfig, device="cpu", scale=None):
     W = scale * Q0 with Q0 the orthogonal factor of a seeded Gaussian P x P matrix, rounded to bf16
     so that both sides use the same numbers; `scale` defaults to 0.5, which keeps the RMS of the layer
     inputs of order one over 64 layers for D ~ N(0,1) (y + x has about (1 + D_h^2)^(1/2) times the RMS
-    of x).  B, C and dt are shared by all layers (those of make_inputs)."""
+    of x).  B, C and dt are shared by all layers (those of make_inputs).  Every layer has its own initial
+    state h0 ~ N(0, h0_std^2), as the single-layer workloads do."""
     dev = torch.device(device)
     g = torch.Generator(device="cpu")
     g.manual_seed(cfg.seed + 7919)
     q0, _ = torch.linalg.qr(torch.randn(cfg.P, cfg.P, generator=g, dtype=torch.float64))
     W = ((0.5 if scale is None else scale) * q0).to(torch.bfloat16).to(torch.float32).to(dev)
-    A, D = [], []
+    A, D, h0 = [], [], []
     for layer in range(cfg.layers):
         gl = torch.Generator(device="cpu")
         gl.manual_seed(cfg.seed + 1 + layer)
         A.append((-torch.exp(torch.rand(cfg.H, generator=gl) * math.log(cfg.a_max))).to(dev))
         D.append(torch.randn(cfg.H, generator=gl).to(dev))
-    return dict(W=W.contiguous(), A=A, D=D)
+        h0.append((torch.randn(cfg.B, cfg.H, cfg.P, cfg.N, generator=gl) * cfg.h0_std).to(dev))
+    return dict(W=W.contiguous(), A=A, D=D, h0=h0)

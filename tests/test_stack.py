@@ -36,20 +36,19 @@ def test_stack_parameters_are_seeded_and_bf16_representable():
     assert not torch.equal(a["A"][0], a["A"][1])
 
 
-@pytest.mark.gpu
-def test_stack_matches_oracle_layer_by_layer():
+def _stack_against_oracle(cfg):
+    """Algorithms 1 and 2 over `cfg.layers` layers, every layer compared with the oracle teacher-forced: the oracle's
+    layer j gets the layer input x_j (and in the backward the output gradient) that the GPU path stored.  Returns the
+    worst per-tensor errors and the end-to-end drift: the stack output against the oracle run freely in fp64 from
+    x_0, where the bf16 rounding of every layer input compounds."""
     from paper_2411_19460_b200.stack import LayerStack
     from tests.parity_util import TOL, relerr
 
-    cfg = CONFIGS[3].scaled(L=1024, H=4, seg=512, layers=3, dh_std=0.0)
     tol = TOL[cfg.dtype]
     inp = make_inputs(cfg, "cuda")
     sp = make_stack_params(cfg, "cuda")
     st = LayerStack(inp["x"], inp["dt"], inp["Bm"], inp["Cm"], sp["A"], sp["D"], sp["W"], chunk=cfg.chunk, seg=cfg.seg)
-    # seeded: the case must not vary from run to run (dA of four heads over 1 024 tokens is a heavily cancelled sum,
-    # so its relative error swings with how small the sum happens to be: 3e-4 to 6e-3 over the first five seeds)
-    gen = torch.Generator(device="cuda").manual_seed(cfg.seed + 1)
-    h0 = [torch.randn(cfg.B, cfg.H, cfg.P, cfg.N, device="cuda", generator=gen) * 0.1 for _ in range(cfg.layers)]
+    h0 = sp["h0"]
     for j in range(cfg.layers):
         st.set_h0(j, h0[j])
     st.forward()
@@ -57,12 +56,22 @@ def test_stack_matches_oracle_layer_by_layer():
 
     f64 = lambda t: t.detach().double().cpu().numpy()
     dt, Bm, Cm, W = f64(inp["dt"]), f64(inp["Bm"]), f64(inp["Cm"]), f64(sp["W"])
+    worst = {}
+
+    def note(name, err, j):
+        assert err <= tol, (name, j, err)
+        worst[name] = max(worst.get(name, 0.0), err)
+
+    free = f64(st.x[0])                    # the oracle's own layer inputs, never rounded
     for j in range(cfg.layers):
         xj = f64(st.x[j])
         y, hf, bd = orc.ssd_fwd(xj, dt, f64(sp["A"][j]), Bm, Cm, f64(sp["D"][j]), f64(h0[j]), seg=cfg.seg)
-        assert relerr(st.x[j + 1], orc.glue_fwd(xj, y, W)) <= tol, j
-        assert relerr(st.bnd[j, st.nseg], hf) <= tol, j
-        assert relerr(st.bnd[j, 1], bd[:, 1]) <= tol, j
+        note("x_next", relerr(st.x[j + 1], orc.glue_fwd(xj, y, W)), j)
+        note("h_final", relerr(st.bnd[j, st.nseg], hf), j)
+        note("boundary", relerr(st.bnd[j, 1], bd[:, 1]), j)
+        yf, _, _ = orc.ssd_fwd(free, dt, f64(sp["A"][j]), Bm, Cm, f64(sp["D"][j]), f64(h0[j]), seg=cfg.seg)
+        free = orc.glue_fwd(free, yf, W)
+    drift = relerr(st.x[cfg.layers], free)
 
     # backward, collecting the per-cell outputs into per-layer tensors
     keep = {k: [torch.zeros_like(inp[src]) for _ in range(cfg.layers)]
@@ -79,15 +88,31 @@ def test_stack_matches_oracle_layer_by_layer():
     for j in range(cfg.layers - 1, -1, -1):
         g_next = f64(g_top) if j == cfg.layers - 1 else f64(keep["dx"][j + 1])
         dz = orc.glue_bwd(g_next, W)
-        assert relerr(keep["dy"][j], dz) <= tol, j
+        note("dz", relerr(keep["dy"][j], dz), j)
         ref = orc.ssd_bwd(f64(st.x[j]), dt, f64(sp["A"][j]), Bm, Cm, f64(sp["D"][j]), f64(h0[j]), f64(keep["dy"][j]), None)
-        errs = dict(dx=relerr(keep["dx"][j], ref["dx"] + f64(keep["dy"][j])), ddt=relerr(keep["ddt"][j], ref["ddt"]),
-                    dB=relerr(keep["dB"][j], ref["dB"]), dC=relerr(keep["dC"][j], ref["dC"]),
-                    dA=relerr(out["dA"][j], ref["dA"]), dD=relerr(out["dD"][j], ref["dD"]),
-                    dh0=relerr(out["dh0"][j], ref["dh0"]))
-        bad = {k: v for k, v in errs.items() if not (v <= tol)}
-        assert not bad, (j, bad, errs)
+        note("dx", relerr(keep["dx"][j], ref["dx"] + f64(keep["dy"][j])), j)
+        for name in ("ddt", "dB", "dC"):
+            note(name, relerr(keep[name][j], ref[name]), j)
+        for name in ("dA", "dD", "dh0"):
+            note(name, relerr(out[name][j], ref[name]), j)
     assert torch.equal(out["dx0"], keep["dx"][0])
+    return worst, drift
+
+
+@pytest.mark.gpu
+def test_stack_matches_oracle_layer_by_layer():
+    # small and seeded: dA of four heads over 1 024 tokens is a heavily cancelled sum, so its relative error swings
+    # with how small the sum happens to be (3e-4 to 6e-3 over a handful of seeds)
+    worst, drift = _stack_against_oracle(CONFIGS[3].scaled(L=1024, H=4, seg=512, layers=3, dh_std=0.0))
+    print("worst per-layer errors", worst, "end-to-end drift of the stack output", drift)
+
+
+@pytest.mark.gpu
+def test_stack_at_config3_dimensions():
+    """The stacked workload's own dimensions (80 heads, 4096-token segments) over 8 layers and two segments."""
+    worst, drift = _stack_against_oracle(CONFIGS[3].scaled(L=8192, layers=8, dh_std=0.0))
+    print("worst per-layer errors", worst, "end-to-end drift of the stack output over 8 layers", drift)
+    assert drift <= 5e-2, drift
 
 
 @pytest.mark.gpu
@@ -102,10 +127,7 @@ def test_layer_interval_changes_no_bit(interval):
     cfg = CONFIGS[3].scaled(L=1024, H=4, seg=256, layers=4, dh_std=0.0)
     inp = make_inputs(cfg, "cuda")
     sp = make_stack_params(cfg, "cuda")
-    # seeded: the case must not vary from run to run (dA of four heads over 1 024 tokens is a heavily cancelled sum,
-    # so its relative error swings with how small the sum happens to be: 3e-4 to 6e-3 over the first five seeds)
-    gen = torch.Generator(device="cuda").manual_seed(cfg.seed + 1)
-    h0 = [torch.randn(cfg.B, cfg.H, cfg.P, cfg.N, device="cuda", generator=gen) * 0.1 for _ in range(cfg.layers)]
+    h0 = sp["h0"]
 
     def run(l):
         st = LayerStack(inp["x"], inp["dt"], inp["Bm"], inp["Cm"], sp["A"], sp["D"], sp["W"], chunk=cfg.chunk,
