@@ -31,6 +31,10 @@ import torch  # noqa: E402
 from paper_2411_19460_b200.inputs import CONFIGS, make_inputs, to_f64_numpy  # noqa: E402
 
 METRIC = "ssd_fwd_bwd_segmented_tokens_per_s"
+# With no --config the line is that of the largest single-layer workload that fits one GPU (the million-token one),
+# and the 2.7B-dimension layer at 131072 tokens and the small fp32 case ride along under "also", device-timed.
+HEADLINE_CONFIG = 4
+ALSO_CONFIGS = (2, 0)
 UNIT = "tokens/s"
 
 
@@ -232,6 +236,12 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     rep = Replicas(backend="nccl", device=dev)
     rank, world = rep.rank, rep.world
+    if args.gpus != world:
+        raise SystemExit("bench.py: --gpus %d but %d rank(s) were launched (WORLD_SIZE); start it with "
+                         "python -m torch.distributed.run --nproc-per-node %d" % (args.gpus, world, args.gpus))
+    headline = args.config is None
+    if headline:
+        args.config = HEADLINE_CONFIG
     cfg = CONFIGS[args.config]
     if args.heads:
         cfg = cfg.scaled(H=args.heads, name="%s_h%d" % (cfg.name, args.heads))
@@ -247,6 +257,30 @@ def run_ours(args):
         return run_gated_norm(args, rep, dev)
     if cfg.layers != 1:
         return run_stack(args, rep, dev)
+    line = measure_layer(args, rep, dev, cfg, full=True)
+    if headline:
+        # the other single-layer workloads from the same run, device-timed only, so that rounds stay comparable
+        also = {}
+        for ci in ALSO_CONFIGS:
+            torch.cuda.empty_cache()
+            sub = measure_layer(args, rep, dev, CONFIGS[ci], full=False)
+            if sub is not None:
+                also[sub["config"]["workload"]] = {k: sub[k] for k in ("value", "unit", "ms_per_step", "dtype",
+                                                                         "config", "step_roofline", "gpu_launches")}
+        if line is not None:
+            line["also"] = also
+    if line is not None:
+        print(json.dumps(line))
+    rep.close()
+
+
+def measure_layer(args, rep, dev, cfg, full=True):
+    """One single-layer workload: the device-resident timing of the step and its roofline; with `full` also the
+    per-kernel-kind table, the end-to-end leg through host buffers and the CPU baseline.  Returns the JSON line as a
+    dict on rank 0, None elsewhere."""
+    from paper_2411_19460_b200 import libssd
+
+    rank, world = rep.rank, rep.world
     seg = args.seg or cfg.seg
     flags = (libssd.SSD_FLAG_FORCE_SIMT if args.simt else 0) | (libssd.SSD_FLAG_SERIAL if args.serial else 0)
     inp = make_inputs(cfg, dev, seed=cfg.seed + rank)
@@ -329,6 +363,32 @@ def run_ours(args):
     ms_per_step = ms_total / args.steps
     value = world * tokens / (ms_per_step * 1e-3)
 
+    fl, by = step_model(cfg, seg)
+    peaks = load_peaks()
+    if cfg.dtype == "bf16":
+        t_roof = max(fl * tokens / (peaks["bf16_tflops"] * 1e12), by * tokens / (peaks["hbm_gbs"] * 1e9))
+        step_roof = dict(flops_per_token=fl, bytes_per_token=by, roofline_ms=t_roof * 1e3,
+                         frac=t_roof * 1e3 / ms_per_step, peaks="bf16 tensor (burst) and HBM copy, " + peaks["source"])
+    else:
+        # fp32 mode runs on the CUDA cores (TF32 cannot hold 1e-4): its flop roof is the plain FFMA rate, measured here
+        ffma = measure_ffma_tflops(dev)
+        t_roof = max(fl * tokens / (ffma * 1e12), by * tokens / (peaks["hbm_gbs"] * 1e9))
+        step_roof = dict(flops_per_token=fl, bytes_per_token=by, roofline_ms=t_roof * 1e3,
+                         frac=t_roof * 1e3 / ms_per_step, ffma_tflops=ffma,
+                         peaks="fp32 FFMA rate measured by an fp32 matrix product with TF32 off, and HBM copy",
+                         note="%d tokens: the roofline time is a few microseconds, below the cost of launching the "
+                              "step's kernels; the configuration is launch-bound" % tokens)
+    if not full:
+        del graph
+        if rank != 0:
+            return None
+        return {"value": value, "unit": UNIT, "ms_per_step": ms_per_step,
+                "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
+                "config": {"workload": cfg.name, "B": B, "L": L, "H": H, "P": P, "N": N, "G": cfg.G,
+                           "chunk": cfg.chunk, "seg": seg, "nseg": nseg,
+                           "launch": "cuda graph replay" if args.graph else "stream launches"},
+                "step_roofline": step_roof, "gpu_launches": int(launches)}
+
     # ---- per-kernel-kind timing (CUDA events on the launch stream, separate pass of the same steps)
     prof_steps = min(args.steps, 3)
     libssd.profile(True)
@@ -400,10 +460,8 @@ def run_ours(args):
         del host_in, host_out, dev_in, dsts
 
     if rank != 0:
-        rep.close()
-        return
+        return None
 
-    peaks = load_peaks()
     model = kind_model(cfg)
     # dominant kernel kind = largest share of device time
     total_prof = sum(v[0] for v in prof.values()) or 1.0
@@ -414,7 +472,7 @@ def run_ours(args):
     avg_s = dom_ms * 1e-3 / max(dom_n, 1)
     if bound == "tensor":
         achieved = fl_tok * tok_per_launch / avg_s / 1e12
-        peak = peaks["bf16_tflops_sustained"]
+        peak = peaks["bf16_tflops"]        # a launch timed by itself with CUDA events: the burst figure
         unit = "TFLOP/s"
     else:
         achieved = by_tok * tok_per_launch / avg_s / 1e9
@@ -423,11 +481,8 @@ def run_ours(args):
     roofline = dict(kernel=dom, bound="tensor" if bound == "tensor" else "hbm", achieved=achieved, peak=peak,
                     unit=unit, frac=achieved / peak, traffic=ncu_traffic(dom, tok_per_launch, H),
                     peak_source=peaks["source"],
+                    peak_kind="bf16 matmul, burst" if bound == "tensor" else "HBM copy",
                     avg_launch_us=avg_s * 1e6, launches=dom_n, share_of_device_time=dom_ms / total_prof)
-    fl, by = step_model(cfg, seg)
-    t_roof = max(fl * tokens / (peaks["bf16_tflops"] * 1e12), by * tokens / (peaks["hbm_gbs"] * 1e9))
-    step_roof = dict(flops_per_token=fl, bytes_per_token=by, roofline_ms=t_roof * 1e3,
-                     frac=t_roof * 1e3 / ms_per_step)
     kinds = {k: dict(ms_per_step=v[0] / prof_steps, launches_per_step=v[1] / prof_steps,
                      share=v[0] / total_prof) for k, v in prof.items() if v[1]}
 
@@ -454,8 +509,34 @@ def run_ours(args):
                    "io_bytes": int(io_bytes)},
         "cpu_baseline": cpu,
     }
-    print(json.dumps(line))
-    rep.close()
+    return line
+
+
+_FFMA = {}
+
+
+def measure_ffma_tflops(dev):
+    """fp32 multiply-add rate of the CUDA cores: the best of five 4096^3 fp32 matrix products with TF32 disabled."""
+    if dev in _FFMA:
+        return _FFMA[dev]
+    old = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = False
+    try:
+        n = 4096
+        a = torch.randn(n, n, device=dev)
+        b = torch.randn(n, n, device=dev)
+        best = float("inf")
+        for _ in range(6):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            torch.matmul(a, b)
+            e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        _FFMA[dev] = 2.0 * n ** 3 / (best * 1e-3) / 1e12
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = old
+    return _FFMA[dev]
 
 
 # ----------------------------------------------------------------------------- the stacked configuration
@@ -834,7 +915,7 @@ def run_reference(args):
     if rank != 0:
         return
     from oracle import ssd_oracle as orc
-    cfg = CONFIGS[args.config]
+    cfg = CONFIGS[HEADLINE_CONFIG if args.config is None else args.config]
     seg = args.seg or cfg.seg
     Ls = min(cfg.L, args.ref_tokens)
     small = cfg.scaled(L=Ls)
@@ -865,8 +946,8 @@ def main():
     ap.add_argument("--steps", type=int, default=6)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=2, help="index into the five workloads (default 2: "
-                    "Mamba-2-2.7B-dim layer, L=131072)")
+    ap.add_argument("--config", type=int, default=None, help="index into the five workloads (default: the largest "
+                    "single-layer one, 4, with workloads 2 and 0 reported beside it)")
     ap.add_argument("--seg", type=int, default=0, help="override the segment length")
     ap.add_argument("--simt", action="store_true", help="force the CUDA-core kernels")
     ap.add_argument("--layer-interval", type=int, default=1, help="config 3: keep the input of every l-th layer")
