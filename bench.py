@@ -94,22 +94,25 @@ def load_peaks():
 
 # ----------------------------------------------------------------------------- DRAM traffic from ncu
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the `ncu --set full` capture summarised in
-# profiles/ncu_full_tc_kernels_cfg1.txt (config 1: one launch = 2048 tokens x 24 heads).  A figure is used
-# only while the kernel's source file still has the hash it had when the counters were taken; it is scaled
-# to the timed workload by tokens x heads per launch (the traffic of these kernels grows in proportion).
-NCU_TRAFFIC_CFG1 = {
+# profiles/ncu_full_all_kernels_cfg2_geometry.txt, taken at workload 2's launch geometry (one launch = 4096 tokens x
+# 80 heads).  A figure is used only while the kernel's source file still has the hash it had when the counters were
+# taken; for the other workloads it is scaled by tokens x heads per launch (the traffic of these kernels grows in
+# proportion).
+NCU_TRAFFIC = {
     # kernel kind: (bytes per launch, source file, sha256 of that file at capture time)
-    "bwd_dBdC": (20.55e6, "ssd_tc_bcf.cu", "86cbdbf8df5a575ff65e77851460b110f53d2ae5c0ef203bece4e8ba5cb8f8ee"),
-    "bwd_dx": (17.24e6, "ssd_tc_scan.cu", "f42132f3fb6c9558b719a6414f8431eb3af4548abcafdc0fcd79735a277d7f32"),
-    "chunk_scan_fwd": (10.94e6, "ssd_tc_scan.cu", "f42132f3fb6c9558b719a6414f8431eb3af4548abcafdc0fcd79735a277d7f32"),
-    "chunk_state": (7.04e6, "ssd_tc.cu", "476c275026f7e136b96cec13cc7c617ea7c59d6fc34edbe9bc79467efbc16aee"),
-    "dstate_contrib": (7.04e6, "ssd_tc.cu", "476c275026f7e136b96cec13cc7c617ea7c59d6fc34edbe9bc79467efbc16aee"),
+    "bwd_dBdC": (140.2e6, "ssd_tc_bcf.cu", "86cbdbf8df5a575ff65e77851460b110f53d2ae5c0ef203bece4e8ba5cb8f8ee"),
+    "bwd_dx": (167.1e6, "ssd_tc_scan.cu", "c081e0c5aefb9cc29b488b38c92dc4a08cd5db9093f566821ba30a2f0cc9fb19"),
+    "chunk_scan_fwd": (89.2e6, "ssd_tc_scan.cu", "c081e0c5aefb9cc29b488b38c92dc4a08cd5db9093f566821ba30a2f0cc9fb19"),
+    "chunk_state": (47.9e6, "ssd_tc.cu", "476c275026f7e136b96cec13cc7c617ea7c59d6fc34edbe9bc79467efbc16aee"),
+    "dstate_contrib": (71.2e6, "ssd_tc.cu", "476c275026f7e136b96cec13cc7c617ea7c59d6fc34edbe9bc79467efbc16aee"),
+    "state_pass_fwd": (45.8e6, "ssd_simt.cu", "6b7a2088a97e108638c59fef85a74dbf4964aee0182467b5d29c4818906c881a"),
+    "state_pass_bwd": (68.9e6, "ssd_simt.cu", "6b7a2088a97e108638c59fef85a74dbf4964aee0182467b5d29c4818906c881a"),
 }
-NCU_CFG1_UNITS = 2048 * 24
+NCU_UNITS = 4096 * 80
 
 
 def ncu_traffic(kind, tokens_per_launch, heads):
-    ent = NCU_TRAFFIC_CFG1.get(kind)
+    ent = NCU_TRAFFIC.get(kind)
     if not ent:
         return None
     import hashlib
@@ -121,7 +124,7 @@ def ncu_traffic(kind, tokens_per_launch, heads):
         return None
     if cur != sha:
         return None
-    return nbytes * (tokens_per_launch * heads) / NCU_CFG1_UNITS
+    return nbytes * (tokens_per_launch * heads) / NCU_UNITS
 
 
 # ----------------------------------------------------------------------------- clocks sampling
