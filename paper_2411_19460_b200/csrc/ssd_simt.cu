@@ -35,7 +35,7 @@ __device__ __forceinline__ size_t vec_off(const SegParams &p, int b, int h, int 
     return (((size_t)b * p.H + h) * p.ncs + c) * (size_t)p.Q;
 }
 
-// ------------------------------------------------------------------ a1: chunk cumsum
+// ------------------------------------------------------------------ chunk cumsum
 // One CTA per (chunk, block of 8 heads, batch), one warp per head.  The dt[b, t, h0..h0+7] pieces
 // (32 contiguous bytes per step) are staged through shared memory; a lane owns Q/32 consecutive
 // steps (serial prefix), lane totals are combined with a warp-shuffle scan.
@@ -85,7 +85,7 @@ cudaError_t launch_chunk_cumsum(const SegParams &p, cudaStream_t st) {
     return cudaGetLastError();
 }
 
-// ------------------------------------------------------------------ a2 / a8: chunk state (FFMA)
+// ------------------------------------------------------------------ chunk sums / state-gradient sums (FFMA)
 // mode FWD   : S_c[p,n] = sum_s exp(cs_last - cs_s) dt_s x_s[p] B_s[n]     -> Hst slot c+1
 // mode DSTATE: E_c[p,n] = sum_t exp(cs_t) dy_t[p] C_t[n]                   -> Gst slot c
 template <typename T, int NS>
@@ -155,7 +155,7 @@ cudaError_t launch_chunk_state_simt(const SegParams &p, int dtype, int mode, cud
     return cudaGetLastError();
 }
 
-// ------------------------------------------------------------------ a3 / a4: forward state passing
+// ------------------------------------------------------------------ forward state passing, boundary store / reload
 // H_{c+1} = exp(cs_last,c) H_c + S_c, strictly sequential in c for every (b,h,p,n) element, so the
 // bits do not depend on how the sequence is cut into segments.  Each thread owns one float4.
 // Also stores the segment-entry state into `boundary` (the sequence-axis checkpoint) and hands the
@@ -222,7 +222,7 @@ cudaError_t launch_state_pass_fwd(const SegParams &p, const float *init, long lo
     return launch_pdl(k_state_pass_fwd, grid, dim3(256), 0, st, p, init, init_bs, boundary_out, bnd_bs, final_out, want_bf16 ? 1 : 0);
 }
 
-// ------------------------------------------------------------------ a9: backward state passing
+// ------------------------------------------------------------------ backward state passing
 // Gslot[nc] = gradient arriving from the segment on the right (or dh_final); going left,
 // Gslot[c] = exp(cs_last,c) Gslot[c+1] + E_c.  Gslot[c+1] is Gout of chunk c.  Also emits, per chunk,
 // the partial sums of exp(cs_last,c) <Gout_c, H_in,c> (one per CTA, summed later in a fixed order):
@@ -309,7 +309,7 @@ cudaError_t launch_state_pass_bwd(const SegParams &p, const float *init, float *
     return launch_pdl(k_state_pass_bwd, grid, dim3(256), 0, st, p, init, left_out, want_bf16 ? 1 : 0);
 }
 
-// ------------------------------------------------------------------ a5+a6, a10, a11: masked products (FFMA)
+// ------------------------------------------------------------------ masked products y, dx, dB, dC (FFMA)
 // One generic "score -> decay mask -> times values (+ inter-chunk term)" kernel, 64x64 tiles:
 //   score[r,c] = <Rv_r, Cv_c>            (length KD)
 //   acc[r,:]  += mask(r,c) * score[r,c] * V_c      (width WD)
@@ -598,7 +598,7 @@ cudaError_t launch_masked_product_simt(const SegParams &p, int dtype, int mode, 
                      : launch_mp_mode<__nv_bfloat16, 128>(p, mode, st);
 }
 
-// ------------------------------------------------------------------ a12 + a13: da, ddt, dA partial
+// ------------------------------------------------------------------ da, ddt, dA partial
 // One warp per (b, h, chunk).  With g_t = dLoss/dh_t and h_{t-1} split into their intra-chunk and
 // inter-chunk parts, da_t = exp(a_t) <g_t, h_{t-1}> is the sum of four terms, none of which
 // subtracts large numbers when the decay inside a chunk is strong:
@@ -674,7 +674,7 @@ cudaError_t launch_bwd_finish(const SegParams &p, cudaStream_t st) {
     return launch_pdl(k_bwd_finish, dim3((p.nc + 3) / 4, p.H, p.B), dim3(128), 0, st, p);
 }
 
-// ------------------------------------------------------------------ a11 tail: sum the head slices of a group
+// ------------------------------------------------------------------ dB / dC: sum the head slices of a group
 template <typename T>
 __global__ void __launch_bounds__(256) k_reduce_dbdc(SegParams p) {
     pdl_launch_dependents();
@@ -720,7 +720,7 @@ cudaError_t launch_reduce_dbdc(const SegParams &p, int dtype, cudaStream_t st) {
     return launch_pdl(k_reduce_dbdc<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, p);
 }
 
-// ------------------------------------------------------------------ a13 tail: dA, dD over (batch, chunks)
+// ------------------------------------------------------------------ dA, dD over (batch, chunks)
 // One warp per head; lanes stride over the per-chunk partials in fp64, then a fixed shuffle tree.
 __global__ void __launch_bounds__(32) k_final_dAdD(SegParams p, float *dA, float *dD, int accumulate) {
     pdl_launch_dependents();

@@ -70,7 +70,7 @@ bool tc_make_maps(const SegParams &p, TcMaps &m) {
     return ok;
 }
 
-// ------------------------------------------------------------------ a2 / a8: chunk state on tensor cores
+// ------------------------------------------------------------------ chunk sums / state-gradient sums on tensor cores
 // One CTA per (chunk, head pair, batch): D[128 = (head-in-pair, p)][N] = sum_s Xw[s][(h2,p)] * V[s][n]
 //   mode FWD   : X = x,  V = Bm, w_s = exp(cs_last - cs_s) dt_s  -> Hst slot c+1   (S_c)
 //   mode DSTATE: X = dy, V = Cm, w_t = exp(cs_t)                 -> Gst slot c     (E_c)
@@ -80,7 +80,7 @@ bool tc_make_maps(const SegParams &p, TcMaps &m) {
 // ONE 64 KB stage (half a chunk) and two to three CTAs share an SM: one CTA's load overlaps the
 // others' scaling, MMAs and epilogue.
 //
-// Mode FWD also computes the chunk cumsum of dt*A (a1) for its two heads and leaves cs / dtT for the
+// Mode FWD also computes the chunk cumsum of dt*A for its two heads and leaves cs / dtT for the
 // later kernels of the segment.  Mode DSTATE also produces, per head, rho2_t = e^{cs_t} dy_t . (H_in C_t): the inter-chunk part of
 // C_t . dC_t that the decay gradient needs.  The C tile is already in shared memory (as rows of
 // time it is a K-major A operand), so it is one more product C (128 x N) * H_in^T (N x P) per head
@@ -135,7 +135,7 @@ k_chunk_state_tc(SegParams p, int mode, const __grid_constant__ CUtensorMap tmX,
     const uint32_t ncol_tmem = dstate ? 256u : 128u;   // E or S: 128 columns; Yoff of two heads: 128 more
     if (warp == 0) tmem_alloc(&tmem_base, ncol_tmem);
     if (!dstate) {
-        // a1 fused in: the chunk's cumulative sums of dt*A for the two heads (warp hh scans head hh: a
+        // the chunk cumsum, fused in: the chunk's cumulative sums of dt*A for the two heads (warp hh scans head hh: a
         // lane owns 8 consecutive steps, lane totals meet in a warp-shuffle scan), kept for every later
         // kernel of the segment in cs / dtT, and turned into the per-row weights right here.
         if (warp < 2) {

@@ -1,11 +1,11 @@
 // Tensor-core kernel for the two masked products whose score matrix is per head and whose result
 // is summed over the heads of a group (bf16 I/O, P = 64, N = 128, Q = 256):
 //
-//   GB_DC (a11): dC_t = sum_h [ sum_{s<=t} W_h[t,s] B_s + e^{cs_t} dy_t^T H_in ]              rows t
-//   GB_DB (a11): dB_s = sum_h [ sum_{t>=s} W_h[t,s] C_t + dt_s e^{cs_last-cs_s} x_s^T Gout ]  rows s
+//   GB_DC: dC_t = sum_h [ sum_{s<=t} W_h[t,s] B_s + e^{cs_t} dy_t^T H_in ]              rows t
+//   GB_DB: dB_s = sum_h [ sum_{t>=s} W_h[t,s] C_t + dt_s e^{cs_last-cs_s} x_s^T Gout ]  rows s
 //   with W_h[t,s] = (dy_t . x_s) e^{cs_t-cs_s} dt_s   (s <= t)
 //
-// and the per-head scalars the decay gradient needs (a12):
+// and the per-head scalars the decay gradient needs:
 //   rho_t = sum_s W_h[t,s] (C_t.B_s)  = C_t . (intra-chunk part of this head's dC_t)     (GB_DC)
 //   psi_s = sum_t W_h[t,s] (C_t.B_s)  = B_s . (intra-chunk part of this head's dB_s)     (GB_DB)
 // (Eq. 1 of the paper regrouped by chunks; cs = inclusive cumsum of dt*A inside the chunk.)

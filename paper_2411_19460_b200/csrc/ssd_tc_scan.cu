@@ -1,8 +1,8 @@
 // Tensor-core kernel for the two masked products whose score matrix is shared by the heads of a
 // group (bf16 I/O, P = 64, N = 128, Q = 256):
 //
-//   SC_FWD (a5+a6): y_t  = sum_{s<=t} (C_t.B_s) e^{cs_t-cs_s} dt_s x_s + e^{cs_t} C_t H_in + D x_t
-//   SC_DX  (a10)  : u_s  = sum_{t>=s} (B_s.C_t) e^{cs_t-cs_s} dy_t      + e^{cs_last-cs_s} B_s Gout
+//   SC_FWD: y_t  = sum_{s<=t} (C_t.B_s) e^{cs_t-cs_s} dt_s x_s + e^{cs_t} C_t H_in + D x_t
+//   SC_DX : u_s  = sum_{t>=s} (B_s.C_t) e^{cs_t-cs_s} dy_t      + e^{cs_last-cs_s} B_s Gout
 //                   dx_s = D dy_s + dt_s u_s ;  ddt_direct_s = x_s . u_s ;  dD partial = sum dy.x ;
 //                   psi2_s = dt_s e^{cs_last-cs_s} x_s . (Gout B_s)   (inter-chunk part of B_s . dB_s)
 //
