@@ -250,6 +250,17 @@ int ssd_gated_norm_bwd(long long rows, int D, int group, int dtype, const void *
                        void *stream);
 
 /*
+ * Self-test of the failure path of the bounded device-side waits (no counterpart in the paper).  Every wait of
+ * the kernels (on a TMA copy, on another warp) has a time limit; when one runs out the kernel sets the status word
+ * at the start of `ws` and runs to its normal end, and ssd_poll_status reports SSD_ETIMEOUT.  This call exercises
+ * exactly that on a barrier that nothing ever arrives on: one warp waits `limit_cycles` clock cycles (a few
+ * thousand is enough), gives up and returns.  Nothing else is in flight, so the context stays fully usable.
+ * `ws`: device memory, 256-byte aligned, at least 512 bytes (the status word, and at ws + 256 the cycles waited).
+ * After synchronising `stream`, ssd_poll_status(ws) must return SSD_ETIMEOUT.
+ */
+int ssd_selftest_wait_timeout(void *ws, size_t ws_bytes, long long limit_cycles, void *stream);
+
+/*
  * Reads the status word at the start of `ws` (device memory) with a blocking copy: call it after
  * synchronising the stream.  Returns SSD_OK, SSD_ETIMEOUT if some kernel abandoned a bounded wait
  * (its outputs are then undefined), or SSD_ECUDA if the copy failed.

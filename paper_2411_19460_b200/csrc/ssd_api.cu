@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "ssd_internal.h"
+#include "ssd_sm100.cuh"
 
 namespace ssd {
 
@@ -436,6 +437,24 @@ static int forward_impl(const ssd_shape_t *shape, const void *x, const float *dt
     return SSD_OK;
 }
 
+// ---- self-test of the bounded device-side wait: a barrier that nothing ever arrives on
+// One warp waits on it with the given limit, gives up, records that in the status word and returns normally: the
+// same mbar_wait path, status word and host read-back that every kernel of the library relies on, with no copy in
+// flight and no tensor memory held, so that giving up is harmless here.
+__global__ void k_selftest_wait(unsigned int *status, long long limit_clk, long long *waited_clk) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        sm100::mbar_init(&bar, 1);
+        abort_flag = 0;
+        sm100::fence_barrier_init();
+    }
+    __syncthreads();
+    const long long t0 = clock64();
+    const bool done = sm100::mbar_wait_limited(&bar, 0, &abort_flag, status, limit_clk);
+    if (threadIdx.x == 0 && waited_clk) *waited_clk = done ? -1 : clock64() - t0;
+}
+
 // ---- built-in scratch for ssd_fwd_static_ws (callers that cannot allocate) ----
 // Lives in the device image of this library: one copy per GPU that loads it, for the life of the
 // process.  In host code `g_static_ws` is only a handle for cudaGetSymbolAddress, never a pointer.
@@ -826,6 +845,18 @@ int ssd_gated_norm_bwd(long long rows, int D, int group, int dtype, const void *
     cudaStream_t st = (cudaStream_t)stream;
     SSD_LAUNCH(KIND_NORM, launch_gated_norm_bwd(dtype, y, z, gamma, eps, dout, dy, dz, dgamma, accumulate ? 1 : 0, (float *)ws,
                                                 rows, D, group, st));
+    return SSD_OK;
+}
+
+int ssd_selftest_wait_timeout(void *ws, size_t ws_bytes, long long limit_cycles, void *stream) {
+    if (!ws || limit_cycles < 0) return SSD_EINVAL;
+    if (((uintptr_t)ws & 255u) || ws_bytes < 512) return SSD_EWORKSPACE;
+    int rc = check_device();
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    SSD_TRY(cudaMemsetAsync(ws, 0, 512, st));
+    k_selftest_wait<<<1, 32, 0, st>>>((unsigned int *)ws, limit_cycles, (long long *)((char *)ws + 256));
+    SSD_TRY(cudaGetLastError());
     return SSD_OK;
 }
 

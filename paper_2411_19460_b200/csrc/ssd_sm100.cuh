@@ -54,13 +54,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 constexpr long long kWaitLimitClk = 4000000000ll;   // about 2 s at 2 GHz
 constexpr long long kWaitAbortedClk = 4000000ll;     // about 2 ms once aborted
 
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                          unsigned int *status) {
+// The wait with an explicit limit (clock cycles) for a wait that has not yet been given up on.
+__device__ __forceinline__ bool mbar_wait_limited(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                                  unsigned int *status, long long limit_clk) {
     if (mbar_try_wait(bar, parity)) return true;
     // Not complete yet: poll with a short sleep in between, so that the waiting warps of a CTA do not
     // flood the shared-memory pipe (every poll is a shared-memory access) that the MMAs read from.
     const long long start = clock64();
-    const long long limit = (*abort_flag) ? kWaitAbortedClk : kWaitLimitClk;
+    const long long limit = (*abort_flag) ? kWaitAbortedClk : limit_clk;
     uint32_t it = 0;
     while (true) {
         __nanosleep(20);
@@ -70,6 +71,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     *abort_flag = 1u;
     atomicExch(status, 1u);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                          unsigned int *status) {
+    return mbar_wait_limited(bar, parity, abort_flag, status, kWaitLimitClk);
 }
 
 // ---------------------------------------------------------------- fences

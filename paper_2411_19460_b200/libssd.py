@@ -27,7 +27,8 @@ EXPORTS = ["ssd_workspace_bytes", "ssd_boundary_bytes", "ssd_fwd", "ssd_fwd_segm
            "ssd_last_cuda_error", "ssd_launch_count", "ssd_kernel_kinds", "ssd_kernel_name",
            "ssd_profile", "ssd_profile_read", "ssd_fwd_static_ws", "ssd_glue_fwd", "ssd_glue_bwd",
            "ssd_glue_residual", "ssd_decode_step", "ssd_conv_fwd", "ssd_conv_bwd",
-           "ssd_conv_workspace_bytes", "ssd_gated_norm_fwd", "ssd_gated_norm_bwd", "ssd_gated_norm_workspace_bytes"]
+           "ssd_conv_workspace_bytes", "ssd_gated_norm_fwd", "ssd_gated_norm_bwd", "ssd_gated_norm_workspace_bytes",
+           "ssd_selftest_wait_timeout"]
 
 
 class SSDShape(ctypes.Structure):
@@ -94,6 +95,8 @@ def lib():
         L.ssd_glue_residual.argtypes = [sp, vp, vp, vp]
         L.ssd_poll_status.restype = ctypes.c_int
         L.ssd_poll_status.argtypes = [vp]
+        L.ssd_selftest_wait_timeout.restype = ctypes.c_int
+        L.ssd_selftest_wait_timeout.argtypes = [vp, ctypes.c_size_t, ctypes.c_longlong, vp]
         L.ssd_strerror.restype = ctypes.c_char_p
         L.ssd_strerror.argtypes = [ctypes.c_int]
         L.ssd_version.restype = ctypes.c_int
@@ -145,6 +148,15 @@ def alloc_workspace(shape, op, device):
 
 def poll_status(ws):
     return int(lib().ssd_poll_status(_ptr(ws)))
+
+
+def selftest_wait_timeout(ws, limit_cycles, stream=None):
+    """Makes one bounded device-side wait run out (a barrier nothing arrives on); see include/ssd.h."""
+    st = torch.cuda.current_stream() if stream is None else stream
+    rc = lib().ssd_selftest_wait_timeout(_ptr(ws), ws.numel() * ws.element_size(), int(limit_cycles),
+                                         ctypes.c_void_p(st.cuda_stream))
+    if rc:
+        raise SSDError(rc, "ssd_selftest_wait_timeout")
 
 
 def launch_count():

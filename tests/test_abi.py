@@ -86,3 +86,28 @@ def test_null_misaligned_and_small_workspace(L):
                                None, ok, big, None) == libssd.SSD_EINVAL
     assert b"workspace" in L.ssd_strerror(libssd.SSD_EWORKSPACE)
     assert L.ssd_poll_status(None) == libssd.SSD_EINVAL
+
+
+@pytest.mark.gpu
+def test_a_bounded_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
+    """The failure path of the device-side waits, made on purpose in the only harmless way: a barrier that nothing
+    arrives on, waited for a few thousand cycles by one warp with nothing else in flight.  The kernel must return by
+    itself, the status word must read SSD_ETIMEOUT, and an ordinary call afterwards must work and poll clean."""
+    import torch
+    from paper_2411_19460_b200.inputs import CONFIGS, make_inputs
+    ws = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    libssd.selftest_wait_timeout(ws, 5000)
+    torch.cuda.synchronize()
+    assert libssd.poll_status(ws) == libssd.SSD_ETIMEOUT
+    waited = int(ws[256:264].view(torch.int64).item())
+    assert 5000 < waited < 50_000_000, waited          # gave up after the limit, and soon after it
+    # the context is intact: a normal forward on the same stream, with its own scratch, runs and polls clean
+    cfg = CONFIGS[1].scaled(L=1024, H=4, seg=512)
+    inp = make_inputs(cfg, "cuda")
+    y, hf, bd = libssd.ssd_fwd_segmented(inp["x"], inp["dt"], inp["A"], inp["Bm"], inp["Cm"], inp["D"], inp["h0"],
+                                         chunk=cfg.chunk, seg=cfg.seg)
+    torch.cuda.synchronize()
+    assert torch.isfinite(y.float()).all()
+    libssd.selftest_wait_timeout(ws, 0)                 # limit 0: gives up at the first check
+    torch.cuda.synchronize()
+    assert libssd.poll_status(ws) == libssd.SSD_ETIMEOUT
