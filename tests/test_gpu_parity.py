@@ -154,6 +154,34 @@ def test_helper_streams_change_no_bit_and_respect_caller_stream(seg):
 
 
 @pytest.mark.gpu
+def test_two_caller_streams_from_one_thread_share_the_helper_streams():
+    """Two calls issued back to back by one host thread on two caller streams: the library's helper streams and
+    events belong to the (thread, device), so the second call's forks queue behind the first call's work on them.
+    That serialises the two calls against each other but must not mix them up: each result equals the result of
+    the same call made alone, bit for bit."""
+    cfg = small(B=1, L=2048, H=8, G=2, seg=256)           # eight segments: every helper stream and twin copy in use
+    inps = [make_inputs(cfg, "cuda", seed=s) for s in (21, 22)]
+    refs = [pu.run_gpu(cfg, i) for i in inps]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for st in streams:
+        st.wait_stream(torch.cuda.current_stream())
+    got = []
+    for i, st in zip(inps, streams):                       # no synchronisation between the two calls
+        with torch.cuda.stream(st):
+            y, hf, bd = libssd.ssd_fwd_segmented(i["x"], i["dt"], i["A"], i["Bm"], i["Cm"], i["D"], i["h0"],
+                                                 chunk=cfg.chunk, seg=cfg.seg, stream=st)
+            g = libssd.ssd_bwd_segmented(i["x"], i["dt"], i["A"], i["Bm"], i["Cm"], i["D"], bd, i["dy"], i["dh_final"],
+                                         chunk=cfg.chunk, seg=cfg.seg, stream=st)
+        got.append(dict(y=y, h_final=hf, boundary=bd, **g))
+    for st in streams:
+        st.synchronize()
+    for ref, out in zip(refs, got):
+        for k, v in out.items():
+            if v is not None:
+                assert torch.equal(v, ref[k]), k
+
+
+@pytest.mark.gpu
 @pytest.mark.parametrize("dtype", ["bf16", "fp32"])
 def test_skip_gradient_flag_adds_dy_to_dx(dtype):
     """SSD_FLAG_SKIP_GRAD: dx = (plain dx) + dy with one rounding; every other output unchanged."""
