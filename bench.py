@@ -473,18 +473,27 @@ def measure_layer(args, rep, dev, cfg, full=True):
     bound, fl_tok, by_tok = model[dom]
     tok_per_launch = tokens * prof_steps / max(dom_n, 1)
     avg_s = dom_ms * 1e-3 / max(dom_n, 1)
-    if bound == "tensor":
+    peak_kind = "HBM copy"
+    if bound == "tensor" and cfg.dtype != "bf16":
+        # the fp32 mode runs these contractions on the CUDA cores: plain-ALU bound, against the measured FFMA rate
+        bound = "alu"
+        achieved = fl_tok * tok_per_launch / avg_s / 1e12
+        peak = measure_ffma_tflops(dev)
+        unit = "TFLOP/s"
+        peak_kind = "fp32 FFMA (fp32 matrix product, TF32 off)"
+    elif bound == "tensor":
         achieved = fl_tok * tok_per_launch / avg_s / 1e12
         peak = peaks["bf16_tflops"]        # a launch timed by itself with CUDA events: the burst figure
         unit = "TFLOP/s"
+        peak_kind = "bf16 matmul, burst"
     else:
         achieved = by_tok * tok_per_launch / avg_s / 1e9
         peak = peaks["hbm_gbs"]
         unit = "GB/s"
-    roofline = dict(kernel=dom, bound="tensor" if bound == "tensor" else "hbm", achieved=achieved, peak=peak,
+    roofline = dict(kernel=dom, bound=bound if bound in ("tensor", "alu") else "hbm", achieved=achieved, peak=peak,
                     unit=unit, frac=achieved / peak, traffic=ncu_traffic(dom, tok_per_launch, H),
                     peak_source=peaks["source"],
-                    peak_kind="bf16 matmul, burst" if bound == "tensor" else "HBM copy",
+                    peak_kind=peak_kind,
                     avg_launch_us=avg_s * 1e6, launches=dom_n, share_of_device_time=dom_ms / total_prof)
     kinds = {k: dict(ms_per_step=v[0] / prof_steps, launches_per_step=v[1] / prof_steps,
                      share=v[0] / total_prof) for k, v in prof.items() if v[1]}

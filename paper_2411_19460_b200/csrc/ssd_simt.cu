@@ -675,46 +675,63 @@ cudaError_t launch_bwd_finish(const SegParams &p, cudaStream_t st) {
 }
 
 // ------------------------------------------------------------------ dB / dC: sum the head slices of a group
+// Four consecutive n per thread (16-byte loads of the fp32 partial slices, one 8- or 16-byte store): the kernel only
+// moves bytes.  The order of the additions per element is fixed: slices in order, a slice's first slot before its second.
+__device__ __forceinline__ void add4(float4 &a, const float4 &b) {
+    a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+}
+__device__ __forceinline__ void st4(float *p, const float4 &v) { *reinterpret_cast<float4 *>(p) = v; }
+__device__ __forceinline__ void st4(__nv_bfloat16 *p, const float4 &v) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<const unsigned int *>(&lo);
+    pk.y = *reinterpret_cast<const unsigned int *>(&hi);
+    *reinterpret_cast<uint2 *>(p) = pk;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) k_reduce_dbdc(SegParams p) {
     pdl_launch_dependents();
     pdl_wait();
-    const size_t total = (size_t)p.B * p.nc * p.Q * p.G * p.N;
+    const int N4 = p.N >> 2;
+    const size_t total = (size_t)p.B * p.nc * p.Q * p.G * N4;
     const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
     if (i >= total) return;
-    const int n = (int)(i % p.N);
-    size_t r = i / p.N;
+    const int n = (int)(i % N4) * 4;
+    size_t r = i / N4;
     const int g = (int)(r % p.G);
     r /= p.G;
     const size_t seglen = (size_t)p.nc * p.Q;
     const size_t tl = r % seglen;
     const int b = (int)(r / seglen);
     const size_t segcap = (size_t)p.ncs * p.Q;
-    const size_t src = ((((size_t)b * segcap + tl) * p.G + g) * p.nsl) * p.N + n;
-    float sB = 0.f, sC = 0.f;
+    float4 sB = make_float4(0.f, 0.f, 0.f, 0.f), sC = sB;
+    auto ld = [](const float *q) { return *reinterpret_cast<const float4 *>(q); };
     if (p.bc_fused) {
         // two slots per slice; the second exists only for dC rows of the upper half of a chunk and dB rows
         // of the lower half (the rows that two tiles of the causal triangle contribute to)
         const bool upper = ((tl % (size_t)p.Q) >= (size_t)(p.Q / 2));
         const size_t src2 = ((((size_t)b * segcap + tl) * p.G + g) * (2 * p.nsl)) * p.N + n;
         for (int s = 0; s < p.nsl; ++s) {
-            sB += p.pB[src2 + (size_t)(2 * s) * p.N];
-            if (!upper) sB += p.pB[src2 + (size_t)(2 * s + 1) * p.N];
-            sC += p.pC[src2 + (size_t)(2 * s) * p.N];
-            if (upper) sC += p.pC[src2 + (size_t)(2 * s + 1) * p.N];
+            add4(sB, ld(p.pB + src2 + (size_t)(2 * s) * p.N));
+            if (!upper) add4(sB, ld(p.pB + src2 + (size_t)(2 * s + 1) * p.N));
+            add4(sC, ld(p.pC + src2 + (size_t)(2 * s) * p.N));
+            if (upper) add4(sC, ld(p.pC + src2 + (size_t)(2 * s + 1) * p.N));
         }
-    } else
-    for (int s = 0; s < p.nsl; ++s) {
-        sB += p.pB[src + (size_t)s * p.N];
-        sC += p.pC[src + (size_t)s * p.N];
+    } else {
+        const size_t src = ((((size_t)b * segcap + tl) * p.G + g) * p.nsl) * p.N + n;
+        for (int s = 0; s < p.nsl; ++s) {
+            add4(sB, ld(p.pB + src + (size_t)s * p.N));
+            add4(sC, ld(p.pC + src + (size_t)s * p.N));
+        }
     }
     const size_t dst = (size_t)b * p.bc_bs + ((size_t)p.t0 + tl) * p.G * p.N + (size_t)g * p.N + n;
-    stf((T *)p.dB + dst, sB);
-    stf((T *)p.dC + dst, sC);
+    st4((T *)p.dB + dst, sB);
+    st4((T *)p.dC + dst, sC);
 }
 
 cudaError_t launch_reduce_dbdc(const SegParams &p, int dtype, cudaStream_t st) {
-    const size_t total = (size_t)p.B * p.nc * p.Q * p.G * p.N;
+    const size_t total = (size_t)p.B * p.nc * p.Q * p.G * (p.N / 4);
     const unsigned blocks = (unsigned)((total + 255) / 256);
     if (dtype == SSD_DTYPE_F32) return launch_pdl(k_reduce_dbdc<float>, dim3(blocks), dim3(256), 0, st, p);
     return launch_pdl(k_reduce_dbdc<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, p);
