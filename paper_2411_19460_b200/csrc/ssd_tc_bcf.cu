@@ -494,32 +494,43 @@ k_grad_bc_fused(SegParams p, const __grid_constant__ CUtensorMap tmX, const __gr
         __syncwarp();
         if (lane == 0) mbar_arrive(&wfull);
 
-        // ---- the CTA's partial slices of the group sums: [B, seg, G, 2 nsl, N] fp32
+        // ---- the CTA's partial slices of the group sums: [B, seg, G, 2 nsl, N] fp32.  Every row of an accumulator is
+        // 512 contiguous bytes of its slice.  Row-per-thread global stores would touch 32 different lines per
+        // instruction, so the two accumulators are staged in shared memory (every operand buffer is dead once the last
+        // products are done), rows padded to 528 bytes (conflict-free row-per-thread writes), and each row leaves as
+        // one bulk copy.
         mbar_wait(&accfull, 0, abortp, p.status);
         tc_fence_after_sync();
         {
-            const size_t segcap = (size_t)p.ncs * 256;
-            const int nsl2 = 2 * nsl;
+            float *stgC = reinterpret_cast<float *>(smem), *stgB = reinterpret_cast<float *>(smem + 128 * 528);
             float a[32];
-            // dC rows t: tiles (1,0) and (0,0) fill the even slot of their rows, (1,1) the odd slot of t-block 1
-            {
-                const size_t tl = (size_t)c * 256 + r;
-                const int slot = sl * 2 + (kind == 2 ? 1 : 0);
-                float *dst = p.pC + ((((size_t)b * segcap + tl) * p.G + g) * nsl2 + slot) * 128 + quar * 32;
-                tmem_ld32(tm + tlane + TF_ACCC + quar * 32, a);
+            tmem_ld32(tm + tlane + TF_ACCC + quar * 32, a);
 #pragma unroll
-                for (int k = 0; k < 32; k += 4)
-                    *reinterpret_cast<float4 *>(dst + k) = make_float4(a[k], a[k + 1], a[k + 2], a[k + 3]);
-            }
-            // dB rows s: tiles (0,0) and (1,1) fill the even slot of their rows, (1,0) the odd slot of s-block 0
-            {
-                const size_t tl = (size_t)c * 256 + rs;
-                const int slot = sl * 2 + (kind == 0 ? 1 : 0);
-                float *dst = p.pB + ((((size_t)b * segcap + tl) * p.G + g) * nsl2 + slot) * 128 + quar * 32;
-                tmem_ld32(tm + tlane + TF_ACCB + quar * 32, a);
+            for (int k = 0; k < 32; k += 4)
+                *reinterpret_cast<float4 *>(stgC + rl * 132 + quar * 32 + k) = make_float4(a[k], a[k + 1], a[k + 2], a[k + 3]);
+            tmem_ld32(tm + tlane + TF_ACCB + quar * 32, a);
 #pragma unroll
-                for (int k = 0; k < 32; k += 4)
-                    *reinterpret_cast<float4 *>(dst + k) = make_float4(a[k], a[k + 1], a[k + 2], a[k + 3]);
+            for (int k = 0; k < 32; k += 4)
+                *reinterpret_cast<float4 *>(stgB + rl * 132 + quar * 32 + k) = make_float4(a[k], a[k + 1], a[k + 2], a[k + 3]);
+            fence_proxy_async_smem();
+            asm volatile("bar.sync 1, 512;" ::: "memory");        // the sixteen mask warps
+            const int m = tid - 64;                               // 0..511 over the mask warps
+            if (m < 256) {
+                const size_t segcap = (size_t)p.ncs * 256;
+                const int nsl2 = 2 * nsl, row = m & 127;
+                if (m < 128) {
+                    // dC rows t: tiles (1,0) and (0,0) fill the even slot of their rows, (1,1) the odd slot of t-block 1
+                    const size_t tl = (size_t)c * 256 + tb * 128 + row;
+                    const int slot = sl * 2 + (kind == 2 ? 1 : 0);
+                    bulk_store(p.pC + ((((size_t)b * segcap + tl) * p.G + g) * nsl2 + slot) * 128, stgC + row * 132, 512);
+                } else {
+                    // dB rows s: tiles (0,0) and (1,1) fill the even slot of their rows, (1,0) the odd slot of s-block 0
+                    const size_t tl = (size_t)c * 256 + sb * 128 + row;
+                    const int slot = sl * 2 + (kind == 0 ? 1 : 0);
+                    bulk_store(p.pB + ((((size_t)b * segcap + tl) * p.G + g) * nsl2 + slot) * 128, stgB + row * 132, 512);
+                }
+                tma_store_commit();
+                tma_store_wait_all();
             }
         }
     }
