@@ -608,12 +608,16 @@ cudaError_t launch_masked_product_simt(const SegParams &p, int dtype, int mode, 
 // + exp(cs_last) <Gout, H_in>
 // (the CUDA-core kernels store rho = rho_intra + rho_inter as one vector and no rho2).  Suffix/prefix scans: serial inside a lane,
 // warp shuffles across lanes.  Then ddt = ddt_direct + A da, dA partial = sum_t dt_t da_t.
-__global__ void __launch_bounds__(128) k_bwd_finish(SegParams p) {
+// One CTA per (chunk, HB consecutive heads), one warp per head.  ddt is [B, L, H]: a head's values of consecutive
+// steps lie H floats apart, so the HB heads' results go through a shared-memory tile and leave as rows of HB
+// consecutive floats (whole 32-byte sectors for HB = 8) instead of one 4-byte store per sector.
+template <int HB>
+__global__ void __launch_bounds__(HB * 32) k_bwd_finish(SegParams p) {
     pdl_launch_dependents();
     pdl_wait();
+    __shared__ float tile[HB > 1 ? 256 * (HB + 1) : 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int c = blockIdx.x * 4 + warp, h = blockIdx.y, b = blockIdx.z;
-    if (c >= p.nc) return;
+    const int c = blockIdx.x, h = blockIdx.y * HB + warp, b = blockIdx.z;
     const int Q = p.Q, per = Q >> 5;
     const size_t vo = vec_off(p, b, h, c) + (size_t)lane * per;
     const int ngh = p.P * p.N / 1024;
@@ -662,16 +666,28 @@ __global__ void __launch_bounds__(128) k_bwd_finish(SegParams p) {
     for (int j = 0; j < 8; ++j)
         if (j < per) {
             const float da = ((sfx[j] + excl) + (pfx[j] + pexcl)) + gh;
-            p.ddt[(size_t)b * p.dt_bs + (tok0 + j) * p.H + h] = fmaf(Ah, da, dd[j]);
+            const float v = fmaf(Ah, da, dd[j]);
+            if (HB > 1) tile[(lane * per + j) * (HB + 1) + warp] = v;
+            else p.ddt[(size_t)b * p.dt_bs + (tok0 + j) * p.H + h] = v;
             sA = fmaf(dtv[j], da, sA);
         }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) sA += __shfl_xor_sync(0xffffffffu, sA, off);
     if (lane == 0) p.dAp[((size_t)b * p.H + h) * p.nct + p.c0 + c] = sA;
+    if (HB > 1) {
+        __syncthreads();
+        float *out = p.ddt + (size_t)b * p.dt_bs + ((size_t)p.t0 + (size_t)c * Q) * p.H + (size_t)blockIdx.y * HB;
+        for (int i = threadIdx.x; i < Q * HB; i += HB * 32) {
+            const int t = i / HB, hh = i % HB;
+            out[(size_t)t * p.H + hh] = tile[t * (HB + 1) + hh];
+        }
+    }
 }
 
 cudaError_t launch_bwd_finish(const SegParams &p, cudaStream_t st) {
-    return launch_pdl(k_bwd_finish, dim3((p.nc + 3) / 4, p.H, p.B), dim3(128), 0, st, p);
+    if (p.H % 8 == 0) return launch_pdl(k_bwd_finish<8>, dim3(p.nc, p.H / 8, p.B), dim3(256), 0, st, p);
+    if (p.H % 4 == 0) return launch_pdl(k_bwd_finish<4>, dim3(p.nc, p.H / 4, p.B), dim3(128), 0, st, p);
+    return launch_pdl(k_bwd_finish<1>, dim3(p.nc, p.H, p.B), dim3(32), 0, st, p);
 }
 
 // ------------------------------------------------------------------ dB / dC: sum the head slices of a group
