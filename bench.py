@@ -100,13 +100,13 @@ def load_peaks():
 # proportion).
 NCU_TRAFFIC = {
     # kernel kind: (bytes per launch, source file, sha256 of that file at capture time)
-    "bwd_dBdC": (140.2e6, "ssd_tc_bcf.cu", "86cbdbf8df5a575ff65e77851460b110f53d2ae5c0ef203bece4e8ba5cb8f8ee"),
-    "bwd_dx": (167.1e6, "ssd_tc_scan.cu", "c081e0c5aefb9cc29b488b38c92dc4a08cd5db9093f566821ba30a2f0cc9fb19"),
-    "chunk_scan_fwd": (89.2e6, "ssd_tc_scan.cu", "c081e0c5aefb9cc29b488b38c92dc4a08cd5db9093f566821ba30a2f0cc9fb19"),
-    "chunk_state": (47.9e6, "ssd_tc.cu", "476c275026f7e136b96cec13cc7c617ea7c59d6fc34edbe9bc79467efbc16aee"),
-    "dstate_contrib": (71.2e6, "ssd_tc.cu", "476c275026f7e136b96cec13cc7c617ea7c59d6fc34edbe9bc79467efbc16aee"),
-    "state_pass_fwd": (45.8e6, "ssd_simt.cu", "6b7a2088a97e108638c59fef85a74dbf4964aee0182467b5d29c4818906c881a"),
-    "state_pass_bwd": (68.9e6, "ssd_simt.cu", "6b7a2088a97e108638c59fef85a74dbf4964aee0182467b5d29c4818906c881a"),
+    "bwd_dBdC": (139.4e6, "ssd_tc_bcf.cu", "dea27dee76a18e163bad504ab1ea872d692421f290753dcb7e87928a10f9f10c"),
+    "bwd_dx": (165.8e6, "ssd_tc_scan.cu", "8456e62e2f5db54b7c0b95e493eead1031cbb85dbd1e34e93385165c68151b98"),
+    "chunk_scan_fwd": (89.2e6, "ssd_tc_scan.cu", "8456e62e2f5db54b7c0b95e493eead1031cbb85dbd1e34e93385165c68151b98"),
+    "chunk_state": (47.8e6, "ssd_tc.cu", "443a66c3f770fd0077e43b67055287dd8166d54e8c90b99a3bedc785227b7f08"),
+    "dstate_contrib": (70.9e6, "ssd_tc.cu", "443a66c3f770fd0077e43b67055287dd8166d54e8c90b99a3bedc785227b7f08"),
+    "state_pass_fwd": (45.4e6, "ssd_simt.cu", "701070c9421ce252f39d2b71218181c3ccaac7433187a73effa60c6cfa5de8f7"),
+    "state_pass_bwd": (68.4e6, "ssd_simt.cu", "701070c9421ce252f39d2b71218181c3ccaac7433187a73effa60c6cfa5de8f7"),
 }
 NCU_UNITS = 4096 * 80
 
