@@ -197,7 +197,7 @@ static void make_layout(const Plan &pl, int op, Layout &lo, bool twins) {
         lo.Gst = take(st * sizeof(float));
         lo.Gbf = take(pl.use_tc ? st * 2 : 0);
         lo.gcarry = take(BH * PN * sizeof(float));
-        lo.ghdot = take(BH * pl.ncs * 8 * sizeof(float));
+        lo.ghdot = take(BH * pl.ncs * 16 * sizeof(float));
         lo.ddt_dir = take(vec);
         lo.rho = take(vec);
         lo.rho2 = take(pl.use_tc ? vec : 0);
@@ -211,7 +211,7 @@ static void make_layout(const Plan &pl, int op, Layout &lo, bool twins) {
         lo.dDp = take(BH * pl.nct * 16 * sizeof(float));
         lo.Gbf_b = take(twin ? st * 2 : 0);
         lo.rho2_b = take(twin ? vec : 0);
-        lo.ghdot_b = take(twin ? BH * pl.ncs * 8 * sizeof(float) : 0);
+        lo.ghdot_b = take(twin ? BH * pl.ncs * 16 * sizeof(float) : 0);
         lo.rhob = take(pl.use_tc ? vec : 0);
         lo.psib = take(pl.use_tc ? vec : 0);
         lo.ddt_dir_b = take(twin ? vec : 0);

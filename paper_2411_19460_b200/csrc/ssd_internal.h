@@ -65,7 +65,7 @@ struct SegParams {
     __nv_bfloat16 *Gbf;    // [B,ncs+1,H,P,N] bf16 copy of Gst (tensor-core path)
     float *hcarry;         // [B,H,P,N]     state handed from segment to segment (forward)
     float *gcarry;         // [B,H,P,N]     state gradient handed right-to-left (backward)
-    float *ghdot;          // [B,H,ncs,8]   partial sums of exp(cs_last) <Gout_c, H_in,c>
+    float *ghdot;          // [B,H,ncs,16]  partial sums of exp(cs_last) <Gout_c, H_in,c>
     float *ddt_dir;        // [B,H,ncs,Q]   direct part of ddt
     float *rho;            // [B,H,ncs,Q]   C_t . dC_t of this head (CUDA-core path: all of it; tensor-core
                            //               path: its intra-chunk part)
