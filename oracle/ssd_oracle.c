@@ -1,7 +1,7 @@
 /*
  * TEST INFRASTRUCTURE — fp64 CPU oracle for the SSD selective-scan layer.
  *
- * This file is the slow, plain definition that the CUDA library is judged against.
+ * This file is the slow, plain definition that the CUDA library is checked against.
  * Only the test-suite, the smoke check and the bench's CPU-baseline leg may call it;
  * the product path never does.  It shares no code with the CUDA kernels.
  *
